@@ -1,0 +1,155 @@
+/*
+ * kda.h -- C ABI of the B200 (sm_100a) Kimi Delta Attention hot path.
+ *
+ * Two operations, both per sequence n and head h independently, with a dk x dv state S:
+ *
+ *   kda_chunk_fwd    chunkwise-parallel forward (prefill) of the recurrence
+ *                      S_t = (I - beta_t k_t k_t^T) Diag(alpha_t) S_{t-1} + beta_t k_t v_t^T
+ *                      o_t = scale * S_t^T q_t
+ *                    (Kimi Linear paper, Section 3, Eq. 1) evaluated with the chunkwise algorithm
+ *                    of Section 3.1: per-chunk cumulative log-decay, WY representation, UT
+ *                    transform, pseudo-values U - W S, output equation and chunk state update.
+ *   kda_decode_step  the same recurrence for ONE new token per sequence, state updated in place
+ *                    (Section 6.3 "Inference strategy": prefill uses the chunk kernel, generation
+ *                    the recurrent kernel).
+ *
+ * Conventions
+ *   - All tensors are dense, innermost dimension contiguous, token-major:
+ *       q, k, log_alpha : [total_tokens, H, dk]     v, o : [total_tokens, H, dv]
+ *       beta            : [total_tokens, H]         S0, S_T, S : [n, H, dk, dv]  (dv contiguous)
+ *   - alpha_t = exp(log_alpha_t), log_alpha <= 0 (a decay).  The cumulative log-decay inside one
+ *     64-token chunk must stay above -160 per channel; below that the intra-chunk products lose
+ *     accuracy (they never overflow: exponents are clamped).
+ *   - dt selects the storage type of q, k, v and o (fp32 or bf16).  Gates, beta and states are
+ *     always fp32.  dt = KDA_BF16 runs the contractions on bf16 tensor cores with fp32
+ *     accumulation; dt = KDA_F32 runs everything in fp32 FMA arithmetic.
+ *   - Supported shapes: dk = dv = 128, chunk = 64.  Anything else returns KDA_ERR_UNSUPPORTED;
+ *     there is no fallback path of any kind.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer, 16-byte aligned, owned by
+ *     the caller.  The library allocates no device memory: scratch comes from the caller's
+ *     workspace.  Calls are asynchronous and ordered on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the default stream); the caller keeps every buffer alive until the stream has
+ *     finished the call.
+ *   - Errors: every entry point returns a kda_status_t; nothing throws, aborts or traps.  Argument
+ *     errors are detected on the host before anything is launched.  kda_last_error() returns a
+ *     description of the calling thread's most recent failure.
+ */
+#ifndef KDA_H_
+#define KDA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KDA_OK = 0,
+    KDA_ERR_INVALID_ARG = 1, /* NULL/misaligned pointer, bad size, non-monotone cu_seqlens */
+    KDA_ERR_UNSUPPORTED = 2, /* shape or dtype outside the supported set */
+    KDA_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than the minimum */
+    KDA_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
+    KDA_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (reported by kda_check_status) */
+} kda_status_t;
+
+typedef enum { KDA_F32 = 0, KDA_BF16 = 1 } kda_dtype_t;
+
+/*
+ * Workspace size that lets kda_chunk_fwd process the whole call in one pass (all chunks of the
+ * intra-chunk stage in flight at once), capped at 8 GiB.  Any workspace of at least
+ * kda_chunk_fwd_min_workspace_bytes() works: a smaller one makes the call proceed in several
+ * passes over ranges of chunks with the state carried between them.  Both return 0 for an
+ * unsupported shape.
+ */
+size_t kda_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
+                                     int chunk, kda_dtype_t dt);
+size_t kda_chunk_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
+                                         int chunk, kda_dtype_t dt);
+
+/*
+ * Chunkwise forward (Section 3.1; pseudo-code in Appendix C).
+ *
+ *   q, k        [total_tokens,H,dk] dt      q may be NULL when o is NULL
+ *   v           [total_tokens,H,dv] dt
+ *   log_alpha   [total_tokens,H,dk] fp32    per-channel log decay of each token
+ *   beta        [total_tokens,H]    fp32
+ *   S0          [n_seqs,H,dk,dv]    fp32    initial states, or NULL = zeros
+ *   o           [total_tokens,H,dv] dt      output, or NULL = not produced (state-only mode)
+ *   S_T         [n_seqs,H,dk,dv]    fp32    state after each sequence's last token, or NULL
+ *   cu_seqlens_dev   [n_seqs+1] int32 device token offsets of a packed batch (cu[0] = 0,
+ *                    cu[n_seqs] = total_tokens, non-decreasing), or NULL = n_seqs sequences of
+ *                    equal length total_tokens / n_seqs
+ *   cu_seqlens_host  the same values in host memory (used for validation and scheduling); NULL
+ *                    exactly when cu_seqlens_dev is NULL
+ *   scale       multiplies q (the paper's pseudo-code uses dk^-0.5; pass 1 for pre-scaled q)
+ *   workspace   device scratch of workspace_bytes bytes, 256-byte aligned
+ *
+ * Chunks restart at every sequence start; a sequence whose length is not a multiple of 64 ends in
+ * a short chunk; a zero-length sequence yields S_T = S0 and no rows of o.  S0 and S_T may alias.
+ * Returns KDA_OK once all work is enqueued on the stream.
+ */
+kda_status_t kda_chunk_fwd(const void *q, const void *k, const void *v, const float *log_alpha,
+                           const float *beta, const float *S0, void *o, float *S_T,
+                           const int32_t *cu_seqlens_dev, const int32_t *cu_seqlens_host,
+                           int n_seqs, int64_t total_tokens, int H, int dk, int dv, int chunk,
+                           float scale, kda_dtype_t dt, void *workspace, size_t workspace_bytes,
+                           void *cuda_stream);
+
+/*
+ * Recurrent decode step (Eq. 1 for one token per sequence).
+ *
+ *   q, k, log_alpha  [n_seqs,H,dk]   v, o  [n_seqs,H,dv]   beta  [n_seqs,H]
+ *   S           [n_slots,H,dk,dv] fp32, read and written IN PLACE
+ *   state_slot  [n_seqs] int32 device: sequence n uses S[state_slot[n]]; NULL = identity.  Slots
+ *               must be distinct within a call and < n_slots (not checked on the device).
+ * Needs no workspace.
+ */
+kda_status_t kda_decode_step(const void *q, const void *k, const void *v, const float *log_alpha,
+                             const float *beta, float *S, const int32_t *state_slot, void *o,
+                             int n_seqs, int H, int dk, int dv, float scale, kda_dtype_t dt,
+                             void *cuda_stream);
+
+/*
+ * Host-buffer variants: same operations with q, k, v, log_alpha, beta, S0 (chunk) and o, S_T read
+ * from / written to HOST memory (pinned memory makes the copies asynchronous).  The device copies
+ * live in the caller's device workspace, so these allocate nothing either.  cu_seqlens is given on
+ * the host only.  For decode the states stay on the device (they are the resident cache);
+ * state_slot is a host array or NULL.  Copies and kernels are enqueued on `cuda_stream`; outputs
+ * are valid after the stream is synchronised.
+ */
+size_t kda_chunk_fwd_host_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
+                                          int chunk, kda_dtype_t dt);
+kda_status_t kda_chunk_fwd_host(const void *q_host, const void *k_host, const void *v_host,
+                                const float *log_alpha_host, const float *beta_host,
+                                const float *S0_host, void *o_host, float *S_T_host,
+                                const int32_t *cu_seqlens_host, int n_seqs, int64_t total_tokens,
+                                int H, int dk, int dv, int chunk, float scale, kda_dtype_t dt,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+size_t kda_decode_step_host_workspace_bytes(int n_seqs, int H, int dk, int dv, kda_dtype_t dt);
+kda_status_t kda_decode_step_host(const void *q_host, const void *k_host, const void *v_host,
+                                  const float *log_alpha_host, const float *beta_host,
+                                  float *S_dev, const int32_t *state_slot_host, void *o_host,
+                                  int n_seqs, int H, int dk, int dv, float scale, kda_dtype_t dt,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Reads back (synchronising the stream) the status word that device code sets when one of its
+ * bounded waits runs out, and clears it.  The word lives at the start of the workspace passed to
+ * kda_chunk_fwd.  Returns KDA_OK or KDA_ERR_TIMEOUT.
+ */
+kda_status_t kda_check_status(void *workspace, void *cuda_stream);
+
+/* Description of the calling thread's last error ("" if none); static storage, never NULL. */
+const char *kda_last_error(void);
+
+/* Number of kernel launches issued by this library in the calling process (for accounting). */
+uint64_t kda_launch_count(void);
+
+/* Library build tag, e.g. "kda-b200 sm_100a". */
+const char *kda_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KDA_H_ */

@@ -1,0 +1,161 @@
+/*
+ * KDA oracle: the token-by-token recurrence in fp64.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain definition that the CUDA library is checked against.  Only the
+ * tests, the smoke check and the CPU-baseline leg of the benchmark may build, load or call it; it
+ * shares no code, header, table or helper with the CUDA path and the product never routes through
+ * it.
+ *
+ * What it computes (Kimi Linear paper, Section 3, Eq. 1), per sequence n and head h independently,
+ * with S a dk x dv matrix:
+ *
+ *     S_t = (I - beta_t k_t k_t^T) Diag(alpha_t) S_{t-1} + beta_t k_t v_t^T ,   o_t = S_t^T q_t
+ *
+ * written out as: decay the rows of S by alpha_t = exp(log_alpha_t); form the residual
+ * r = v_t - S^T k_t against the *decayed* state; add the rank-one term beta_t k_t r^T; read the
+ * output from the *updated* state.  The chunkwise algorithm of Section 3.1 is an exact regrouping
+ * of this recurrence (Appendix B proves it), so this definition is the expected result of the
+ * chunk kernel as well as of the decode kernel.
+ *
+ * Inputs are float arrays holding the exact stored values (bf16 values widen exactly to float);
+ * every operation below is carried out in double.
+ *
+ * Layouts (d contiguous):  q,k,log_alpha [T_total,H,dk]  v,o [T_total,H,dv]  beta [T_total,H]
+ *                          S0,S_T [n_seqs,H,dk,dv]        cu_seqlens [n_seqs+1] (token offsets)
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* One token of Eq. 1 on one head's state S (dk x dv, row-major).  o may be NULL. */
+static void kda_token_step(double *S, const float *q, const float *k, const float *v,
+                           const float *log_alpha, double beta, double scale, int dk, int dv,
+                           double *r, double *o)
+{
+    /* Diag(alpha_t) S_{t-1}: row i of S is scaled by alpha_{t,i}. */
+    for (int i = 0; i < dk; ++i) {
+        double a = exp((double)log_alpha[i]);
+        double *Si = S + (size_t)i * dv;
+        for (int j = 0; j < dv; ++j) Si[j] *= a;
+    }
+    /* r = v_t - (decayed S)^T k_t */
+    for (int j = 0; j < dv; ++j) r[j] = (double)v[j];
+    for (int i = 0; i < dk; ++i) {
+        double ki = (double)k[i];
+        const double *Si = S + (size_t)i * dv;
+        for (int j = 0; j < dv; ++j) r[j] -= ki * Si[j];
+    }
+    /* S_t = decayed S + beta_t k_t r^T   ( = (I - beta k k^T) Diag(alpha) S + beta k v^T ) */
+    for (int i = 0; i < dk; ++i) {
+        double bk = beta * (double)k[i];
+        double *Si = S + (size_t)i * dv;
+        for (int j = 0; j < dv; ++j) Si[j] += bk * r[j];
+    }
+    /* o_t = scale * S_t^T q_t */
+    if (o) {
+        for (int j = 0; j < dv; ++j) o[j] = 0.0;
+        for (int i = 0; i < dk; ++i) {
+            double qi = (double)q[i];
+            const double *Si = S + (size_t)i * dv;
+            for (int j = 0; j < dv; ++j) o[j] += qi * Si[j];
+        }
+        for (int j = 0; j < dv; ++j) o[j] *= scale;
+    }
+}
+
+/*
+ * Whole sequences (Eq. 1 applied to every token in order).
+ *   S0   : initial states or NULL (= zeros)
+ *   o    : [T_total,H,dv] or NULL
+ *   S_T  : final states or NULL
+ *   cu_seqlens : n_seqs+1 token offsets, cu[0] = 0, non-decreasing
+ * Returns 0, or -1 on a bad argument / failed allocation.
+ */
+int kda_oracle_recurrence(const float *q, const float *k, const float *v, const float *log_alpha,
+                          const float *beta, const double *S0, double *o, double *S_T,
+                          const int64_t *cu_seqlens, int n_seqs, int H, int dk, int dv,
+                          double scale, int n_threads)
+{
+    if (!k || !v || !log_alpha || !beta || !cu_seqlens || n_seqs < 0 || H <= 0 || dk <= 0 || dv <= 0)
+        return -1;
+    if (o && !q) return -1;
+    int failed = 0;
+    long n_items = (long)n_seqs * H;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+    (void)n_threads;
+#endif
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long item = 0; item < n_items; ++item) {
+        int n = (int)(item / H), h = (int)(item % H);
+        double *S = (double *)malloc(sizeof(double) * dk * dv);
+        double *r = (double *)malloc(sizeof(double) * dv);
+        if (!S || !r) {
+            failed = 1;
+            free(S);
+            free(r);
+            continue;
+        }
+        size_t sofs = ((size_t)n * H + h) * dk * dv;
+        if (S0) memcpy(S, S0 + sofs, sizeof(double) * dk * dv);
+        else memset(S, 0, sizeof(double) * dk * dv);
+        for (int64_t t = cu_seqlens[n]; t < cu_seqlens[n + 1]; ++t) {
+            size_t th = (size_t)t * H + h;
+            kda_token_step(S, q ? q + th * dk : NULL, k + th * dk, v + th * dv,
+                           log_alpha + th * dk, (double)beta[th], scale, dk, dv, r,
+                           o ? o + th * dv : NULL);
+        }
+        if (S_T) memcpy(S_T + sofs, S, sizeof(double) * dk * dv);
+        free(S);
+        free(r);
+    }
+    return failed ? -1 : 0;
+}
+
+/*
+ * One decode step (the body of the recurrence once per sequence and head), state updated in place.
+ *   q,k,log_alpha [n_seqs,H,dk]   v,o [n_seqs,H,dv]   beta [n_seqs,H]
+ *   S [n_slots,H,dk,dv]; sequence n uses slot state_slot[n] (or n when state_slot is NULL)
+ */
+int kda_oracle_decode_step(const float *q, const float *k, const float *v, const float *log_alpha,
+                           const float *beta, double *S, const int32_t *state_slot, double *o,
+                           int n_seqs, int H, int dk, int dv, double scale, int n_threads)
+{
+    if (!q || !k || !v || !log_alpha || !beta || !S || !o || n_seqs < 0 || H <= 0) return -1;
+    int failed = 0;
+    long n_items = (long)n_seqs * H;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+    (void)n_threads;
+#endif
+#pragma omp parallel for schedule(static)
+    for (long item = 0; item < n_items; ++item) {
+        int n = (int)(item / H), h = (int)(item % H);
+        double *r = (double *)malloc(sizeof(double) * dv);
+        if (!r) {
+            failed = 1;
+            continue;
+        }
+        size_t th = (size_t)n * H + h;
+        size_t slot = state_slot ? (size_t)state_slot[n] : (size_t)n;
+        kda_token_step(S + (slot * H + h) * dk * dv, q + th * dk, k + th * dk, v + th * dv,
+                       log_alpha + th * dk, (double)beta[th], scale, dk, dv, r, o + th * dv);
+        free(r);
+    }
+    return failed ? -1 : 0;
+}
+
+int kda_oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

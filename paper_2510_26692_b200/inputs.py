@@ -1,0 +1,96 @@
+"""Seeded synthetic inputs shaped like the KDA workloads of the Kimi Linear paper.
+
+This module only draws random tensors; it holds none of the method's arithmetic and is the one
+module that both the CUDA-path tests/benchmark and the oracle-side tests may use.
+
+Recipe (the paper's parameterisation, Section 4 "Neural Parameterization"): q and k are
+L2-normalised per (token, head); q additionally carries the dk^-0.5 factor that the paper's
+chunkwise pseudo-code applies (Appendix C); v ~ N(0,1); the per-channel log-decay is
+logsigmoid(x) with x ~ N(gate_mean, 1); beta = sigmoid(N(0,1)); initial states ~ N(0, s0_std).
+Each tensor has its own generator (seed*16 + index, in the order q,k,v,x,beta,S0) so that a
+tensor's values do not depend on which other tensors are requested.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional, Sequence
+
+import torch
+
+_ORDER = {"q": 0, "k": 1, "v": 2, "x": 3, "beta": 4, "S0": 5, "S": 6, "lens": 7}
+
+
+def _gen(seed: int, name: str, device) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed) * 16 + _ORDER[name])
+    return g
+
+
+def _randn(shape, seed, name, device):
+    return torch.randn(*shape, generator=_gen(seed, name, device), device=device,
+                       dtype=torch.float32)
+
+
+def _l2norm(x: torch.Tensor) -> torch.Tensor:
+    return x * torch.rsqrt((x * x).sum(-1, keepdim=True) + 1e-6)
+
+
+def varlen_lengths(n_seqs: int, lo: int, hi: int, seed: int) -> list:
+    """Integer-uniform sequence lengths on [lo, hi] (inclusive), seeded."""
+    g = _gen(seed, "lens", "cpu")
+    return [int(x) for x in torch.randint(lo, hi + 1, (n_seqs,), generator=g)]
+
+
+def cu_seqlens_of(lengths: Sequence[int]) -> torch.Tensor:
+    cu = [0]
+    for n in lengths:
+        cu.append(cu[-1] + int(n))
+    return torch.tensor(cu, dtype=torch.int32)
+
+
+def chunk_inputs(lengths: Sequence[int], H: int, dk: int = 128, dv: int = 128,
+                 dtype: torch.dtype = torch.bfloat16, seed: int = 0, gate_mean: float = 4.0,
+                 s0_std: float = 0.0, scale_q: bool = True, device="cpu",
+                 want_q: bool = True) -> Dict[str, Optional[torch.Tensor]]:
+    """Inputs of one prefill call over ``len(lengths)`` packed sequences.
+
+    Returns q,k [T,H,dk] and v [T,H,dv] in ``dtype`` (rounded after scaling), log_alpha [T,H,dk]
+    and beta [T,H] in fp32, S0 [N,H,dk,dv] fp32 (None when s0_std == 0), cu_seqlens int32 [N+1].
+    """
+    T = int(sum(lengths))
+    N = len(lengths)
+    out: Dict[str, Optional[torch.Tensor]] = {}
+    if want_q:
+        q = _l2norm(_randn((T, H, dk), seed, "q", device))
+        if scale_q:
+            q = q * (dk ** -0.5)
+        out["q"] = q.to(dtype)
+        del q
+    else:
+        out["q"] = None
+    out["k"] = _l2norm(_randn((T, H, dk), seed, "k", device)).to(dtype)
+    out["v"] = _randn((T, H, dv), seed, "v", device).to(dtype)
+    x = _randn((T, H, dk), seed, "x", device)
+    x += gate_mean
+    out["log_alpha"] = torch.nn.functional.logsigmoid(x)
+    del x
+    out["beta"] = torch.sigmoid(_randn((T, H), seed, "beta", device))
+    out["S0"] = (_randn((N, H, dk, dv), seed, "S0", device) * s0_std) if s0_std > 0 else None
+    out["cu_seqlens"] = cu_seqlens_of(lengths)
+    return out
+
+
+def decode_inputs(n_seqs: int, H: int, steps: int, dk: int = 128, dv: int = 128,
+                  dtype: torch.dtype = torch.bfloat16, seed: int = 4, gate_mean: float = 4.0,
+                  s_std: float = 0.05, device="cpu") -> Dict[str, torch.Tensor]:
+    """Inputs of ``steps`` consecutive decode steps: q,k,log_alpha [steps,N,H,dk], v [steps,N,H,dv],
+    beta [steps,N,H], and the starting states S [N,H,dk,dv] fp32.  q and k are L2-normalised and q
+    carries no dk^-0.5 factor (the decode workload states none)."""
+    out = {}
+    out["q"] = _l2norm(_randn((steps, n_seqs, H, dk), seed, "q", device)).to(dtype)
+    out["k"] = _l2norm(_randn((steps, n_seqs, H, dk), seed, "k", device)).to(dtype)
+    out["v"] = _randn((steps, n_seqs, H, dv), seed, "v", device).to(dtype)
+    x = _randn((steps, n_seqs, H, dk), seed, "x", device) + gate_mean
+    out["log_alpha"] = torch.nn.functional.logsigmoid(x)
+    out["beta"] = torch.sigmoid(_randn((steps, n_seqs, H), seed, "beta", device))
+    out["S"] = _randn((n_seqs, H, dk, dv), seed, "S", device) * s_std
+    return out
