@@ -1,6 +1,14 @@
 """B200-native KDA (Kimi Delta Attention) hot path: chunkwise prefill and recurrent decode.
 
 The product is the CUDA library behind the C ABI declared in ``include/kda.h``; this package holds
-its sources (``csrc/``), the build step and a thin ctypes binding with the same entry-point names
-(``paper_2510_26692_b200.api``).  ``inputs`` draws the seeded synthetic workloads.
+its sources (``csrc/``), the build step (``build``) and a thin ctypes binding with the same
+entry-point names (``api``).  ``inputs`` draws the seeded synthetic workloads.  The library is
+loaded on first use and there is no fallback path: a missing ``libkda_b200.so`` raises.
 """
+from .api import (  # noqa: F401
+    KDA_BF16, KDA_F32, KdaError, kda_check_status, kda_chunk_fwd, kda_chunk_fwd_host,
+    kda_chunk_fwd_host_workspace_bytes, kda_chunk_fwd_min_workspace_bytes,
+    kda_chunk_fwd_workspace_bytes, kda_decode_step, kda_decode_step_host,
+    kda_decode_step_host_workspace_bytes, kda_last_error, kda_launch_count, kda_version,
+    library_path,
+)

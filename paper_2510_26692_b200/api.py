@@ -1,0 +1,208 @@
+"""ctypes binding of ``include/kda.h``: argument marshalling only.
+
+Every function has the name and argument order of its C entry point; tensors are ``torch`` tensors
+(used for device memory and streams only) whose ``data_ptr()`` is passed through.  Nothing is
+computed here, and there is no fallback: if ``libkda_b200.so`` is missing or does not load, the
+first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+KDA_F32 = 0
+KDA_BF16 = 1
+_STATUS = {0: "KDA_OK", 1: "KDA_ERR_INVALID_ARG", 2: "KDA_ERR_UNSUPPORTED", 3: "KDA_ERR_WORKSPACE",
+           4: "KDA_ERR_CUDA", 5: "KDA_ERR_TIMEOUT"}
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libkda_b200.so")
+_lib = None
+
+
+class KdaError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("%s: %s" % (_STATUS.get(code, str(code)), msg))
+        self.code = code
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load():
+    """Loads the CUDA library (built by ``paper_2510_26692_b200.build``); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError("libkda_b200.so not found at %s: run `python -m "
+                          "paper_2510_26692_b200.build` (needs nvcc); there is no fallback path"
+                          % _LIB_PATH)
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64, f32, sz = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float,
+                             ctypes.c_size_t)
+    lib.kda_chunk_fwd_workspace_bytes.restype = sz
+    lib.kda_chunk_fwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32, i32]
+    lib.kda_chunk_fwd_min_workspace_bytes.restype = sz
+    lib.kda_chunk_fwd_min_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32, i32]
+    lib.kda_chunk_fwd.restype = i32
+    lib.kda_chunk_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32,
+                                  i32, f32, i32, vp, sz, vp]
+    lib.kda_decode_step.restype = i32
+    lib.kda_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp]
+    lib.kda_chunk_fwd_host_workspace_bytes.restype = sz
+    lib.kda_chunk_fwd_host_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32, i32]
+    lib.kda_chunk_fwd_host.restype = i32
+    lib.kda_chunk_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32,
+                                       i32, f32, i32, vp, sz, vp]
+    lib.kda_decode_step_host_workspace_bytes.restype = sz
+    lib.kda_decode_step_host_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
+    lib.kda_decode_step_host.restype = i32
+    lib.kda_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f32,
+                                         i32, vp, sz, vp]
+    lib.kda_check_status.restype = i32
+    lib.kda_check_status.argtypes = [vp, vp]
+    lib.kda_last_error.restype = ctypes.c_char_p
+    lib.kda_launch_count.restype = ctypes.c_uint64
+    lib.kda_version.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def kda_last_error() -> str:
+    return load().kda_last_error().decode()
+
+
+def kda_launch_count() -> int:
+    return int(load().kda_launch_count())
+
+
+def kda_version() -> str:
+    return load().kda_version().decode()
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise KdaError(rc, kda_last_error())
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return KDA_BF16
+    if t.dtype == torch.float32:
+        return KDA_F32
+    raise TypeError("q/k/v/o must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _ptr(t: Optional[torch.Tensor], cuda: bool, dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor):
+        raise TypeError("%s must be a torch.Tensor" % name)
+    if t.is_cuda != cuda:
+        raise ValueError("%s must live on %s" % (name, "the GPU" if cuda else "the host"))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("%s must be %s, got %s" % (name, dtype, t.dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def kda_chunk_fwd_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64, dt=KDA_BF16):
+    return int(load().kda_chunk_fwd_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt))
+
+
+def kda_chunk_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64,
+                                      dt=KDA_BF16):
+    return int(load().kda_chunk_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt))
+
+
+def kda_chunk_fwd_host_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64,
+                                       dt=KDA_BF16):
+    return int(load().kda_chunk_fwd_host_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt))
+
+
+def kda_decode_step_host_workspace_bytes(n_seqs, H, dk=128, dv=128, dt=KDA_BF16):
+    return int(load().kda_decode_step_host_workspace_bytes(n_seqs, H, dk, dv, dt))
+
+
+def kda_chunk_fwd(q, k, v, log_alpha, beta, S0, o, S_T, cu_seqlens_dev, cu_seqlens_host, n_seqs,
+                  total_tokens, H, dk, dv, chunk, scale, dt, workspace, workspace_bytes=None,
+                  stream=None):
+    """``kda_chunk_fwd`` of ``include/kda.h``; device tensors, ``cu_seqlens_host`` a CPU int32
+    tensor.  Asynchronous on ``stream`` (default: torch's current stream)."""
+    f32 = torch.float32
+    et = torch.bfloat16 if dt == KDA_BF16 else torch.float32
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    rc = load().kda_chunk_fwd(
+        _ptr(q, True, et, "q"), _ptr(k, True, et, "k"), _ptr(v, True, et, "v"),
+        _ptr(log_alpha, True, f32, "log_alpha"), _ptr(beta, True, f32, "beta"),
+        _ptr(S0, True, f32, "S0"), _ptr(o, True, et, "o"), _ptr(S_T, True, f32, "S_T"),
+        _ptr(cu_seqlens_dev, True, torch.int32, "cu_seqlens_dev"),
+        _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
+        int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale), int(dt),
+        _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
+    _check(rc)
+
+
+def kda_decode_step(q, k, v, log_alpha, beta, S, state_slot, o, n_seqs, H, dk, dv, scale, dt,
+                    stream=None):
+    """``kda_decode_step`` of ``include/kda.h``; ``S`` is updated in place."""
+    f32 = torch.float32
+    et = torch.bfloat16 if dt == KDA_BF16 else torch.float32
+    rc = load().kda_decode_step(
+        _ptr(q, True, et, "q"), _ptr(k, True, et, "k"), _ptr(v, True, et, "v"),
+        _ptr(log_alpha, True, f32, "log_alpha"), _ptr(beta, True, f32, "beta"),
+        _ptr(S, True, f32, "S"), _ptr(state_slot, True, torch.int32, "state_slot"),
+        _ptr(o, True, et, "o"), int(n_seqs), int(H), int(dk), int(dv), float(scale), int(dt),
+        _stream(stream))
+    _check(rc)
+
+
+def kda_chunk_fwd_host(q, k, v, log_alpha, beta, S0, o, S_T, cu_seqlens_host, n_seqs, total_tokens,
+                       H, dk, dv, chunk, scale, dt, workspace, workspace_bytes=None, stream=None):
+    """``kda_chunk_fwd_host``: q..S_T are HOST tensors (pinned for asynchronous copies),
+    ``workspace`` a device tensor."""
+    f32 = torch.float32
+    et = torch.bfloat16 if dt == KDA_BF16 else torch.float32
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    rc = load().kda_chunk_fwd_host(
+        _ptr(q, False, et, "q"), _ptr(k, False, et, "k"), _ptr(v, False, et, "v"),
+        _ptr(log_alpha, False, f32, "log_alpha"), _ptr(beta, False, f32, "beta"),
+        _ptr(S0, False, f32, "S0"), _ptr(o, False, et, "o"), _ptr(S_T, False, f32, "S_T"),
+        _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
+        int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale), int(dt),
+        _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
+    _check(rc)
+
+
+def kda_decode_step_host(q, k, v, log_alpha, beta, S_dev, state_slot_host, o, n_seqs, H, dk, dv,
+                         scale, dt, workspace, workspace_bytes=None, stream=None):
+    """``kda_decode_step_host``: per-token inputs and ``o`` on the host, states on the device."""
+    f32 = torch.float32
+    et = torch.bfloat16 if dt == KDA_BF16 else torch.float32
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    rc = load().kda_decode_step_host(
+        _ptr(q, False, et, "q"), _ptr(k, False, et, "k"), _ptr(v, False, et, "v"),
+        _ptr(log_alpha, False, f32, "log_alpha"), _ptr(beta, False, f32, "beta"),
+        _ptr(S_dev, True, f32, "S"), _ptr(state_slot_host, False, torch.int32, "state_slot"),
+        _ptr(o, False, et, "o"), int(n_seqs), int(H), int(dk), int(dv), float(scale), int(dt),
+        _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
+    _check(rc)
+
+
+def kda_check_status(workspace, stream=None):
+    _check(load().kda_check_status(_ptr(workspace, True, None, "workspace"), _stream(stream)))

@@ -1,0 +1,365 @@
+// C ABI of the KDA library: argument validation, workspace carving, pass scheduling.  Every step
+// of the computation runs in the kernels of the other translation units; this file only decides
+// what to launch.
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "kda_common.cuh"
+
+namespace kda {
+
+static thread_local char g_err[512] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+kda_status_t fail(kda_status_t code, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr size_t kWorkspaceCap = (size_t)8 << 30;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t esize(kda_dtype_t dt) { return dt == KDA_BF16 ? 2 : 4; }
+
+bool shape_ok(int dk, int dv, int chunk, kda_dtype_t dt)
+{
+    return dk == kD && dv == kD && chunk == kC && (dt == KDA_F32 || dt == KDA_BF16);
+}
+
+size_t tile_bytes(kda_dtype_t dt)
+{
+    (void)dt;
+    return simt_tile_bytes();
+}
+
+struct WsLayout {
+    size_t off_table, off_state, off_tiles, fixed;
+};
+WsLayout ws_layout(int n_seqs, int H)
+{
+    WsLayout L;
+    L.off_table = sizeof(WsHeader);
+    L.off_state = L.off_table + align_up((size_t)(n_seqs + 1) * sizeof(int32_t));
+    L.off_tiles = L.off_state + align_up((size_t)n_seqs * H * kD * kD * sizeof(float));
+    L.fixed = L.off_tiles;
+    return L;
+}
+int64_t max_chunks(int64_t total_tokens, int n_seqs)
+{
+    return (total_tokens + kC - 1) / kC + n_seqs;
+}
+
+}  // namespace
+}  // namespace kda
+
+using namespace kda;
+
+extern "C" {
+
+const char* kda_last_error(void) { return g_err; }
+uint64_t kda_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+const char* kda_version(void) { return "kda-b200 sm_100a"; }
+
+size_t kda_chunk_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
+                                         int chunk, kda_dtype_t dt)
+{
+    if (!shape_ok(dk, dv, chunk, dt) || total_tokens < 0 || n_seqs < 0 || H <= 0) return 0;
+    return ws_layout(n_seqs, H).fixed + align_up((size_t)H * tile_bytes(dt));
+}
+
+size_t kda_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
+                                     int chunk, kda_dtype_t dt)
+{
+    if (!shape_ok(dk, dv, chunk, dt) || total_tokens < 0 || n_seqs < 0 || H <= 0) return 0;
+    const size_t fixed = ws_layout(n_seqs, H).fixed;
+    size_t want = fixed + align_up((size_t)max_chunks(total_tokens, n_seqs) * H * tile_bytes(dt));
+    const size_t lo = kda_chunk_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt);
+    if (want > kWorkspaceCap) want = kWorkspaceCap;
+    return want < lo ? lo : want;
+}
+
+kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const float* log_alpha,
+                           const float* beta, const float* S0, void* o, float* S_T,
+                           const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host,
+                           int n_seqs, int64_t total_tokens, int H, int dk, int dv, int chunk,
+                           float scale, kda_dtype_t dt, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream)
+{
+    if (!shape_ok(dk, dv, chunk, dt))
+        return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: only dk=dv=128, chunk=64, dt in {f32,bf16} "
+                    "are supported (got dk=%d dv=%d chunk=%d dt=%d)", dk, dv, chunk, (int)dt);
+    if (n_seqs < 0 || total_tokens < 0 || H <= 0 || H > 65535)
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: bad sizes n_seqs=%d total_tokens=%lld H=%d",
+                    n_seqs, (long long)total_tokens, H);
+    if ((cu_seqlens_dev == nullptr) != (cu_seqlens_host == nullptr))
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: cu_seqlens_dev and cu_seqlens_host must be "
+                    "given together");
+    if (n_seqs == 0) {
+        if (total_tokens != 0)
+            return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: n_seqs=0 with total_tokens=%lld",
+                        (long long)total_tokens);
+        return KDA_OK;
+    }
+    if (total_tokens > 0 && (!k || !v || !log_alpha || !beta))
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: k, v, log_alpha, beta must not be NULL");
+    if (o && total_tokens > 0 && !q)
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: q is NULL but o is requested");
+    const void* ptrs[] = {q, k, v, log_alpha, beta, S0, o, S_T, cu_seqlens_dev};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: pointer %p is not "
+                                       "16-byte aligned", p);
+    if (total_tokens * (int64_t)H > ((int64_t)1 << 40))
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: total_tokens*H too large");
+
+    // chunk table on the host (validation + scheduling)
+    std::vector<int64_t> chunk_cu((size_t)n_seqs + 1, 0);
+    int64_t seq_len = 0, chunks_per_seq = 0;
+    if (cu_seqlens_host) {
+        if (cu_seqlens_host[0] != 0 || (int64_t)cu_seqlens_host[n_seqs] != total_tokens)
+            return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: cu_seqlens must start at 0 and end at "
+                        "total_tokens");
+        for (int n = 0; n < n_seqs; ++n) {
+            const int64_t len = (int64_t)cu_seqlens_host[n + 1] - cu_seqlens_host[n];
+            if (len < 0) return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: cu_seqlens decreases at %d", n);
+            chunk_cu[n + 1] = chunk_cu[n] + (len + kC - 1) / kC;
+        }
+    } else {
+        if (total_tokens % n_seqs != 0)
+            return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: total_tokens not divisible by n_seqs "
+                        "for an equal-length batch");
+        seq_len = total_tokens / n_seqs;
+        chunks_per_seq = (seq_len + kC - 1) / kC;
+        for (int n = 0; n < n_seqs; ++n) chunk_cu[n + 1] = chunk_cu[n] + chunks_per_seq;
+    }
+    const int64_t total_chunks = chunk_cu[n_seqs];
+    if (total_chunks > 0x7fffffff)
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: too many chunks");
+
+    const WsLayout L = ws_layout(n_seqs, H);
+    const size_t tb = tile_bytes(dt);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) ||
+        workspace_bytes < L.fixed + (size_t)H * tb)
+        return fail(KDA_ERR_WORKSPACE, "kda_chunk_fwd: workspace must be 256-byte aligned and at "
+                    "least %zu bytes (got %zu)", L.fixed + (size_t)H * tb, workspace_bytes);
+    char* ws = static_cast<char*>(workspace);
+    int64_t cap = (int64_t)((workspace_bytes - L.fixed) / ((size_t)H * tb));
+    if (cap > 0x7fffffff) cap = 0x7fffffff;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
+    int32_t* chunk_cu_dev = reinterpret_cast<int32_t*>(ws + L.off_table);
+    kda_status_t rc = launch_prep(hdr, cu_seqlens_dev, chunk_cu_dev, n_seqs, st);
+    if (rc != KDA_OK) return rc;
+    if (!o && !S_T) return KDA_OK;   // nothing observable to produce
+
+    float* state = S_T ? S_T : reinterpret_cast<float*>(ws + L.off_state);
+    ChunkArgs a;
+    a.q = q; a.k = k; a.v = v; a.log_alpha = log_alpha; a.beta = beta;
+    a.o = o; a.cu_seqlens = cu_seqlens_dev; a.chunk_cu = cu_seqlens_dev ? chunk_cu_dev : nullptr;
+    a.n_seqs = n_seqs; a.H = H; a.total_tokens = total_tokens; a.seq_len = seq_len;
+    a.chunks_per_seq = chunks_per_seq; a.scale = scale;
+    a.S_out = state;
+
+    int64_t g0 = 0;
+    bool first = true;
+    do {
+        const int64_t g1 = (total_chunks - g0 > cap) ? g0 + cap : total_chunks;
+        a.g0 = g0; a.g1 = g1;
+        a.S_in = first ? S0 : state;
+        int n_begin = 0, n_count = n_seqs;
+        if (!first) {   // only the sequences that own a chunk of this pass
+            n_begin = 0;
+            while (n_begin < n_seqs && chunk_cu[n_begin + 1] <= g0) ++n_begin;
+            int n_end = n_begin;
+            while (n_end < n_seqs && chunk_cu[n_end] < g1) ++n_end;
+            n_count = n_end - n_begin;
+        }
+        rc = launch_chunk_simt(a, dt, ws + L.off_tiles, n_begin, n_count, st);
+        if (rc != KDA_OK) return rc;
+        g0 = g1;
+        first = false;
+    } while (g0 < total_chunks);
+    return KDA_OK;
+}
+
+kda_status_t kda_decode_step(const void* q, const void* k, const void* v, const float* log_alpha,
+                             const float* beta, float* S, const int32_t* state_slot, void* o,
+                             int n_seqs, int H, int dk, int dv, float scale, kda_dtype_t dt,
+                             void* cuda_stream)
+{
+    if (dk != kD || dv != kD || (dt != KDA_F32 && dt != KDA_BF16))
+        return fail(KDA_ERR_UNSUPPORTED, "kda_decode_step: only dk=dv=128, dt in {f32,bf16} are "
+                    "supported (got dk=%d dv=%d dt=%d)", dk, dv, (int)dt);
+    if (n_seqs < 0 || H <= 0 || (int64_t)n_seqs * H > 0x7fffffff)
+        return fail(KDA_ERR_INVALID_ARG, "kda_decode_step: bad sizes n_seqs=%d H=%d", n_seqs, H);
+    if (n_seqs == 0) return KDA_OK;
+    if (!q || !k || !v || !log_alpha || !beta || !S || !o)
+        return fail(KDA_ERR_INVALID_ARG, "kda_decode_step: NULL pointer argument");
+    const void* ptrs[] = {q, k, v, log_alpha, beta, S, o, state_slot};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return fail(KDA_ERR_INVALID_ARG, "kda_decode_step: pointer %p is not "
+                                       "16-byte aligned", p);
+    return launch_decode(q, k, v, log_alpha, beta, S, state_slot, o, n_seqs, H, scale, dt,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---- host-buffer variants -------------------------------------------------------------------------
+
+namespace {
+struct HostChunkLayout {
+    size_t q, k, v, g, b, s0, o, st, cu, inner, total;
+};
+HostChunkLayout host_chunk_layout(int64_t T, int n_seqs, int H, kda_dtype_t dt, size_t inner_bytes)
+{
+    HostChunkLayout L;
+    const size_t e = esize(dt), td = (size_t)T * H * kD;
+    size_t off = 0;
+    L.q = off; off += align_up(td * e);
+    L.k = off; off += align_up(td * e);
+    L.v = off; off += align_up(td * e);
+    L.g = off; off += align_up(td * 4);
+    L.b = off; off += align_up((size_t)T * H * 4);
+    L.s0 = off; off += align_up((size_t)n_seqs * H * kD * kD * 4);
+    L.o = off; off += align_up(td * e);
+    L.st = off; off += align_up((size_t)n_seqs * H * kD * kD * 4);
+    L.cu = off; off += align_up((size_t)(n_seqs + 1) * 4);
+    L.inner = off; off += inner_bytes;
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+size_t kda_chunk_fwd_host_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
+                                          int chunk, kda_dtype_t dt)
+{
+    const size_t inner = kda_chunk_fwd_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt);
+    if (inner == 0) return 0;
+    return host_chunk_layout(total_tokens, n_seqs, H, dt, inner).total;
+}
+
+kda_status_t kda_chunk_fwd_host(const void* q_host, const void* k_host, const void* v_host,
+                                const float* log_alpha_host, const float* beta_host,
+                                const float* S0_host, void* o_host, float* S_T_host,
+                                const int32_t* cu_seqlens_host, int n_seqs, int64_t total_tokens,
+                                int H, int dk, int dv, int chunk, float scale, kda_dtype_t dt,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!shape_ok(dk, dv, chunk, dt))
+        return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd_host: unsupported shape or dtype");
+    if (n_seqs < 0 || total_tokens < 0 || H <= 0)
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd_host: bad sizes");
+    const size_t inner_min =
+        kda_chunk_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt);
+    const HostChunkLayout L0 = host_chunk_layout(total_tokens, n_seqs, H, dt, 0);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) ||
+        workspace_bytes < L0.total + inner_min)
+        return fail(KDA_ERR_WORKSPACE, "kda_chunk_fwd_host: workspace must be 256-byte aligned and "
+                    "at least %zu bytes (got %zu)", L0.total + inner_min, workspace_bytes);
+    if (total_tokens > 0 && (!k_host || !v_host || !log_alpha_host || !beta_host))
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd_host: NULL input");
+    if (o_host && total_tokens > 0 && !q_host)
+        return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd_host: q is NULL but o is requested");
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    const size_t e = esize(dt), td = (size_t)total_tokens * H * kD;
+    const size_t sb = (size_t)n_seqs * H * kD * kD * 4;
+    if (q_host && td) KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.q, q_host, td * e, cudaMemcpyHostToDevice, st));
+    if (td) {
+        KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.k, k_host, td * e, cudaMemcpyHostToDevice, st));
+        KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.v, v_host, td * e, cudaMemcpyHostToDevice, st));
+        KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.g, log_alpha_host, td * 4, cudaMemcpyHostToDevice, st));
+        KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.b, beta_host, (size_t)total_tokens * H * 4,
+                                     cudaMemcpyHostToDevice, st));
+    }
+    if (S0_host && sb) KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.s0, S0_host, sb, cudaMemcpyHostToDevice, st));
+    if (cu_seqlens_host)
+        KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.cu, cu_seqlens_host, (size_t)(n_seqs + 1) * 4,
+                                     cudaMemcpyHostToDevice, st));
+    kda_status_t rc = kda_chunk_fwd(
+        q_host ? ws + L0.q : nullptr, ws + L0.k, ws + L0.v, reinterpret_cast<float*>(ws + L0.g),
+        reinterpret_cast<float*>(ws + L0.b), S0_host ? reinterpret_cast<float*>(ws + L0.s0) : nullptr,
+        o_host ? ws + L0.o : nullptr, S_T_host ? reinterpret_cast<float*>(ws + L0.st) : nullptr,
+        cu_seqlens_host ? reinterpret_cast<int32_t*>(ws + L0.cu) : nullptr, cu_seqlens_host, n_seqs,
+        total_tokens, H, dk, dv, chunk, scale, dt, ws + L0.inner, workspace_bytes - L0.inner, st);
+    if (rc != KDA_OK) return rc;
+    if (o_host && td) KDA_CUDA_TRY(cudaMemcpyAsync(o_host, ws + L0.o, td * e, cudaMemcpyDeviceToHost, st));
+    if (S_T_host && sb) KDA_CUDA_TRY(cudaMemcpyAsync(S_T_host, ws + L0.st, sb, cudaMemcpyDeviceToHost, st));
+    return KDA_OK;
+}
+
+size_t kda_decode_step_host_workspace_bytes(int n_seqs, int H, int dk, int dv, kda_dtype_t dt)
+{
+    if (dk != kD || dv != kD || n_seqs < 0 || H <= 0) return 0;
+    const size_t e = esize(dt), nd = (size_t)n_seqs * H * kD;
+    return 4 * align_up(nd * e) + align_up(nd * 4) + align_up((size_t)n_seqs * H * 4) +
+           align_up((size_t)n_seqs * 4) + kAlign;
+}
+
+kda_status_t kda_decode_step_host(const void* q_host, const void* k_host, const void* v_host,
+                                  const float* log_alpha_host, const float* beta_host,
+                                  float* S_dev, const int32_t* state_slot_host, void* o_host,
+                                  int n_seqs, int H, int dk, int dv, float scale, kda_dtype_t dt,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    const size_t need = kda_decode_step_host_workspace_bytes(n_seqs, H, dk, dv, dt);
+    if (need == 0) return fail(KDA_ERR_UNSUPPORTED, "kda_decode_step_host: unsupported shape");
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) || workspace_bytes < need)
+        return fail(KDA_ERR_WORKSPACE, "kda_decode_step_host: workspace must be 256-byte aligned and "
+                    "at least %zu bytes", need);
+    if (n_seqs == 0) return KDA_OK;
+    if (!q_host || !k_host || !v_host || !log_alpha_host || !beta_host || !S_dev || !o_host)
+        return fail(KDA_ERR_INVALID_ARG, "kda_decode_step_host: NULL pointer argument");
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    const size_t e = esize(dt), nd = (size_t)n_seqs * H * kD;
+    size_t off = 0;
+    char* dq = ws + off; off += align_up(nd * e);
+    char* dkk = ws + off; off += align_up(nd * e);
+    char* dvv = ws + off; off += align_up(nd * e);
+    char* dout = ws + off; off += align_up(nd * e);
+    char* dg = ws + off; off += align_up(nd * 4);
+    char* db = ws + off; off += align_up((size_t)n_seqs * H * 4);
+    char* ds = ws + off;
+    KDA_CUDA_TRY(cudaMemcpyAsync(dq, q_host, nd * e, cudaMemcpyHostToDevice, st));
+    KDA_CUDA_TRY(cudaMemcpyAsync(dkk, k_host, nd * e, cudaMemcpyHostToDevice, st));
+    KDA_CUDA_TRY(cudaMemcpyAsync(dvv, v_host, nd * e, cudaMemcpyHostToDevice, st));
+    KDA_CUDA_TRY(cudaMemcpyAsync(dg, log_alpha_host, nd * 4, cudaMemcpyHostToDevice, st));
+    KDA_CUDA_TRY(cudaMemcpyAsync(db, beta_host, (size_t)n_seqs * H * 4, cudaMemcpyHostToDevice, st));
+    if (state_slot_host)
+        KDA_CUDA_TRY(cudaMemcpyAsync(ds, state_slot_host, (size_t)n_seqs * 4, cudaMemcpyHostToDevice, st));
+    kda_status_t rc = kda_decode_step(dq, dkk, dvv, reinterpret_cast<float*>(dg),
+                                      reinterpret_cast<float*>(db), S_dev,
+                                      state_slot_host ? reinterpret_cast<int32_t*>(ds) : nullptr, dout,
+                                      n_seqs, H, dk, dv, scale, dt, st);
+    if (rc != KDA_OK) return rc;
+    KDA_CUDA_TRY(cudaMemcpyAsync(o_host, dout, nd * e, cudaMemcpyDeviceToHost, st));
+    return KDA_OK;
+}
+
+kda_status_t kda_check_status(void* workspace, void* cuda_stream)
+{
+    if (!workspace) return fail(KDA_ERR_INVALID_ARG, "kda_check_status: NULL workspace");
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    WsHeader h;
+    KDA_CUDA_TRY(cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, st));
+    KDA_CUDA_TRY(cudaStreamSynchronize(st));
+    if (h.status != 0) {
+        KDA_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st));
+        return fail((kda_status_t)h.status, "device code reported status %d at location %d",
+                    h.status, h.where);
+    }
+    return KDA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,129 @@
+// Internal helpers shared by the translation units of the KDA library (host side error plumbing,
+// launch accounting, workspace header layout, small device utilities).  Not part of the C ABI.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kda.h"
+
+namespace kda {
+
+constexpr int kD = 128;      // dk = dv (head size fixed by the paper's models)
+constexpr int kC = 64;       // chunk length (Section 3.1 uses C = 64)
+
+// ---- host-side plumbing (defined in kda_api.cu) -------------------------------------------------
+kda_status_t fail(kda_status_t code, const char* fmt, ...);
+void count_launch(int n = 1);
+#define KDA_CUDA_TRY(expr)                                                                   \
+    do {                                                                                     \
+        cudaError_t e__ = (expr);                                                            \
+        if (e__ != cudaSuccess)                                                              \
+            return ::kda::fail(KDA_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+
+// ---- workspace header ---------------------------------------------------------------------------
+// The first 256 bytes of the caller's workspace hold a status word (set by device code whose
+// bounded wait ran out); the chunk table follows.
+struct WsHeader {
+    int status;       // 0 = ok, otherwise a kda_status_t
+    int where;        // implementation-defined location code of the first failure
+    int pad[62];
+};
+static_assert(sizeof(WsHeader) == 256, "header is one 256-byte block");
+
+// Work description of one chunk-forward pass, passed by value to the kernels.
+struct ChunkArgs {
+    const void* q;
+    const void* k;
+    const void* v;
+    const float* log_alpha;
+    const float* beta;
+    const float* S_in;        // state entering this pass ([n_seqs,H,dk,dv]) or nullptr = zeros
+    float* S_out;             // state leaving this pass (may equal S_in), never nullptr
+    void* o;                  // or nullptr
+    const int32_t* cu_seqlens;  // device, or nullptr = equal lengths
+    const int32_t* chunk_cu;    // device [n_seqs+1]: first global chunk index of each sequence
+    int n_seqs;
+    int H;
+    int64_t total_tokens;
+    int64_t seq_len;          // equal-length case
+    int64_t chunks_per_seq;   // equal-length case
+    int64_t g0, g1;           // global chunk range of this pass
+    float scale;
+};
+
+// ---- dtype helpers ------------------------------------------------------------------------------
+template <typename T> struct IO;
+template <> struct IO<float> {
+    __device__ static __forceinline__ float4 load4(const float* p) {
+        return *reinterpret_cast<const float4*>(p);
+    }
+    __device__ static __forceinline__ void store4(float* p, float4 x) {
+        *reinterpret_cast<float4*>(p) = x;
+    }
+};
+template <> struct IO<__nv_bfloat16> {
+    __device__ static __forceinline__ float4 load4(const __nv_bfloat16* p) {
+        uint2 r = *reinterpret_cast<const uint2*>(p);
+        __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&r.x);
+        __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&r.y);
+        float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+        return make_float4(fa.x, fa.y, fb.x, fb.y);
+    }
+    __device__ static __forceinline__ void store4(__nv_bfloat16* p, float4 x) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(x.x, x.y), b = __floats2bfloat162_rn(x.z, x.w);
+        uint2 r;
+        r.x = *reinterpret_cast<uint32_t*>(&a);
+        r.y = *reinterpret_cast<uint32_t*>(&b);
+        *reinterpret_cast<uint2*>(p) = r;
+    }
+};
+
+// Locate global chunk g: sequence index, first token, number of valid tokens (1..64).
+struct ChunkLoc {
+    int n;
+    int64_t tok0;
+    int len;
+    int64_t c;   // chunk index inside the sequence
+};
+__device__ __forceinline__ ChunkLoc locate_chunk(const ChunkArgs& a, int64_t g) {
+    ChunkLoc L;
+    if (a.cu_seqlens == nullptr) {
+        L.n = (int)(g / a.chunks_per_seq);
+        L.c = g - (int64_t)L.n * a.chunks_per_seq;
+        int64_t t = L.c * kC;
+        L.tok0 = (int64_t)L.n * a.seq_len + t;
+        int64_t rem = a.seq_len - t;
+        L.len = rem < kC ? (int)rem : kC;
+    } else {
+        int lo = 0, hi = a.n_seqs - 1;   // last n with chunk_cu[n] <= g
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if ((int64_t)a.chunk_cu[mid] <= g) lo = mid; else hi = mid - 1;
+        }
+        L.n = lo;
+        L.c = g - a.chunk_cu[lo];
+        int64_t b = a.cu_seqlens[lo], e = a.cu_seqlens[lo + 1];
+        L.tok0 = b + L.c * kC;
+        int64_t rem = e - L.tok0;
+        L.len = rem < kC ? (int)rem : kC;
+    }
+    return L;
+}
+
+// ---- launchers implemented by the kernel translation units --------------------------------------
+kda_status_t launch_decode(const void* q, const void* k, const void* v, const float* log_alpha,
+                           const float* beta, float* S, const int32_t* slot, void* o, int n_seqs,
+                           int H, float scale, kda_dtype_t dt, cudaStream_t st);
+
+// fp32 FMA path (also accepts bf16 storage): per-tile scratch size and pass launcher
+size_t simt_tile_bytes();
+kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, int n_begin,
+                               int n_count, cudaStream_t st);
+
+// clears the status word and (packed batches) builds chunk_cu[n_seqs+1] from cu_seqlens
+kda_status_t launch_prep(WsHeader* hdr, const int32_t* cu_seqlens, int32_t* chunk_cu, int n_seqs,
+                         cudaStream_t st);
+
+}  // namespace kda

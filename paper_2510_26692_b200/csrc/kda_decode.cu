@@ -1,0 +1,128 @@
+// Recurrent decode step of KDA (paper Section 3, Eq. 1, one token per sequence and head):
+//     Sd = Diag(alpha) S;  r = v - Sd^T k;  S = Sd + beta k r^T;  o = scale S^T q
+// evaluated in ONE pass over the 128x128 fp32 state using the identity
+//     o = scale (Sd^T q + beta (q.k) r),
+// so that both column reductions (Sd^T k and Sd^T q) are taken while the state streams through
+// registers, and the state is written back exactly once.  HBM-bound: 64 KiB read + 64 KiB written
+// per (sequence, head).
+//
+// One CTA of 256 threads owns one state.  Thread (warp w, lane l) holds rows w, w+8, ... and the
+// four columns 4l..4l+3 of each: every warp-level access is one fully coalesced 512-byte row, and
+// all 16 loads of a thread are issued before the first use (64 KiB in flight per CTA).
+#include "kda_common.cuh"
+
+namespace kda {
+namespace {
+
+__device__ __forceinline__ float4 ld_stream(const float* p) {
+    float4 r;
+    asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
+                 : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st_stream(float* p, float4 x) {
+    asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(x.x),
+                 "f"(x.y), "f"(x.z), "f"(x.w)
+                 : "memory");
+}
+template <typename T> __device__ __forceinline__ float to_f(T x);
+template <> __device__ __forceinline__ float to_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 x) {
+    return __bfloat162float(x);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256, 2)
+kda_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                  const float* __restrict__ log_alpha, const float* __restrict__ beta, float* S,
+                  const int32_t* __restrict__ slot, T* __restrict__ o, int H, float scale)
+{
+    __shared__ float s_a[kD], s_k[kD], s_q[kD];
+    __shared__ float4 s_red[2][8][32];
+    const int item = blockIdx.x;
+    const int n = item / H, h = item - n * H;
+    const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
+    const size_t sl = slot ? (size_t)slot[n] : (size_t)n;
+    float* Sp = S + (sl * H + h) * (size_t)(kD * kD) + lane * 4;
+
+    float4 x[16];
+#pragma unroll
+    for (int m = 0; m < 16; ++m) x[m] = ld_stream(Sp + (size_t)(warp + 8 * m) * kD);
+
+    const size_t vec = (size_t)item * kD;
+    if (t < kD) {
+        s_a[t] = expf(log_alpha[vec + t]);
+        s_k[t] = to_f<T>(k[vec + t]);
+        s_q[t] = to_f<T>(q[vec + t]);
+    }
+    __syncthreads();
+
+    // q.k, redundantly per warp (4 rows per lane, butterfly reduce)
+    float qk = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) qk += s_q[lane * 4 + i] * s_k[lane * 4 + i];
+#pragma unroll
+    for (int ofs = 16; ofs > 0; ofs >>= 1) qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
+
+    float4 p = make_float4(0.f, 0.f, 0.f, 0.f), s = p;
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+        const int row = warp + 8 * m;
+        const float a = s_a[row], kk = s_k[row], qq = s_q[row];
+        x[m].x *= a; x[m].y *= a; x[m].z *= a; x[m].w *= a;
+        p.x += kk * x[m].x; p.y += kk * x[m].y; p.z += kk * x[m].z; p.w += kk * x[m].w;
+        s.x += qq * x[m].x; s.y += qq * x[m].y; s.z += qq * x[m].z; s.w += qq * x[m].w;
+    }
+    s_red[0][warp][lane] = p;
+    s_red[1][warp][lane] = s;
+    __syncthreads();
+    p = s_red[0][0][lane];
+    s = s_red[1][0][lane];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) {   // fixed order: bitwise reproducible
+        float4 a = s_red[0][w][lane], b = s_red[1][w][lane];
+        p.x += a.x; p.y += a.y; p.z += a.z; p.w += a.w;
+        s.x += b.x; s.y += b.y; s.z += b.z; s.w += b.w;
+    }
+    const float bt = beta[item];
+    float4 vv = IO<T>::load4(v + vec + lane * 4);
+    float4 r = make_float4(vv.x - p.x, vv.y - p.y, vv.z - p.z, vv.w - p.w);
+    if (warp == 0) {
+        const float c = bt * qk;
+        float4 ov = make_float4(scale * (s.x + c * r.x), scale * (s.y + c * r.y),
+                                scale * (s.z + c * r.z), scale * (s.w + c * r.w));
+        IO<T>::store4(o + vec + lane * 4, ov);
+    }
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+        const int row = warp + 8 * m;
+        const float c = bt * s_k[row];
+        x[m].x += c * r.x; x[m].y += c * r.y; x[m].z += c * r.z; x[m].w += c * r.w;
+        st_stream(Sp + (size_t)row * kD, x[m]);
+    }
+}
+
+}  // namespace
+
+kda_status_t launch_decode(const void* q, const void* k, const void* v, const float* log_alpha,
+                           const float* beta, float* S, const int32_t* slot, void* o, int n_seqs,
+                           int H, float scale, kda_dtype_t dt, cudaStream_t st)
+{
+    if (n_seqs == 0) return KDA_OK;
+    const unsigned grid = (unsigned)((size_t)n_seqs * H);
+    if (dt == KDA_BF16) {
+        using T = __nv_bfloat16;
+        kda_decode_kernel<T><<<grid, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v,
+                                                   log_alpha, beta, S, slot, (T*)o, H, scale);
+    } else {
+        kda_decode_kernel<float><<<grid, 256, 0, st>>>((const float*)q, (const float*)k,
+                                                       (const float*)v, log_alpha, beta, S, slot,
+                                                       (float*)o, H, scale);
+    }
+    count_launch();
+    KDA_CUDA_TRY(cudaGetLastError());
+    return KDA_OK;
+}
+
+}  // namespace kda

@@ -1,0 +1,230 @@
+"""Parity of the CUDA library (through its C ABI) with the fp64 oracle on the paper-shaped
+workloads.  Tolerances: max relative L2 error on o and on the final state, 1e-4 for the fp32 path
+and 2e-2 for bf16 storage."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2510_26692_b200 as K
+from paper_2510_26692_b200 import inputs
+from kda_testlib import TOL, check_chunk, oracle_chunk, rel_l2, run_chunk, to_np32
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config0_fp32(oracle_mod):
+    """fp32 path: B=1, T=256, H=2, S0 = 0, seed 0."""
+    d = inputs.chunk_inputs([256], H=2, dtype=torch.float32, seed=0)
+    errs = check_chunk(oracle_mod, d, TOL[K.KDA_F32])
+    print("config0", errs)
+
+
+def test_config1_bf16_prefill(oracle_mod):
+    """bf16 q/k/v: B=1, T=4096, H=32, S0 ~ N(0, 0.02)."""
+    d = inputs.chunk_inputs([4096], H=32, dtype=torch.bfloat16, seed=1, s0_std=0.02)
+    errs = check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
+    print("config1", errs)
+
+
+def test_config2_varlen(oracle_mod):
+    """16 packed sequences, lengths uniform on [512, 16384], per-sequence S0."""
+    lens = inputs.varlen_lengths(16, 512, 16384, seed=2)
+    d = inputs.chunk_inputs(lens, H=32, dtype=torch.bfloat16, seed=2, s0_std=0.02)
+    errs = check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
+    print("config2 lens", lens, "worst", max(errs.values()))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T", [1, 63, 64, 65, 127, 200])
+def test_ragged_lengths(oracle_mod, dtype, T):
+    d = inputs.chunk_inputs([T], H=3, dtype=dtype, seed=10 + T, s0_std=0.02)
+    check_chunk(oracle_mod, d, TOL[K.KDA_BF16 if dtype == torch.bfloat16 else K.KDA_F32])
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_varlen_edge_cases(oracle_mod, dtype):
+    """Short sequences (< C), a zero-length sequence (S_T = S0), lengths straddling chunk ends."""
+    lens = [5, 0, 64, 129, 1, 70]
+    d = inputs.chunk_inputs(lens, H=2, dtype=dtype, seed=21, s0_std=0.02)
+    tol = TOL[K.KDA_BF16 if dtype == torch.bfloat16 else K.KDA_F32]
+    check_chunk(oracle_mod, d, tol)
+    _, S_T = run_chunk(d)
+    assert torch.equal(S_T[1].cpu(), d["S0"][1])     # empty sequence: state passes through
+
+
+def test_s0_null_and_state_only(oracle_mod):
+    d = inputs.chunk_inputs([300], H=2, dtype=torch.bfloat16, seed=22)
+    assert d["S0"] is None
+    check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
+    # state-only mode: o = NULL, q = NULL
+    d2 = dict(d)
+    d2["q"] = None
+    _, S_only = run_chunk(d2, want_o=False)
+    _, S_full = run_chunk(d)
+    assert torch.equal(S_only, S_full)
+    # o only
+    o_only, none = run_chunk(d, want_state=False)
+    o_full, _ = run_chunk(d)
+    assert none is None and torch.equal(o_only, o_full)
+
+
+def test_small_workspace_multi_pass(oracle_mod):
+    """A workspace that holds only a few chunks forces several passes with the state carried
+    between them; results must not change."""
+    lens = [700, 130, 64, 900]
+    d = inputs.chunk_inputs(lens, H=2, dtype=torch.float32, seed=23, s0_std=0.02)
+    full = run_chunk(d)
+    N, T = len(lens), sum(lens)
+    lo = K.kda_chunk_fwd_min_workspace_bytes(T, N, 2, dt=K.KDA_F32)
+    hi = K.kda_chunk_fwd_workspace_bytes(T, N, 2, dt=K.KDA_F32)
+    for nbytes in (lo, lo + (hi - lo) // 7):
+        part = run_chunk(d, workspace_bytes=nbytes)
+        assert torch.equal(part[0], full[0]) and torch.equal(part[1], full[1])
+    check_chunk(oracle_mod, d, TOL[K.KDA_F32], workspace_bytes=lo)
+
+
+def test_scale_argument(oracle_mod):
+    d = inputs.chunk_inputs([130], H=2, dtype=torch.float32, seed=24, scale_q=False)
+    check_chunk(oracle_mod, d, TOL[K.KDA_F32], scale=128 ** -0.5)
+
+
+def test_resume_and_decode_continuation(oracle_mod):
+    """fwd(T1) then fwd(T2, S0 = S_T1) equals fwd(T1+T2); fwd(T) then one decode step equals the
+    recurrence on T+1 tokens."""
+    T1, T2, H = 150, 107, 2
+    d = inputs.chunk_inputs([T1 + T2 + 1], H=H, dtype=torch.float32, seed=25, s0_std=0.02)
+    cut = lambda a, b: {n: (t[a:b] if isinstance(t, torch.Tensor) and n not in ("S0", "cu_seqlens")
+                            else t) for n, t in d.items()}
+    da = cut(0, T1); da["cu_seqlens"] = inputs.cu_seqlens_of([T1])
+    oa, Sa = run_chunk(da)
+    db = cut(T1, T1 + T2); db["cu_seqlens"] = inputs.cu_seqlens_of([T2]); db["S0"] = Sa
+    ob, Sb = run_chunk(db)
+    dab = cut(0, T1 + T2); dab["cu_seqlens"] = inputs.cu_seqlens_of([T1 + T2])
+    oab, Sab = run_chunk(dab)
+    assert rel_l2(to_np32(torch.cat([oa, ob])), to_np32(oab)) < 1e-5
+    assert rel_l2(to_np32(Sb), to_np32(Sab)) < 1e-5
+    # one decode step on top of the prefill state
+    t = T1 + T2
+    dev = "cuda:0"
+    S = Sab.clone()
+    o1 = torch.empty((1, H, 128), dtype=torch.float32, device=dev)
+    K.kda_decode_step(d["q"][t:t + 1].to(dev), d["k"][t:t + 1].to(dev), d["v"][t:t + 1].to(dev),
+                      d["log_alpha"][t:t + 1].to(dev), d["beta"][t:t + 1].to(dev), S, None, o1,
+                      1, H, 128, 128, 1.0, K.KDA_F32)
+    torch.cuda.synchronize()
+    o_ref, S_ref = oracle_chunk(oracle_mod, d)
+    assert rel_l2(to_np32(o1[0]), o_ref[t]) < 1e-4
+    assert rel_l2(to_np32(S), S_ref) < 1e-4
+
+
+def test_run_to_run_bitwise(oracle_mod):
+    d = inputs.chunk_inputs([1000, 333], H=4, dtype=torch.bfloat16, seed=26, s0_std=0.02)
+    a = run_chunk(d)
+    b = run_chunk(d)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_harsh_gates(oracle_mod):
+    """Fast decay, logsigmoid(N(-1,1)): cumulative log-decay of a chunk reaches about -100."""
+    d = inputs.chunk_inputs([256], H=2, dtype=torch.float32, seed=27, gate_mean=-1.0, s0_std=0.02)
+    check_chunk(oracle_mod, d, TOL[K.KDA_F32])
+    d = inputs.chunk_inputs([256], H=2, dtype=torch.bfloat16, seed=27, gate_mean=-1.0, s0_std=0.02)
+    check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
+
+
+def test_beta_extremes(oracle_mod):
+    d = inputs.chunk_inputs([192], H=2, dtype=torch.float32, seed=28, s0_std=0.02)
+    for val in (0.0, 1.0):
+        d["beta"] = torch.full_like(d["beta"], val)
+        check_chunk(oracle_mod, d, TOL[K.KDA_F32])
+
+
+def test_config4_decode(oracle_mod):
+    """256 sequences x 32 heads, 64 consecutive in-place steps, bf16 q/k/v."""
+    N, H, steps = 256, 32, 64
+    d = inputs.decode_inputs(N, H, steps, seed=4)
+    dev = "cuda:0"
+    g = {n: t.to(dev) for n, t in d.items()}
+    S = g["S"].clone()
+    o = torch.empty((steps, N, H, 128), dtype=torch.bfloat16, device=dev)
+    for s in range(steps):
+        K.kda_decode_step(g["q"][s], g["k"][s], g["v"][s], g["log_alpha"][s], g["beta"][s], S,
+                          None, o[s], N, H, 128, 128, 1.0, K.KDA_BF16)
+    torch.cuda.synchronize()
+    S_ref = d["S"].double().numpy().copy()
+    worst = 0.0
+    for s in range(steps):
+        o_ref = oracle_mod.decode_step(to_np32(d["q"][s]), to_np32(d["k"][s]), to_np32(d["v"][s]),
+                                       to_np32(d["log_alpha"][s]), to_np32(d["beta"][s]), S_ref)
+        worst = max(worst, rel_l2(to_np32(o[s]), o_ref))
+    assert worst <= TOL[K.KDA_BF16], worst
+    assert rel_l2(to_np32(S), S_ref) <= TOL[K.KDA_BF16]
+    print("config4 worst o err", worst, "S err", rel_l2(to_np32(S), S_ref))
+
+
+def test_decode_fp32_and_slots(oracle_mod):
+    N, H = 7, 3
+    d = inputs.decode_inputs(N, H, 1, dtype=torch.float32, seed=31)
+    dev = "cuda:0"
+    slots = torch.tensor([9, 2, 5, 0, 7, 3, 8], dtype=torch.int32)
+    S = (torch.randn((10, H, 128, 128), generator=torch.Generator().manual_seed(5)) * 0.05)
+    Sg = S.to(dev)
+    o = torch.empty((N, H, 128), dtype=torch.float32, device=dev)
+    K.kda_decode_step(d["q"][0].to(dev), d["k"][0].to(dev), d["v"][0].to(dev),
+                      d["log_alpha"][0].to(dev), d["beta"][0].to(dev), Sg, slots.to(dev), o,
+                      N, H, 128, 128, 0.5, K.KDA_F32)
+    torch.cuda.synchronize()
+    S_ref = S.double().numpy().copy()
+    o_ref = oracle_mod.decode_step(to_np32(d["q"][0]), to_np32(d["k"][0]), to_np32(d["v"][0]),
+                                   to_np32(d["log_alpha"][0]), to_np32(d["beta"][0]), S_ref,
+                                   state_slot=slots.numpy(), scale=0.5)
+    assert rel_l2(to_np32(o), o_ref) < 1e-5
+    assert rel_l2(to_np32(Sg), S_ref) < 1e-6
+    untouched = [1, 4, 6]
+    assert torch.equal(Sg[untouched].cpu(), S[untouched])
+
+
+def test_host_buffer_entry_points(oracle_mod):
+    """The host-pointer variants give the same results as the device-pointer calls."""
+    lens = [100, 260]
+    d = inputs.chunk_inputs(lens, H=2, dtype=torch.bfloat16, seed=32, s0_std=0.02)
+    T, N, H = sum(lens), len(lens), 2
+    o_dev, S_dev = run_chunk(d)
+    pin = {n: (t.pin_memory() if isinstance(t, torch.Tensor) else t) for n, t in d.items()}
+    o_h = torch.empty_like(pin["v"]).pin_memory()
+    S_h = torch.empty((N, H, 128, 128), dtype=torch.float32).pin_memory()
+    nbytes = K.kda_chunk_fwd_host_workspace_bytes(T, N, H)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda:0")
+    K.kda_chunk_fwd_host(pin["q"], pin["k"], pin["v"], pin["log_alpha"], pin["beta"], pin["S0"],
+                         o_h, S_h, pin["cu_seqlens"], N, T, H, 128, 128, 64, 1.0, K.KDA_BF16, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(o_h, o_dev.cpu()) and torch.equal(S_h, S_dev.cpu())
+    # decode
+    dd = inputs.decode_inputs(5, 2, 1, seed=33)
+    S1 = dd["S"].to("cuda:0")
+    S2 = S1.clone()
+    o1 = torch.empty((5, 2, 128), dtype=torch.bfloat16, device="cuda:0")
+    K.kda_decode_step(dd["q"][0].cuda(), dd["k"][0].cuda(), dd["v"][0].cuda(),
+                      dd["log_alpha"][0].cuda(), dd["beta"][0].cuda(), S1, None, o1, 5, 2, 128,
+                      128, 1.0, K.KDA_BF16)
+    o2 = torch.empty((5, 2, 128), dtype=torch.bfloat16).pin_memory()
+    ws2 = torch.empty(K.kda_decode_step_host_workspace_bytes(5, 2), dtype=torch.uint8,
+                      device="cuda:0")
+    K.kda_decode_step_host(dd["q"][0].contiguous().pin_memory(), dd["k"][0].contiguous().pin_memory(),
+                           dd["v"][0].contiguous().pin_memory(),
+                           dd["log_alpha"][0].contiguous().pin_memory(),
+                           dd["beta"][0].contiguous().pin_memory(), S2, None, o2, 5, 2, 128, 128,
+                           1.0, K.KDA_BF16, ws2)
+    torch.cuda.synchronize()
+    assert torch.equal(o2, o1.cpu()) and torch.equal(S1, S2)
+
+
+def test_status_word_clean(oracle_mod):
+    d = inputs.chunk_inputs([128], H=2, dtype=torch.bfloat16, seed=34)
+    g = {n: (t.cuda() if isinstance(t, torch.Tensor) else t) for n, t in d.items()}
+    nbytes = K.kda_chunk_fwd_workspace_bytes(128, 1, 2)
+    ws = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda:0")
+    o = torch.empty_like(g["v"])
+    K.kda_chunk_fwd(g["q"], g["k"], g["v"], g["log_alpha"], g["beta"], None, o, None, None, None,
+                    1, 128, 2, 128, 128, 64, 1.0, K.KDA_BF16, ws)
+    K.kda_check_status(ws)   # raises KdaError on a device-side timeout
