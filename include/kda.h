@@ -140,6 +140,15 @@ kda_status_t kda_decode_step_host(const void *q_host, const void *k_host, const 
  */
 kda_status_t kda_check_status(void *workspace, void *cuda_stream);
 
+/*
+ * Optional per-kernel timing for benchmarks.  While enabled, every kernel launch of this library
+ * is bracketed by CUDA events on the launching stream (at most 8192 launches are recorded; enabling
+ * resets the record).  kda_profile_read synchronises the device and returns the summed duration and
+ * the launch count of one kernel kind: 0 = prologue, 1 = intra-chunk, 2 = inter-chunk, 3 = decode.
+ */
+void kda_profile_enable(int on);
+kda_status_t kda_profile_read(int kind, double *total_ms, int *launches);
+
 /* Description of the calling thread's last error ("" if none); static storage, never NULL. */
 const char *kda_last_error(void);
 

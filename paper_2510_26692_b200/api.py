@@ -66,6 +66,10 @@ def load():
                                          i32, vp, sz, vp]
     lib.kda_check_status.restype = i32
     lib.kda_check_status.argtypes = [vp, vp]
+    lib.kda_profile_enable.restype = None
+    lib.kda_profile_enable.argtypes = [i32]
+    lib.kda_profile_read.restype = i32
+    lib.kda_profile_read.argtypes = [i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
     lib.kda_last_error.restype = ctypes.c_char_p
     lib.kda_launch_count.restype = ctypes.c_uint64
     lib.kda_version.restype = ctypes.c_char_p
@@ -202,6 +206,18 @@ def kda_decode_step_host(q, k, v, log_alpha, beta, S_dev, state_slot_host, o, n_
         _ptr(o, False, et, "o"), int(n_seqs), int(H), int(dk), int(dv), float(scale), int(dt),
         _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
     _check(rc)
+
+
+def kda_profile_enable(on: bool):
+    load().kda_profile_enable(1 if on else 0)
+
+
+def kda_profile_read(kind: int):
+    """Returns (total_ms, launches) of one kernel kind (0 prologue, 1 intra, 2 inter, 3 decode)."""
+    ms = ctypes.c_double(0.0)
+    n = ctypes.c_int(0)
+    _check(load().kda_profile_read(int(kind), ctypes.byref(ms), ctypes.byref(n)))
+    return ms.value, n.value
 
 
 def kda_check_status(workspace, stream=None):

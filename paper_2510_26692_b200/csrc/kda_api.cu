@@ -5,6 +5,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "kda_common.cuh"
@@ -23,6 +24,39 @@ kda_status_t fail(kda_status_t code, const char* fmt, ...)
     return code;
 }
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// ---- per-kernel event timing ------------------------------------------------------------------------
+namespace {
+constexpr int kProfMax = 8192;
+struct ProfState {
+    std::mutex mu;
+    bool on = false;
+    int used = 0;
+    std::vector<cudaEvent_t> ev0, ev1;
+    std::vector<int> kind;
+} g_prof;
+}  // namespace
+
+ProfScope::ProfScope(int kind, cudaStream_t s) : slot(-1), st(s)
+{
+    if (!g_prof.on) return;
+    std::lock_guard<std::mutex> lk(g_prof.mu);
+    if (g_prof.used >= kProfMax) return;
+    if ((int)g_prof.ev0.size() <= g_prof.used) {
+        cudaEvent_t a, b;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+        g_prof.ev0.push_back(a);
+        g_prof.ev1.push_back(b);
+        g_prof.kind.push_back(0);
+    }
+    slot = g_prof.used++;
+    g_prof.kind[slot] = kind;
+    cudaEventRecord(g_prof.ev0[slot], st);
+}
+ProfScope::~ProfScope()
+{
+    if (slot >= 0) cudaEventRecord(g_prof.ev1[slot], st);
+}
 
 namespace {
 
@@ -344,6 +378,33 @@ kda_status_t kda_decode_step_host(const void* q_host, const void* k_host, const 
                                       n_seqs, H, dk, dv, scale, dt, st);
     if (rc != KDA_OK) return rc;
     KDA_CUDA_TRY(cudaMemcpyAsync(o_host, dout, nd * e, cudaMemcpyDeviceToHost, st));
+    return KDA_OK;
+}
+
+void kda_profile_enable(int on)
+{
+    std::lock_guard<std::mutex> lk(g_prof.mu);
+    g_prof.on = on != 0;
+    g_prof.used = 0;
+}
+
+kda_status_t kda_profile_read(int kind, double* total_ms, int* launches)
+{
+    if (kind < 0 || kind >= PROF_KINDS || !total_ms || !launches)
+        return fail(KDA_ERR_INVALID_ARG, "kda_profile_read: bad argument");
+    KDA_CUDA_TRY(cudaDeviceSynchronize());
+    std::lock_guard<std::mutex> lk(g_prof.mu);
+    double sum = 0.0;
+    int cnt = 0;
+    for (int i = 0; i < g_prof.used; ++i) {
+        if (g_prof.kind[i] != kind) continue;
+        float ms = 0.f;
+        KDA_CUDA_TRY(cudaEventElapsedTime(&ms, g_prof.ev0[i], g_prof.ev1[i]));
+        sum += ms;
+        ++cnt;
+    }
+    *total_ms = sum;
+    *launches = cnt;
     return KDA_OK;
 }
 

@@ -339,12 +339,14 @@ kda_status_t launch_simt_t(const ChunkArgs& a, float* tiles, int n_begin, int n_
     const int64_t n_chunks = a.g1 - a.g0;
     if (n_chunks > 0) {
         dim3 grid((unsigned)n_chunks, (unsigned)a.H);
+        ProfScope ps(PROF_INTRA, st);
         kda_intra_simt<T><<<grid, 256, kIntraSmem, st>>>(a, tiles);
         count_launch();
         KDA_CUDA_TRY(cudaGetLastError());
     }
     if (n_count > 0) {
         dim3 grid(kD / NS, (unsigned)a.H, (unsigned)n_count);
+        ProfScope ps(PROF_INTER, st);
         kda_inter_simt<T><<<grid, 256, kInterSmem, st>>>(a, tiles, n_begin);
         count_launch();
         KDA_CUDA_TRY(cudaGetLastError());
@@ -366,6 +368,7 @@ kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, 
 kda_status_t launch_prep(WsHeader* hdr, const int32_t* cu_seqlens, int32_t* chunk_cu, int n_seqs,
                          cudaStream_t st)
 {
+    ProfScope ps(PROF_PREP, st);
     kda_prep_kernel<<<1, 32, 0, st>>>(hdr, cu_seqlens, chunk_cu, n_seqs);
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());

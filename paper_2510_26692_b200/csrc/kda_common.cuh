@@ -22,6 +22,16 @@ void count_launch(int n = 1);
             return ::kda::fail(KDA_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
     } while (0)
 
+// Optional per-kernel timing (kda_profile_*): when enabled, every launch site is bracketed by a pair
+// of CUDA events on the launching stream.  A no-op when disabled.
+enum ProfKind { PROF_PREP = 0, PROF_INTRA = 1, PROF_INTER = 2, PROF_DECODE = 3, PROF_KINDS = 8 };
+struct ProfScope {
+    ProfScope(int kind, cudaStream_t st);
+    ~ProfScope();
+    int slot;
+    cudaStream_t st;
+};
+
 // ---- workspace header ---------------------------------------------------------------------------
 // The first 256 bytes of the caller's workspace hold a status word (set by device code whose
 // bounded wait ran out); the chunk table follows.

@@ -111,6 +111,7 @@ kda_status_t launch_decode(const void* q, const void* k, const void* v, const fl
 {
     if (n_seqs == 0) return KDA_OK;
     const unsigned grid = (unsigned)((size_t)n_seqs * H);
+    ProfScope ps(PROF_DECODE, st);
     if (dt == KDA_BF16) {
         using T = __nv_bfloat16;
         kda_decode_kernel<T><<<grid, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v,
