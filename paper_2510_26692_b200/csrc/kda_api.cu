@@ -73,8 +73,7 @@ bool shape_ok(int dk, int dv, int chunk, kda_dtype_t dt)
 
 size_t tile_bytes(kda_dtype_t dt)
 {
-    (void)dt;
-    return simt_tile_bytes();
+    return dt == KDA_BF16 ? tc_tile_bytes() : simt_tile_bytes();
 }
 
 struct WsLayout {
@@ -219,7 +218,10 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
             while (n_end < n_seqs && chunk_cu[n_end] < g1) ++n_end;
             n_count = n_end - n_begin;
         }
-        rc = launch_chunk_simt(a, dt, ws + L.off_tiles, n_begin, n_count, st);
+        if (dt == KDA_BF16)
+            rc = launch_chunk_tc(a, ws + L.off_tiles, n_begin, n_count, hdr, st);
+        else
+            rc = launch_chunk_simt(a, dt, ws + L.off_tiles, n_begin, n_count, st);
         if (rc != KDA_OK) return rc;
         g0 = g1;
         first = false;

@@ -1,0 +1,26 @@
+// Layout of the per-(chunk, head) scratch tile that the intra-chunk stage hands to the inter-chunk
+// stage on the bf16 tensor-core path.  Every matrix operand is stored as the exact shared-memory
+// image the tcgen05 MMA expects (K-major, 128-byte swizzle, see ptx::sw128_off), so the consumer
+// brings it in with plain 1-D bulk copies.
+#pragma once
+#include <stdint.h>
+
+namespace kda {
+namespace tc {
+// A operand of  [ (Gamma.Q) ; W ] S : two K-halves of [128 rows][64], rows 0-63 = scale*Gamma.Q,
+// rows 64-127 = W
+constexpr uint32_t OFF_QW = 0;
+constexpr uint32_t QW_HALF = 128 * 128;
+// A operand of the state update: ((gamma^C/Gamma).K)^T as [128 dk][64 tokens]
+constexpr uint32_t OFF_KT = 32768;
+// A operand of the intra-chunk output term: Aqk [64][64] (lower triangular incl. diagonal)
+constexpr uint32_t OFF_AQ = 49152;
+// U in four column blocks of [32 columns][64 tokens] bf16 (token index contiguous)
+constexpr uint32_t OFF_U = 57344;
+constexpr uint32_t U_BLOCK = 32 * 64 * 2;
+// gamma^C: 128 fp32
+constexpr uint32_t OFF_GC = 73728;
+constexpr uint32_t TILE_BYTES = 74240;
+static_assert(TILE_BYTES % 256 == 0, "tiles stay 256-byte aligned");
+}  // namespace tc
+}  // namespace kda
