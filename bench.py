@@ -145,6 +145,30 @@ def oracle_arm(args, rank):
     return 0
 
 
+def decode_only(args, K, inputs, torch, dev, peaks):
+    """Short decode-only run (used under a profiler): one block of 64 in-place steps, timed."""
+    dd = inputs.decode_inputs(DEC_SEQS, H, DEC_STEPS, seed=4)
+    gd = {n: t.to(dev) for n, t in dd.items()}
+    S = gd["S"].clone()
+    od = torch.empty((DEC_STEPS, DEC_SEQS, H, D), dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for rep in range(2):
+        if rep == 1:
+            e0.record(stream)
+        for s in range(DEC_STEPS):
+            K.kda_decode_step(gd["q"][s], gd["k"][s], gd["v"][s], gd["log_alpha"][s], gd["beta"][s],
+                              S, None, od[s], DEC_SEQS, H, D, D, 1.0, K.KDA_BF16, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / DEC_STEPS
+    gbs = DEC_SEQS * H * DEC_BYTES_PER_STATE / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "KDA decode tokens/s", "value": DEC_SEQS / (ms * 1e-3),
+                      "ms_per_step": ms, "achieved_gbs": gbs, "frac": gbs / peaks["hbm_gbs"],
+                      "partial": "decode-only"}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -153,6 +177,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-reps", type=int, default=5)
+    ap.add_argument("--prefill-only", action="store_true",
+                    help="time only the device-resident prefill loop (short runs under a profiler)")
+    ap.add_argument("--decode-only", action="store_true",
+                    help="time only the decode loop (short runs under a profiler)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -187,6 +215,9 @@ def main():
         t = torch.tensor([x], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
+
+    if args.decode_only:
+        return decode_only(args, K, inputs, torch, dev, peaks)
 
     # ---- prefill workload: 3 input copies (each 206 MB > L2) rotated between steps ---------------
     n_copies = 3
@@ -249,6 +280,15 @@ def main():
         "hbm_bound_tokens_per_s": peaks["hbm_gbs"] * 1e9 / (step_bytes / T_PREFILL),
         "note": "HBM is the slower bound at d=128, C=64; the tensor-pipe bound is above it",
     }
+
+    if args.prefill_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": tokens_per_s, "unit": "tokens/s",
+                              "ms_per_step": ms_step, "steps": args.steps, "warmup": args.warmup,
+                              "gpu_launches": launches, "kernels": kern, "partial": "prefill-only"}))
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
 
     # ---- end to end through the host-buffer entry point -------------------------------------------
     g0 = copies[0]

@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __re
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
                     st_bf16(tct + tc::OFF_U + ((c + e) >> 5) * tc::U_BLOCK +
-                                (((c + e) & 31) * 64 + i) * 2, uu[e]);
+                                (i * 32 + ((c + e) & 31)) * 2, uu[e]);
             } else {
                 *reinterpret_cast<float4*>(tile + T_W + i * kD + c) = w[m];
                 *reinterpret_cast<float4*>(tile + T_U + i * kD + c) = u[m];

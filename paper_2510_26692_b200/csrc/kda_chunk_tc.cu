@@ -17,6 +17,8 @@
 // kind::f16) issued by one thread, accumulators in TMEM, read back with tcgen05.ld.
 // Every wait is bounded: on a timeout the CTA records KDA_ERR_TIMEOUT in the workspace header,
 // drains its copies, frees its TMEM and returns.
+#include <cstdlib>
+
 #include "kda_common.cuh"
 #include "kda_ptx.cuh"
 #include "kda_tiles.cuh"
@@ -24,6 +26,7 @@
 namespace kda {
 
 kda_status_t launch_intra_fma_tc(const ChunkArgs& a, void* tiles, cudaStream_t st);
+kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cudaStream_t st);
 
 namespace {
 
@@ -128,7 +131,8 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         ptx::bulk_g2s(sb + Cfg::kQW, tile + tc::OFF_QW, 32768, &full[s]);
         ptx::bulk_g2s(sb + Cfg::kKT, tile + tc::OFF_KT, 16384, &full[s]);
         ptx::bulk_g2s(sb + Cfg::kAQ, tile + tc::OFF_AQ, 8192, &full[s]);
-        ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)col0 * 128, Cfg::kUBytes, &full[s]);
+        ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 32) * tc::U_BLOCK,
+                      Cfg::kUBytes, &full[s]);
         ptx::bulk_g2s(sb + Cfg::kGC, tile + tc::OFF_GC, 512, &full[s]);
     };
     auto wait = [&](uint64_t* bar, uint32_t parity, int where) {
@@ -166,17 +170,20 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
 
         if (warp >= 2) {   // a6: V_new = U - W S  (token row = tid - 64)
             const int i = tid - 64;
-            const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(sb + Cfg::kU);
             uint8_t* vn = smem + Cfg::kVn;
 #pragma unroll
             for (int blk = 0; blk < NS / 32; ++blk) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x32b_x32(tmem_lane + blk * 32, r);
+                // this token's 32 values of U (one 64-byte row of the column block)
+                const uint4* up = reinterpret_cast<const uint4*>(sb + Cfg::kU + blk * tc::U_BLOCK + i * 64);
+                uint4 uq[4] = {up[0], up[1], up[2], up[3]};
+                const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
                 ptx::tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     const int nn = blk * 32 + j;
-                    const float x = __bfloat162float(U[nn * 64 + i]) - __uint_as_float(r[j]);
+                    const float x = __bfloat162float(U[j]) - __uint_as_float(r[j]);
                     *reinterpret_cast<__nv_bfloat16*>(vn + ptx::sw128_off(nn, i)) =
                         __float2bfloat16_rn(x);
                 }
@@ -294,7 +301,8 @@ size_t tc_tile_bytes() { return tc::TILE_BYTES; }
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
                              WsHeader* hdr, cudaStream_t st)
 {
-    kda_status_t rc = launch_intra_fma_tc(a, tiles, st);
+    static const bool fma_intra = getenv("KDA_INTRA_FMA") != nullptr;   // debugging aid
+    kda_status_t rc = fma_intra ? launch_intra_fma_tc(a, tiles, st) : launch_intra_tc(a, tiles, hdr, st);
     if (rc != KDA_OK) return rc;
     if (n_count <= 0) return KDA_OK;
     return launch_inter_tc_t<32>(a, (const char*)tiles, n_begin, n_count, hdr, st);

@@ -15,7 +15,7 @@ constexpr uint32_t QW_HALF = 128 * 128;
 constexpr uint32_t OFF_KT = 32768;
 // A operand of the intra-chunk output term: Aqk [64][64] (lower triangular incl. diagonal)
 constexpr uint32_t OFF_AQ = 49152;
-// U in four column blocks of [32 columns][64 tokens] bf16 (token index contiguous)
+// U in four column blocks of [64 tokens][32 columns] bf16 (row-major inside a block)
 constexpr uint32_t OFF_U = 57344;
 constexpr uint32_t U_BLOCK = 32 * 64 * 2;
 // gamma^C: 128 fp32
