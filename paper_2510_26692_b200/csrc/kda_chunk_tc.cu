@@ -82,6 +82,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     if (ce > a.g1) ce = a.g1;
     const int nchunks = ce > cb ? (int)(ce - cb) : 0;
 
+    KDA_PHASE_DECL;
     if (tid == 0) {
         ptx::mbar_init(&full[0], 1);
         ptx::mbar_init(&full[1], 1);
@@ -143,6 +144,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         }
     };
 
+    KDA_PHASE(hdr, 16);  // set-up
     int loads_issued = 0;
     if (tid == 0 && nchunks > 0) { issue_loads(0, 0); loads_issued = 1; }
     uint32_t mma_phase = 0;
@@ -152,6 +154,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         uint8_t* sb = smem + s * Cfg::kStage;
         if (tid == 0 && it + 1 < nchunks) { issue_loads(s ^ 1, it + 1); loads_issued = it + 2; }
         wait(&full[s], (uint32_t)(it >> 1) & 1u, 1);
+        KDA_PHASE(hdr, 17);  // operand wait
 
         if (tid == 0) {   // MMA1: D1 = [Gamma.Q ; W] S
             ptx::tc_fence_after();
@@ -165,6 +168,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             ptx::umma_commit(mma_bar);
         }
         wait(mma_bar, mma_phase, 2);
+        KDA_PHASE(hdr, 18);  // MMA1
         mma_phase ^= 1;
         ptx::tc_fence_after();
 
@@ -192,6 +196,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         ptx::fence_async_smem();
         ptx::tc_fence_before();
         __syncthreads();
+        KDA_PHASE(hdr, 19);  // V_new
 
         if (tid == 0) {   // MMA2: D1 += [Aqk ; 0] V_new,  D3 = Kt^T V_new
             ptx::tc_fence_after();
@@ -208,6 +213,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             ptx::umma_commit(mma_bar);
         }
         wait(mma_bar, mma_phase, 3);
+        KDA_PHASE(hdr, 20);  // MMA2
         mma_phase ^= 1;
         ptx::tc_fence_after();
 
@@ -256,6 +262,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         ptx::fence_async_smem();
         ptx::tc_fence_before();
         if (__syncthreads_or((int)*abort_flag)) break;
+        KDA_PHASE(hdr, 21);  // state update + output
     }
 
     const bool aborted = *abort_flag != 0;

@@ -104,6 +104,11 @@ __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src_gmem,
                  "l"(src_gmem), "r"(src_bytes)
                  : "memory");
 }
+__device__ __forceinline__ void cp_async4(void* dst_smem, const void* src_gmem, uint32_t src_bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst_smem)),
+                 "l"(src_gmem), "r"(src_bytes)
+                 : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
