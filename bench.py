@@ -105,6 +105,22 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(self.reasons), "samples": len(s)}
 
 
+def reduce_max(x: float, world: int, device=None) -> float:
+    """Max of a per-rank scalar over all ranks (the slowest rank defines the step time)."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Units per second of the whole job: every rank processes `units_per_rank` per step."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 def oracle_arm(args, rank):
     """--impl reference: the fp64 oracle as it stands on the host cores, on the prefill workload."""
     if rank != 0:
@@ -210,11 +226,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_max(x, world, dev)
 
     if args.decode_only:
         return decode_only(args, K, inputs, torch, dev, peaks)
@@ -254,7 +266,7 @@ def main():
     clocks = sampler.finish()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     ms_step = ms_total / args.steps
-    tokens_per_s = world * T_PREFILL / (ms_step * 1e-3)
+    tokens_per_s = whole_job_rate(T_PREFILL, world, ms_step)
 
     # per-kernel durations (separate pass: the event pairs perturb back-to-back launches slightly)
     K.kda_profile_enable(True)
