@@ -97,6 +97,40 @@ kda_status_t kda_chunk_fwd(const void *q, const void *k, const void *v, const fl
                            void *cuda_stream);
 
 /*
+ * kda_chunk_fwd without a workspace argument, for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a deployment convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc and every allocating routine are off limits -- a
+ * serving loop whose memory pool was fixed at start-up, a plug-in that receives tensors but no
+ * allocator, a process whose framework has reserved all device memory.  The scratch that
+ * kda_chunk_fwd takes from the caller is replaced by a fixed array of
+ * kda_chunk_fwd_static_max_bytes() = 16 MiB that is part of the library image: every GPU that
+ * loads the library holds those 16 MiB until the process exits.
+ *
+ * Same arguments, results and error codes as kda_chunk_fwd, with these differences:
+ *   - A call whose minimum scratch (kda_chunk_fwd_min_workspace_bytes) exceeds the 16 MiB is
+ *     rejected with KDA_ERR_WORKSPACE and a message naming both sizes; nothing is launched.  The
+ *     minimum grows with n_seqs * H (64 KiB of state scratch per sequence and head) and with H
+ *     (one tile per head), so this entry point is for small batches -- e.g. up to 6 sequences of
+ *     32 heads; long sequences are fine, they are processed in several passes.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with the calling thread's current device).  Make that first call
+ *     before starting any stream capture.
+ *   - The entry point calls no cudaMalloc, cudaFree or allocating library routine.
+ *   - All calls on one device share the one array, and it keeps the previous call's contents.
+ *     Nothing in it has to be cleared by the caller (the call clears the status word itself), but
+ *     two calls that overlap on the GPU -- different streams, or one stream per thread -- race on
+ *     it: serialise them.  kda_check_status does not apply (no workspace pointer to pass).
+ */
+size_t kda_chunk_fwd_static_max_bytes(void);
+kda_status_t kda_chunk_fwd_static(const void *q, const void *k, const void *v,
+                                  const float *log_alpha, const float *beta, const float *S0,
+                                  void *o, float *S_T, const int32_t *cu_seqlens_dev,
+                                  const int32_t *cu_seqlens_host, int n_seqs, int64_t total_tokens,
+                                  int H, int dk, int dv, int chunk, float scale, kda_dtype_t dt,
+                                  void *cuda_stream);
+
+/*
  * Recurrent decode step (Eq. 1 for one token per sequence).
  *
  *   q, k, log_alpha  [n_seqs,H,dk]   v, o  [n_seqs,H,dv]   beta  [n_seqs,H]

@@ -52,6 +52,11 @@ def load():
     lib.kda_chunk_fwd.restype = i32
     lib.kda_chunk_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32,
                                   i32, f32, i32, vp, sz, vp]
+    lib.kda_chunk_fwd_static_max_bytes.restype = sz
+    lib.kda_chunk_fwd_static_max_bytes.argtypes = []
+    lib.kda_chunk_fwd_static.restype = i32
+    lib.kda_chunk_fwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32,
+                                         i32, i32, f32, i32, vp]
     lib.kda_decode_step.restype = i32
     lib.kda_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp]
     lib.kda_chunk_fwd_host_workspace_bytes.restype = sz
@@ -157,6 +162,31 @@ def kda_chunk_fwd(q, k, v, log_alpha, beta, S0, o, S_T, cu_seqlens_dev, cu_seqle
         _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
         int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale), int(dt),
         _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
+    _check(rc)
+
+
+def kda_chunk_fwd_static_max_bytes() -> int:
+    return int(load().kda_chunk_fwd_static_max_bytes())
+
+
+def kda_chunk_fwd_static(q, k, v, log_alpha, beta, S0, o, S_T, cu_seqlens_dev, cu_seqlens_host,
+                         n_seqs, total_tokens, H, dk, dv, chunk, scale, dt, stream=None):
+    """``kda_chunk_fwd_static``: the prefill for callers that may not allocate device memory (a
+    fixed-pool serving loop, a plug-in without an allocator).  Takes no workspace: the scratch is a
+    16 MiB array inside the library, shared by all calls on the device, so calls that overlap on
+    the GPU must be serialised; calls that need more scratch raise ``KdaError``
+    (KDA_ERR_WORKSPACE).  The first call on a device does a one-time address look-up and should
+    come before any stream capture."""
+    f32 = torch.float32
+    et = torch.bfloat16 if dt == KDA_BF16 else torch.float32
+    rc = load().kda_chunk_fwd_static(
+        _ptr(q, True, et, "q"), _ptr(k, True, et, "k"), _ptr(v, True, et, "v"),
+        _ptr(log_alpha, True, f32, "log_alpha"), _ptr(beta, True, f32, "beta"),
+        _ptr(S0, True, f32, "S0"), _ptr(o, True, et, "o"), _ptr(S_T, True, f32, "S_T"),
+        _ptr(cu_seqlens_dev, True, torch.int32, "cu_seqlens_dev"),
+        _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
+        int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale), int(dt),
+        _stream(stream))
     _check(rc)
 
 
