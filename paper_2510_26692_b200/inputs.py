@@ -79,6 +79,35 @@ def chunk_inputs(lengths: Sequence[int], H: int, dk: int = 128, dv: int = 128,
     return out
 
 
+def chunk_inputs_slabbed(T: int, H: int, dk: int = 128, dv: int = 128, seed: int = 3,
+                         gate_mean: float = 6.0, s0_std: float = 0.02, device="cuda",
+                         slab: int = 65536, want_q: bool = True) -> Dict[str, Optional[torch.Tensor]]:
+    """One long sequence (bf16 q/k/v) drawn slab by slab on ``device`` so that the fp32
+    temporaries stay small; slab s of a tensor uses the generator seed (seed*4096 + s)*16 + index.
+    Same distributions as :func:`chunk_inputs`."""
+    bf = torch.bfloat16
+    out: Dict[str, Optional[torch.Tensor]] = {
+        "q": torch.empty((T, H, dk), dtype=bf, device=device) if want_q else None,
+        "k": torch.empty((T, H, dk), dtype=bf, device=device),
+        "v": torch.empty((T, H, dv), dtype=bf, device=device),
+        "log_alpha": torch.empty((T, H, dk), dtype=torch.float32, device=device),
+        "beta": torch.empty((T, H), dtype=torch.float32, device=device),
+    }
+    for s, t0 in enumerate(range(0, T, slab)):
+        n = min(slab, T - t0)
+        sd = seed * 4096 + s
+        if want_q:
+            out["q"][t0:t0 + n] = (_l2norm(_randn((n, H, dk), sd, "q", device)) * (dk ** -0.5)).to(bf)
+        out["k"][t0:t0 + n] = _l2norm(_randn((n, H, dk), sd, "k", device)).to(bf)
+        out["v"][t0:t0 + n] = _randn((n, H, dv), sd, "v", device).to(bf)
+        out["log_alpha"][t0:t0 + n] = torch.nn.functional.logsigmoid(
+            _randn((n, H, dk), sd, "x", device) + gate_mean)
+        out["beta"][t0:t0 + n] = torch.sigmoid(_randn((n, H), sd, "beta", device))
+    out["S0"] = (_randn((1, H, dk, dv), seed, "S0", device) * s0_std) if s0_std > 0 else None
+    out["cu_seqlens"] = cu_seqlens_of([T])
+    return out
+
+
 def decode_inputs(n_seqs: int, H: int, steps: int, dk: int = 128, dv: int = 128,
                   dtype: torch.dtype = torch.bfloat16, seed: int = 4, gate_mean: float = 4.0,
                   s_std: float = 0.05, device="cpu") -> Dict[str, torch.Tensor]:

@@ -34,6 +34,57 @@ def test_config2_varlen(oracle_mod):
     print("config2 lens", lens, "worst", max(errs.values()))
 
 
+def test_config3_long_context(oracle_mod):
+    """B=1, T=1 Mi, H=32, slow decay (x ~ N(6,1)).  The timed mode returns the final state only
+    (o = NULL, q unused).  With these gates the state forgets its past at about e^-0.004 per token,
+    so the oracle, run on the last 16 Ki tokens from a zero state, gives S_T to e^-60; an
+    untimed second call with o is compared on windows at the start, across token 2^19 (where a
+    32-bit element offset would wrap) and at the end."""
+    T, H = 1 << 20, 32
+    free, _ = torch.cuda.mem_get_info()
+    if free < 75 * (1 << 30):
+        pytest.skip("needs ~70 GB of free device memory")
+    d = inputs.chunk_inputs_slabbed(T, H, seed=3, gate_mean=6.0, s0_std=0.02, device="cuda:0")
+    dev = "cuda:0"
+    nbytes = K.kda_chunk_fwd_workspace_bytes(T, 1, H)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    S_T = torch.full((1, H, 128, 128), float("nan"), dtype=torch.float32, device=dev)
+    # state-only call: q = NULL, o = NULL
+    K.kda_chunk_fwd(None, d["k"], d["v"], d["log_alpha"], d["beta"], d["S0"], None, S_T, None, None,
+                    1, T, H, 128, 128, 64, 1.0, K.KDA_BF16, ws, nbytes)
+    K.kda_check_status(ws)
+    W = 16384
+
+    def oracle_window(t0, t1, S0=None, want_o=True):
+        sl = slice(t0, t1)
+        return oracle_mod.recurrence(to_np32(d["q"][sl]) if want_o else None, to_np32(d["k"][sl]),
+                                     to_np32(d["v"][sl]), to_np32(d["log_alpha"][sl]),
+                                     to_np32(d["beta"][sl]), S0=S0, want_o=want_o)
+
+    _, S_ref = oracle_window(T - W, T, want_o=False)
+    err_S = rel_l2(to_np32(S_T), S_ref)
+    assert err_S <= TOL[K.KDA_BF16], err_S
+    # second call with o
+    o = torch.empty_like(d["v"])
+    S_T2 = torch.empty_like(S_T)
+    K.kda_chunk_fwd(d["q"], d["k"], d["v"], d["log_alpha"], d["beta"], d["S0"], o, S_T2, None, None,
+                    1, T, H, 128, 128, 64, 1.0, K.KDA_BF16, ws, nbytes)
+    torch.cuda.synchronize()
+    assert torch.equal(S_T, S_T2)
+    errs = {"S_T": err_S}
+    # start of the sequence: depends on S0
+    o_ref, _ = oracle_window(0, 2048, S0=d["S0"].double().cpu().numpy())
+    errs["o[0:2048]"] = rel_l2(to_np32(o[0:2048]), o_ref)
+    # across token 2^19 and at the end: warm the state up over W tokens, compare the last 2048
+    for name, t1 in (("o[2^19]", (1 << 19) + 1024), ("o[end]", T)):
+        o_ref, _ = oracle_window(t1 - 2048 - W, t1)
+        errs[name] = rel_l2(to_np32(o[t1 - 2048:t1]), o_ref[-2048:])
+    print("config3", errs)
+    assert max(errs.values()) <= TOL[K.KDA_BF16], errs
+    del d, o, ws
+    torch.cuda.empty_cache()
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("T", [1, 63, 64, 65, 127, 200])
 def test_ragged_lengths(oracle_mod, dtype, T):
@@ -129,6 +180,23 @@ def test_harsh_gates(oracle_mod):
     d = inputs.chunk_inputs([256], H=2, dtype=torch.float32, seed=27, gate_mean=-1.0, s0_std=0.02)
     check_chunk(oracle_mod, d, TOL[K.KDA_F32])
     d = inputs.chunk_inputs([256], H=2, dtype=torch.bfloat16, seed=27, gate_mean=-1.0, s0_std=0.02)
+    check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
+
+
+def test_equal_length_batch(oracle_mod):
+    """cu_seqlens = NULL with n_seqs > 1: equal-length sequences laid out back to back."""
+    N, Ls, H = 3, 130, 2
+    d = inputs.chunk_inputs([Ls] * N, H=H, dtype=torch.bfloat16, seed=29, s0_std=0.02)
+    o_var, S_var = run_chunk(d)                       # packed form of the same batch
+    g = {n: (t.cuda() if isinstance(t, torch.Tensor) else t) for n, t in d.items()}
+    nb = K.kda_chunk_fwd_workspace_bytes(N * Ls, N, H)
+    ws = torch.empty(nb, dtype=torch.uint8, device="cuda:0")
+    o = torch.empty_like(g["v"])
+    S_T = torch.empty((N, H, 128, 128), dtype=torch.float32, device="cuda:0")
+    K.kda_chunk_fwd(g["q"], g["k"], g["v"], g["log_alpha"], g["beta"], g["S0"], o, S_T, None, None,
+                    N, N * Ls, H, 128, 128, 64, 1.0, K.KDA_BF16, ws, nb)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o_var) and torch.equal(S_T, S_var)
     check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
 
 
