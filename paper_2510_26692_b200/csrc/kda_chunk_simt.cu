@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __re
         *reinterpret_cast<float4*>(sQg + i * LD + c) = make_float4(oqg[0], oqg[1], oqg[2], oqg[3]);
         *reinterpret_cast<float4*>(sKG + i * LD + c) = make_float4(oKG[0], oKG[1], oKG[2], oKG[3]);
         if (kTc) {
-            st_bf16x4(tct + tc::OFF_QW + (c >> 6) * tc::QW_HALF + ptx::sw128_off(i, c & 63), oQG[0],
+            st_bf16x4(tct + tc::OFF_QW + (c >> 6) * tc::QW_HALF + ptx::sw128_off(64 + i, c & 63), oQG[0],
                       oQG[1], oQG[2], oQG[3]);
 #pragma unroll
             for (int e = 0; e < 4; ++e) st_bf16(tct + tc::OFF_KT + ptx::sw128_off(c + e, i), oKT[e]);
@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __re
         for (int m = 0; m < 8; ++m) {
             const int c = cq * 4 + 16 * m;
             if (kTc) {
-                st_bf16x4(tct + tc::OFF_QW + (c >> 6) * tc::QW_HALF + ptx::sw128_off(64 + i, c & 63),
+                st_bf16x4(tct + tc::OFF_QW + (c >> 6) * tc::QW_HALF + ptx::sw128_off(i, c & 63),
                           w[m].x, w[m].y, w[m].z, w[m].w);
                 const float uu[4] = {u[m].x, u[m].y, u[m].z, u[m].w};
 #pragma unroll

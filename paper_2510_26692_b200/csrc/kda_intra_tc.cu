@@ -21,6 +21,8 @@
 // Outputs go to the scratch tile of kda_tiles.cuh as ready-made operand images of the inter-chunk
 // kernel.  Tail chunks: rows past the sequence end behave as identity steps (log alpha = 0,
 // beta = 0, k = q = v = 0).
+#include <cuda.h>
+
 #include "kda_common.cuh"
 #include "kda_ptx.cuh"
 #include "kda_tiles.cuh"
@@ -30,7 +32,6 @@ namespace {
 
 constexpr uint64_t kWaitLimitNs = 1000000000ull;
 constexpr int LDT = 68;                                   // padded fp32 row of the 64x64 matrices
-constexpr float kExpClamp = 80.f;
 
 // shared-memory map (bytes from a 1024-aligned base)
 constexpr uint32_t S_KQ = 0;          // [2 K-halves][128 rows][64] bf16: rows 0-63 Kg, 64-127 Qg
@@ -45,16 +46,18 @@ constexpr uint32_t S_T = S_A + 64 * LDT * 4;   // fp32 [64][LDT]: T
 // staging of outputs for bulk stores (aliases buffers that are dead at the time):
 constexpr uint32_t S_QG = S_M;                 // scale Q exp(G): [2 halves][64][64] bf16, 16 KiB   (phase 1)
 constexpr uint32_t S_KT = S_M + 16384;         // (K exp(G_C - G))^T: [128][64] bf16, 16 KiB        (phase 1)
-constexpr uint32_t S_TOT = S_M + 32768;        // scan exchange [16][128] fp32, 8 KiB
+constexpr uint32_t S_TOT = S_M + 32768;        // scan exchange [8][128] fp32, 4 KiB
 constexpr uint32_t S_AQ = S_KI;                // Aqk image [64][64] bf16 (after the first MMA group)
 constexpr uint32_t S_W = S_M;                  // W image [2 halves][64][64] bf16 (after the second group)
 constexpr uint32_t S_U = S_M + 16384;          // U [4 blocks][64][32] bf16
 constexpr uint32_t S_BETA = S_T + 64 * LDT * 4;
 constexpr uint32_t S_CG = S_BETA + 256;        // exp(G_m) per channel (undoes the Kg reference)
-constexpr uint32_t S_BAR = S_CG + 512;
+constexpr uint32_t S_BAR = S_CG + 512;          // mma barrier, tma barrier, TMEM slot
 constexpr uint32_t S_TOTAL = S_BAR + 64;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kClamp2 = 80.f * 1.4426950408889634f;   // the +-80 clamp in the log2 domain
 constexpr uint32_t kIntraTcSmem = S_TOTAL + 1024;
-static_assert(S_TOT + 16 * 128 * 4 <= S_BETA, "staging + scan exchange fit below the small arrays");
+static_assert(S_TOT + 8 * 128 * 4 <= S_BETA, "staging + scan exchange fit below the small arrays");
 constexpr uint32_t kTmemCols = 256;
 
 // loads that the compiler may not sink below their issue point (register prefetch of the next tile)
@@ -63,29 +66,19 @@ __device__ __forceinline__ void ld_nc_f4(const float* p, float& a, float& b, flo
                  : "=f"(a), "=f"(b), "=f"(c), "=f"(d)
                  : "l"(p));
 }
-__device__ __forceinline__ uint4 ld_nc_u4(const void* p) {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-                 : "l"(p));
-    return r;
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&p);
 }
-__device__ __forceinline__ void unpack8(const uint4& r, float (&f)[8]) {
-    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&r);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        float2 x = __bfloat1622float2(p[e]);
-        f[2 * e] = x.x;
-        f[2 * e + 1] = x.y;
-    }
-}
-
 __global__ void __launch_bounds__(256, 2)
-kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
+kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
+             const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+             const __grid_constant__ CUtensorMap tm_v, int has_q)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(
@@ -96,17 +89,19 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
     float* sBeta = reinterpret_cast<float*>(smem + S_BETA);
     float* sCG = reinterpret_cast<float*>(smem + S_CG);
     uint64_t* mma_bar = reinterpret_cast<uint64_t*>(smem + S_BAR);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_bar + 1);
+    uint64_t* tma_bar = mma_bar + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_bar + 2);
 
     const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
-    const __nv_bfloat16* qp = reinterpret_cast<const __nv_bfloat16*>(a.q);
-    const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(a.k);
-    const __nv_bfloat16* vp = reinterpret_cast<const __nv_bfloat16*>(a.v);
 
     KDA_PHASE_DECL;
     if (t == 0) {
         ptx::mbar_init(mma_bar, 1);
+        ptx::mbar_init(tma_bar, 1);
         ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tm_k);
+        ptx::prefetch_tmap(&tm_q);
+        ptx::prefetch_tmap(&tm_v);
     }
     if (warp == 0) {
         ptx::tmem_alloc(tmem_slot, kTmemCols);
@@ -114,47 +109,38 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
     }
 
     // Persistent CTA: tiles cur, cur + gridDim.x, ...  (tile = chunk-in-pass * H + head).  The
-    // inputs of the next tile are requested while the current one is being processed: log alpha,
-    // k and q into registers (thread (rg, dc) owns rows 4rg..4rg+3, channels 8dc..8dc+7), v and
-    // beta by asynchronous copies into shared memory.
-    const int dc = t & 15, rg = t >> 4;
-    const int d0 = dc * 8, i0 = rg * 4;
-    const int64_t ntiles = (a.g1 - a.g0) * a.H;
-    float G[4][8];
-    auto locate = [&](int64_t tl, ChunkLoc& Lo, int& ho) {
-        const int64_t gl = tl / a.H;
-        ho = (int)(tl - gl * a.H);
+    // inputs of the next tile are requested as soon as the buffers of the current one are free:
+    // k, q and v by 2-D tiled TMA loads straight into the swizzled operand images (k and q are then
+    // gated in place), log alpha into registers (thread (w, c4) owns rows 8w..8w+7 and channels
+    // 4c4..4c4+3), beta by small asynchronous copies.
+    const int c4 = lane, d0 = c4 * 4, i0 = warp * 8;
+    const uint32_t ntiles = (uint32_t)((a.g1 - a.g0) * a.H);
+    float G[8][4];
+    auto locate = [&](uint32_t tl, ChunkLoc& Lo, int& ho) {
+        const uint32_t gl = tl / (uint32_t)a.H;
+        ho = (int)(tl - gl * (uint32_t)a.H);
         Lo = locate_chunk(a, a.g0 + gl);
     };
-    const int half = dc >> 3, cc = dc & 7;
     auto issue_prefetch = [&](const ChunkLoc& Lo, int ho) {
-        // log alpha -> registers; k, q -> their slots of the [Kg ; Qg] operand image (each thread
-        // copies exactly the 16-byte chunks it will later read and overwrite in place); v -> its
-        // token-major image; beta.  Rows past the sequence end are zero-filled.
+        const float* gp = a.log_alpha + ((size_t)Lo.tok0 * a.H + ho) * kD + d0;
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
+        for (int r = 0; r < 8; ++r) {
             const int i = i0 + r;
-            const bool ok = i < Lo.len;
-            const size_t off = ((Lo.tok0 + (ok ? i : 0)) * a.H + ho) * kD + d0;
-            if (ok) {
-                ld_nc_f4(a.log_alpha + off, G[r][0], G[r][1], G[r][2], G[r][3]);
-                ld_nc_f4(a.log_alpha + off + 4, G[r][4], G[r][5], G[r][6], G[r][7]);
+            if (i < Lo.len) {
+                ld_nc_f4(gp + (size_t)i * a.H * kD, G[r][0], G[r][1], G[r][2], G[r][3]);
             } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) G[r][e] = 0.f;
+                G[r][0] = G[r][1] = G[r][2] = G[r][3] = 0.f;
             }
-            const uint32_t sw = (uint32_t)((cc ^ (i & 7)) << 4);
-            ptx::cp_async16(smem + S_KQ + half * S_KQ_HALF + i * 128 + sw, kp + off, ok ? 16u : 0u);
-            ptx::cp_async16(smem + S_KQ + half * S_KQ_HALF + (64 + i) * 128 + sw, qp ? qp + off : kp + off,
-                            (ok && qp) ? 16u : 0u);
         }
+        if (t == 0) {
+            ptx::mbar_expect_tx(tma_bar, 3 * 16384);
+            const int x = ho * kD, y = (int)Lo.tok0;
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const int j = (t >> 4) + 16 * m, c16 = t & 15;
-            const bool ok = j < Lo.len;
-            const __nv_bfloat16* src = vp + ((Lo.tok0 + (ok ? j : 0)) * a.H + ho) * kD + c16 * 8;
-            ptx::cp_async16(smem + S_V + (c16 >> 3) * S_V_BLOCK + j * 128 + (((c16 & 7) ^ (j & 7)) << 4),
-                            src, ok ? 16u : 0u);
+            for (int hf = 0; hf < 2; ++hf) {
+                ptx::tma_load_2d(smem + S_KQ + hf * S_KQ_HALF, &tm_k, x + hf * 64, y, tma_bar);
+                ptx::tma_load_2d(smem + S_KQ + hf * S_KQ_HALF + 8192, &tm_q, x + hf * 64, y, tma_bar);
+                ptx::tma_load_2d(smem + S_V + hf * S_V_BLOCK, &tm_v, x + hf * 64, y, tma_bar);
+            }
         }
         if (t < kC) {
             const bool ok = t < Lo.len;
@@ -168,8 +154,9 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool timed_out = false;
+    uint32_t tma_parity = 0;
 
-    int64_t cur = blockIdx.x;
+    uint32_t cur = blockIdx.x;
     ChunkLoc L;
     int h = 0;
     if (cur < ntiles) {
@@ -178,31 +165,31 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
     }
     for (; cur < ntiles; cur += gridDim.x) {
     char* tile = tiles + (size_t)cur * tc::TILE_BYTES;
-    const int64_t nxt = cur + gridDim.x;
+    const uint32_t nxt = cur + gridDim.x;
     ChunkLoc Ln = L;
     int hn = h;
 
-    // ---- a1: cumulative log-decay ---------------------------------------------------------------------
+    // ---- a1: cumulative log-decay, in the log2 domain (exponentials below are bare ex2) -------
 #pragma unroll
-    for (int r = 1; r < 4; ++r)
+    for (int e = 0; e < 4; ++e) G[0][e] *= kLog2e;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) G[r][e] += G[r - 1][e];
-    *reinterpret_cast<float4*>(sTot + rg * kD + d0) = make_float4(G[3][0], G[3][1], G[3][2], G[3][3]);
-    *reinterpret_cast<float4*>(sTot + rg * kD + d0 + 4) = make_float4(G[3][4], G[3][5], G[3][6], G[3][7]);
+    for (int r = 1; r < 8; ++r)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) G[r][e] = fmaf(G[r][e], kLog2e, G[r - 1][e]);
+    *reinterpret_cast<float4*>(sTot + warp * kD + d0) = make_float4(G[7][0], G[7][1], G[7][2], G[7][3]);
+    if (t == 0) ptx::bulk_wait_read0();   // the previous tile's output staging has been read out
+    ptx::cp_async_wait_all();             // beta
     __syncthreads();
     KDA_PHASE(hdr, 0);   // loads arrived + local scan
-    float base[8], gref[8], glast[8];
+    float base[4] = {0.f, 0.f, 0.f, 0.f}, gref[4] = {0.f, 0.f, 0.f, 0.f}, glast[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int e = 0; e < 8; ++e) base[e] = gref[e] = glast[e] = 0.f;
+    for (int r2 = 0; r2 < 8; ++r2) {
+        const float4 x4 = *reinterpret_cast<const float4*>(sTot + r2 * kD + d0);
+        const float x[4] = {x4.x, x4.y, x4.z, x4.w};
 #pragma unroll
-    for (int r2 = 0; r2 < 16; ++r2) {
-        const float4 x0 = *reinterpret_cast<const float4*>(sTot + r2 * kD + d0);
-        const float4 x1 = *reinterpret_cast<const float4*>(sTot + r2 * kD + d0 + 4);
-        const float x[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            if (r2 < rg) base[e] += x[e];
-            if (r2 < 8) gref[e] += x[e];
+        for (int e = 0; e < 4; ++e) {
+            if (r2 < warp) base[e] += x[e];
+            if (r2 < 4) gref[e] += x[e];    // rows 0..31
             glast[e] += x[e];
         }
     }
@@ -211,74 +198,89 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
     // exp(G) = exp(G - G_m) exp(G_m) and exp(G_C - G) = exp(G_m - G) exp(G_C - G_m) reuse the two
     // exponentials of the intra-chunk operands unless a channel decays by more than e^-80 on one
     // side of the middle row, in which case they are evaluated directly (no underflow of the factor)
-    float cg[8], ct[8];
+    float cg[4], ct[4];
     bool harsh = false;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        cg[e] = __expf(gref[e]);               // exp(G_m)
-        ct[e] = __expf(glast[e] - gref[e]);    // exp(G_C - G_m)
-        harsh = harsh || (gref[e] < -kExpClamp) || (glast[e] - gref[e] < -kExpClamp);
+    for (int e = 0; e < 4; ++e) {
+        cg[e] = ex2(gref[e]);               // exp(G_m)
+        ct[e] = ex2(glast[e] - gref[e]);    // exp(G_C - G_m)
+        harsh = harsh || (gref[e] < -kClamp2) || (glast[e] - gref[e] < -kClamp2);
     }
-    if (rg == 0) {
-        float gc[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) gc[e] = __expf(glast[e]);
-        *reinterpret_cast<float4*>(tile + tc::OFF_GC + d0 * 4) = make_float4(gc[0], gc[1], gc[2], gc[3]);
-        *reinterpret_cast<float4*>(tile + tc::OFF_GC + d0 * 4 + 16) = make_float4(gc[4], gc[5], gc[6], gc[7]);
+    if (warp == 0) {
+        *reinterpret_cast<float4*>(tile + tc::OFF_GC + d0 * 4) =
+            make_float4(ex2(glast[0]), ex2(glast[1]), ex2(glast[2]), ex2(glast[3]));
         *reinterpret_cast<float4*>(sCG + d0) = make_float4(cg[0], cg[1], cg[2], cg[3]);
-        *reinterpret_cast<float4*>(sCG + d0 + 4) = make_float4(cg[4], cg[5], cg[6], cg[7]);
     }
     KDA_PHASE(hdr, 10);  // prefix + per-channel factors
-    ptx::cp_async_wait_all();   // this thread's k, q chunks (and its share of v, beta) have landed
-    KDA_PHASE(hdr, 11);  // cp.async wait
-    float kt[4][8];   // K exp(G_C - G) for the transposed store
+    if (!ptx::mbar_wait(tma_bar, tma_parity, kWaitLimitNs)) timed_out = true;   // k, q, v have landed
+    tma_parity ^= 1;
+    KDA_PHASE(hdr, 11);  // TMA wait
+    if (L.len < kC) {   // short last chunk: rows past the end hold the next sequence's v; zero them
+        for (int idx = t; idx < (kC - L.len) * 16; idx += 256) {
+            const int j = L.len + (idx >> 4), c16 = idx & 15;
+            *reinterpret_cast<uint4*>(smem + S_V + (c16 >> 3) * S_V_BLOCK + j * 128 +
+                                      (((c16 & 7) ^ (j & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    const int hf = c4 >> 4;                       // K-half (channels 0-63 / 64-127)
+    uint32_t ktb[4][4];                           // (K exp(G_C - G))^T: 4 channels x 8 tokens, bf16 pairs
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
+    for (int r = 0; r < 8; ++r) {
         const int i = i0 + r;
-        float kf[8], qf[8];
-        const uint32_t sw = (uint32_t)((cc ^ (i & 7)) << 4);
-        unpack8(*reinterpret_cast<const uint4*>(smem + S_KQ + half * S_KQ_HALF + i * 128 + sw), kf);
-        unpack8(*reinterpret_cast<const uint4*>(smem + S_KQ + half * S_KQ_HALF + (64 + i) * 128 + sw), qf);
-        float okg[8], oqg[8], oki[8], oqt[8];
+        const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
+        uint8_t* pk = smem + S_KQ + hf * S_KQ_HALF + off;
+        uint2 k2 = *reinterpret_cast<const uint2*>(pk);
+        uint2 q2 = *reinterpret_cast<const uint2*>(pk + 8192);
+        if (i >= L.len) k2 = q2 = make_uint2(0u, 0u);
+        if (!has_q) q2 = make_uint2(0u, 0u);
+        const float kf[4] = {__uint_as_float(k2.x << 16), __uint_as_float(k2.x & 0xffff0000u),
+                             __uint_as_float(k2.y << 16), __uint_as_float(k2.y & 0xffff0000u)};
+        const float qf[4] = {__uint_as_float(q2.x << 16), __uint_as_float(q2.x & 0xffff0000u),
+                             __uint_as_float(q2.y << 16), __uint_as_float(q2.y & 0xffff0000u)};
+        float okg[4], oqg[4], oki[4], oqt[4], okt[4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
+        for (int e = 0; e < 4; ++e) {
             const float gg = G[r][e] + base[e];
-            const float x = fminf(fmaxf(gg - gref[e], -kExpClamp), kExpClamp);
-            const float e1 = __expf(x);                  // exp(G - G_m)
-            const float e2 = __expf(-x);                 // exp(G_m - G)
+            const float x = fminf(fmaxf(gg - gref[e], -kClamp2), kClamp2);
+            const float e1 = ex2(x);                     // exp(G - G_m)
+            const float e2 = ex2(-x);                    // exp(G_m - G)
             const float qs = a.scale * qf[e];
             okg[e] = kf[e] * e1;
             oqg[e] = qs * e1;
             oki[e] = kf[e] * e2;
             if (!harsh) {
                 oqt[e] = oqg[e] * cg[e];
-                kt[r][e] = oki[e] * ct[e];
+                okt[e] = oki[e] * ct[e];
             } else {
-                oqt[e] = qs * __expf(gg);
-                kt[r][e] = kf[e] * __expf(glast[e] - gg);
+                oqt[e] = qs * ex2(gg);
+                okt[e] = kf[e] * ex2(glast[e] - gg);
             }
         }
-        *reinterpret_cast<uint4*>(smem + S_KQ + half * S_KQ_HALF + i * 128 + sw) =
-            make_uint4(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]), pack_bf16(okg[4], okg[5]),
-                       pack_bf16(okg[6], okg[7]));
-        *reinterpret_cast<uint4*>(smem + S_KQ + half * S_KQ_HALF + (64 + i) * 128 + sw) =
-            make_uint4(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]), pack_bf16(oqg[4], oqg[5]),
-                       pack_bf16(oqg[6], oqg[7]));
-        *reinterpret_cast<uint4*>(smem + S_KI + half * S_KI_HALF + i * 128 + sw) =
-            make_uint4(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]), pack_bf16(oki[4], oki[5]),
-                       pack_bf16(oki[6], oki[7]));
-        *reinterpret_cast<uint4*>(smem + S_QG + half * 8192 + i * 128 + sw) =
-            make_uint4(pack_bf16(oqt[0], oqt[1]), pack_bf16(oqt[2], oqt[3]), pack_bf16(oqt[4], oqt[5]),
-                       pack_bf16(oqt[6], oqt[7]));
-    }
-    // (K exp(G_C - G))^T: row = channel, 4 consecutive tokens per 8-byte store
+        *reinterpret_cast<uint2*>(pk) = make_uint2(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]));
+        *reinterpret_cast<uint2*>(pk + 8192) = make_uint2(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]));
+        *reinterpret_cast<uint2*>(smem + S_KI + hf * S_KI_HALF + off) =
+            make_uint2(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]));
+        *reinterpret_cast<uint2*>(smem + S_QG + hf * 8192 + off) =
+            make_uint2(pack_bf16(oqt[0], oqt[1]), pack_bf16(oqt[2], oqt[3]));
+        if (r & 1) {
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        uint2 p;
-        p.x = pack_bf16(kt[0][e], kt[1][e]);
-        p.y = pack_bf16(kt[2][e], kt[3][e]);
-        *reinterpret_cast<uint2*>(smem + S_KT + ptx::sw128_off(d0 + e, i0)) = p;
+            for (int e = 0; e < 4; ++e) {
+                __nv_bfloat16 hi = __float2bfloat16_rn(okt[e]);
+                ktb[e][r >> 1] |= (uint32_t)(*reinterpret_cast<uint16_t*>(&hi)) << 16;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                __nv_bfloat16 lo = __float2bfloat16_rn(okt[e]);
+                ktb[e][r >> 1] = (uint32_t)(*reinterpret_cast<uint16_t*>(&lo));
+            }
+        }
     }
+    // (K exp(G_C - G))^T: row = channel, this warp's 8 tokens are one 16-byte chunk
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+        *reinterpret_cast<uint4*>(smem + S_KT + (d0 + e) * 128 + ((warp ^ ((d0 + e) & 7)) << 4)) =
+            make_uint4(ktb[e][0], ktb[e][1], ktb[e][2], ktb[e][3]);
 
     KDA_PHASE(hdr, 12);  // element loop + stores (thread 0)
     ptx::fence_async_smem();
@@ -290,8 +292,8 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
     // ---- a2 + a5: [Kg ; Qg] Ki^T ------------------------------------------------------------------------
     if (t == 0) {
         // phase-1 outputs leave through the TMA engine while the MMA runs
-        ptx::bulk_s2g(tile + tc::OFF_QW, smem + S_QG, 8192);
-        ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF, smem + S_QG + 8192, 8192);
+        ptx::bulk_s2g(tile + tc::OFF_QW + 8192, smem + S_QG, 8192);
+        ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF + 8192, smem + S_QG + 8192, 8192);
         ptx::bulk_s2g(tile + tc::OFF_KT, smem + S_KT, 16384);
         ptx::bulk_commit();
         const uint32_t idesc = ptx::umma_idesc_bf16(128, 64);
@@ -506,11 +508,10 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
     ptx::tc_fence_before();
     __syncthreads();
     if (t == 0) {
-        ptx::bulk_s2g(tile + tc::OFF_QW + 8192, smem + S_W, 8192);
-        ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF + 8192, smem + S_W + 8192, 8192);
+        ptx::bulk_s2g(tile + tc::OFF_QW, smem + S_W, 8192);
+        ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF, smem + S_W + 8192, 8192);
         ptx::bulk_s2g(tile + tc::OFF_U, smem + S_U, 16384);
-        ptx::bulk_commit();
-        ptx::bulk_wait_read0();   // shared memory must outlive the reads of every bulk store
+        ptx::bulk_commit();   // read-out completion is awaited before the staging area is reused
     }
     KDA_PHASE(hdr, 9);   // W, U epilogue
     L = Ln;
@@ -518,12 +519,50 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr)
     }   // tile loop
 
     if (timed_out && atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = 10;
+    KDA_PHASE_FLUSH(hdr);
+    if (t == 0) ptx::bulk_wait_read0();   // shared memory must outlive the reads of every bulk store
     ptx::cp_async_wait_all();
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 0) ptx::tmem_dealloc(tmem_base, kTmemCols);
 }
 
+}  // namespace
+
+namespace {
+// cuTensorMapEncodeTiled through the runtime's driver entry-point query (no link dependency on
+// libcuda, so the library still loads on a machine without a driver)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+// [total_tokens, H*128] bf16 matrix, boxes of 64 tokens x 64 channels, 128-byte swizzle
+kda_status_t make_tmap(CUtensorMap* tm, const void* base, int64_t total_tokens, int H)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return fail(KDA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    const cuuint64_t dims[2] = {(cuuint64_t)H * kD, (cuuint64_t)total_tokens};
+    const cuuint64_t strides[1] = {(cuuint64_t)H * kD * 2};
+    const cuuint32_t box[2] = {64, 64};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(KDA_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return KDA_OK;
+}
 }  // namespace
 
 kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cudaStream_t st)
@@ -536,16 +575,23 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cud
     }
     const int64_t n_tiles = (a.g1 - a.g0) * a.H;
     if (n_tiles <= 0) return KDA_OK;
+    if (n_tiles > 0x7fffffff || a.total_tokens > 0x7fffffff)
+        return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: more than 2^31 tokens or tiles in one pass");
     static int n_sm = 0;
     if (n_sm == 0) {
         int dev = 0;
         KDA_CUDA_TRY(cudaGetDevice(&dev));
         KDA_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     }
+    CUtensorMap tm_k, tm_q, tm_v;
+    kda_status_t rc = make_tmap(&tm_k, a.k, a.total_tokens, a.H);
+    if (rc == KDA_OK) rc = make_tmap(&tm_v, a.v, a.total_tokens, a.H);
+    if (rc == KDA_OK) rc = make_tmap(&tm_q, a.q ? a.q : a.k, a.total_tokens, a.H);
+    if (rc != KDA_OK) return rc;
     const int64_t resident = 2 * (int64_t)n_sm;   // two CTAs per SM
     const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
     ProfScope ps(PROF_INTRA, st);
-    kda_intra_tc<<<grid, 256, kIntraTcSmem, st>>>(a, (char*)tiles, hdr);
+    kda_intra_tc<<<grid, 256, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, a.q ? 1 : 0);
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;

@@ -43,15 +43,25 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: polls the barrier; after `limit_ns` of wall time gives up and returns false.
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: try_wait suspends the thread in hardware for a short, implementation-defined time
+// and returns false if the phase has not completed by then; after `limit_ns` of wall time the
+// wait gives up and returns false.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns) {
-    if (mbar_test(bar, parity)) return true;
+    if (mbar_try(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
-    uint32_t spins = 0;
-    while (!mbar_test(bar, parity)) {
-        if ((++spins & 255u) == 0u) {
-            if (globaltimer_ns() - t0 > limit_ns) return false;
-        }
+    while (!mbar_try(bar, parity)) {
+        if (globaltimer_ns() - t0 > limit_ns) return false;
     }
     return true;
 }

@@ -7,8 +7,8 @@
 
 namespace kda {
 namespace tc {
-// A operand of  [ (Gamma.Q) ; W ] S : two K-halves of [128 rows][64], rows 0-63 = scale*Gamma.Q,
-// rows 64-127 = W
+// A operand of  [ W ; (Gamma.Q) ] S : two K-halves of [128 rows][64], rows 0-63 = W,
+// rows 64-127 = scale*Gamma.Q
 constexpr uint32_t OFF_QW = 0;
 constexpr uint32_t QW_HALF = 128 * 128;
 // A operand of the state update: ((gamma^C/Gamma).K)^T as [128 dk][64 tokens]
