@@ -41,16 +41,17 @@ template <int NS> struct InterCfg {
     static constexpr uint32_t kQW = 0;                      // [2 K-halves][128][64]: rows 0-63 W, 64-127 Gamma.Q
     static constexpr uint32_t kKT = 32768;                  // [128 dk][64 tokens]
     static constexpr uint32_t kAQ = 49152;                  // [64][64]; used as rows 64-127 of a 128-row operand
-    static constexpr uint32_t kU = 57344;                   // [64 tokens][NS]
+    static constexpr uint32_t kGC = 57344;                  // gamma^C, 128 fp32
+    static constexpr uint32_t kMainBytes = 57856;           // QW | Kt | Aqk | gamma^C are contiguous in a tile
+    static constexpr uint32_t kU = 57856;                   // [64 tokens][NS]
     static constexpr uint32_t kUBytes = 64 * NS * 2;
-    static constexpr uint32_t kGC = kU + kUBytes;
-    static constexpr uint32_t kStage = (kGC + 512 + 1023) / 1024 * 1024;
+    static constexpr uint32_t kStage = (kU + kUBytes + 1023) / 1024 * 1024;
     static constexpr uint32_t kSbf = kStages * kStage;      // B operand of MMA1, MN-major: [128 dk rows][128 B]
     static constexpr uint32_t kVn = kSbf + 128 * 128;       // B operand of MMA2, MN-major: [64 token rows][128 B]
     static constexpr uint32_t kBars = kVn + 64 * 128;
     static constexpr uint32_t kTotal = kBars + 64;
     static constexpr uint32_t kSmem = kTotal + 1024;        // slack for manual 1024-byte alignment
-    static constexpr uint32_t kTxBytes = 32768 + 16384 + 8192 + kUBytes + 512;
+    static constexpr uint32_t kTxBytes = kMainBytes + kUBytes;
     static constexpr uint32_t kTmemCols = 128;              // D1 (two buffers) + D3, NS columns each
 };
 
@@ -69,8 +70,12 @@ __device__ __forceinline__ void store_row32(uint8_t* img, int row, const float (
                        pack2(x[8 * c + 4], x[8 * c + 5]), pack2(x[8 * c + 6], x[8 * c + 7]));
 }
 
+// Thread roles: warps 0-3 compute (TMEM lane quadrant = warp index; thread = token row for
+// V_new / O, thread = dk row for the state), warp 4 is the control warp whose lane 0 issues every
+// bulk copy and every MMA.  The roles meet only on mbarriers, so issue latencies never sit on the
+// compute warps' path and the output conversion overlaps the next chunk's first MMA.
 template <int NS>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(160, 1)
 kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader* hdr)
 {
     using Cfg = InterCfg<NS>;
@@ -78,9 +83,12 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + Cfg::kBars);        // [NSTG]
-    uint64_t* mma_bar = full + NSTG;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_bar + 1);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + Cfg::kBars);        // [NSTG] operands landed
+    uint64_t* mma1_bar = full + NSTG;      // MMA1 of a chunk complete
+    uint64_t* mma2_bar = mma1_bar + 1;     // MMA2 of a chunk complete
+    uint64_t* sbf_ready = mma2_bar + 1;    // 128 arrivals: bf16 state copy written (and stage reads done)
+    uint64_t* vn_ready = sbf_ready + 1;    // 64 arrivals: V_new written
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(vn_ready + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     uint8_t* sbf = smem + Cfg::kSbf;
     uint8_t* vn = smem + Cfg::kVn;
@@ -107,7 +115,10 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < NSTG; ++s) ptx::mbar_init(&full[s], 1);
-        ptx::mbar_init(mma_bar, 1);
+        ptx::mbar_init(mma1_bar, 1);
+        ptx::mbar_init(mma2_bar, 1);
+        ptx::mbar_init(sbf_ready, 128);
+        ptx::mbar_init(vn_ready, 64);
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -115,44 +126,11 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         ptx::tmem_alloc(tmem_slot, Cfg::kTmemCols);
         ptx::tmem_relinquish();
     }
-
-    auto issue_loads = [&](int it) {
-        const int s = it % NSTG;
-        const char* tile = tiles + ((size_t)(cb + it - a.g0) * a.H + h) * tc::TILE_BYTES;
-        uint8_t* sb = smem + s * Cfg::kStage;
-        ptx::mbar_expect_tx(&full[s], Cfg::kTxBytes);
-        ptx::bulk_g2s(sb + Cfg::kQW, tile + tc::OFF_QW, 32768, &full[s]);
-        ptx::bulk_g2s(sb + Cfg::kKT, tile + tc::OFF_KT, 16384, &full[s]);
-        ptx::bulk_g2s(sb + Cfg::kAQ, tile + tc::OFF_AQ, 8192, &full[s]);
-        ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 32) * tc::U_BLOCK,
-                      Cfg::kUBytes, &full[s]);
-        ptx::bulk_g2s(sb + Cfg::kGC, tile + tc::OFF_GC, 512, &full[s]);
-    };
-    int loads_issued = 0;
-    if (tid == 0) {   // the operand ring fills while the state is being read
-        ptx::fence_async_smem();
-        for (; loads_issued < NSTG && loads_issued < nchunks; ++loads_issued) issue_loads(loads_issued);
-    }
-
-    // state: fp32 master in registers (thread = dk row), bf16 copy as the B operand of MMA1
-    float S[NS];
-    const size_t sbase = ((size_t)n * a.H + h) * (size_t)(kD * kD) + (size_t)tid * kD + col0;
-#pragma unroll
-    for (int j = 0; j < NS; j += 4) {
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (a.S_in) x = *reinterpret_cast<const float4*>(a.S_in + sbase + j);
-        S[j] = x.x; S[j + 1] = x.y; S[j + 2] = x.z; S[j + 3] = x.w;
-    }
-    store_row32(sbf, tid, S);
-
-    ptx::fence_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
-    const uint32_t d3 = 2 * NS;   // column offsets: D1 buffers at 0 and NS, D3 at 2 NS
-    const uint32_t idesc = ptx::umma_idesc_bf16(128, NS) | ptx::kIdescBMajorMN;
+    const uint32_t d3 = 2 * NS;   // TMEM column offsets: D1 buffers at 0 and NS, D3 at 2 NS
 
     auto wait = [&](uint64_t* bar, uint32_t parity, int where) {
         if (*abort_flag) return;
@@ -161,125 +139,143 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             if (atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = where;
         }
     };
-    // MMA1(it): D1[it & 1] = [W ; Gamma.Q] S      (issued by thread 0 only)
-    auto issue_mma1 = [&](int it) {
-        const int s = it % NSTG;
-        wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);
-        ptx::tc_fence_after();
-        const uint32_t a0 = ptx::smem_u32(smem + s * Cfg::kStage + Cfg::kQW), b0 = ptx::smem_u32(sbf);
-        const uint32_t d1 = tmem_base + (uint32_t)(it & 1) * NS;
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-            ptx::umma_bf16(d1, ptx::umma_desc_sw128(a0 + (k >> 2) * tc::QW_HALF + (k & 3) * 32),
-                           ptx::umma_desc_sw128_mn(b0 + k * 2048, 8192), idesc, k > 0);
-        ptx::umma_commit(mma_bar);
-    };
 
-    KDA_PHASE(hdr, 16);  // set-up
-    if (tid == 0 && nchunks > 0) issue_mma1(0);
-    uint32_t mma_phase = 0;
-    int it = 0;
-    for (; it < nchunks; ++it) {
-        const int s = it % NSTG;
-        uint8_t* sb = smem + s * Cfg::kStage;
-        const uint32_t d1 = (uint32_t)(it & 1) * NS;
-        wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);   // U and gamma^C are read with plain loads
-        KDA_PHASE(hdr, 17);  // operand wait
-        wait(mma_bar, mma_phase, 2);
-        KDA_PHASE(hdr, 18);  // MMA1
-        mma_phase ^= 1;
-        ptx::tc_fence_after();
-
-        if (warp < 2) {   // a6: V_new = U - W S  (token row = tid)
-            uint32_t r[32];
-            ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
-            const uint4* up = reinterpret_cast<const uint4*>(sb + Cfg::kU + tid * 64);
-            uint4 uq[4] = {up[0], up[1], up[2], up[3]};
-            const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
-            ptx::tmem_ld_wait();
-            float x[32];
+    if (warp == 4) {
+        // ================= control warp: lane 0 issues all copies and MMAs =================
+        if (tid == 128) {
+            const uint32_t idesc = ptx::umma_idesc_bf16(128, NS) | ptx::kIdescBMajorMN;
+            const uint32_t sbf_a = ptx::smem_u32(sbf), vn_a = ptx::smem_u32(vn);
+            auto issue_loads = [&](int it) {
+                const int s = it % NSTG;
+                const char* tile = tiles + ((size_t)(cb + it - a.g0) * a.H + h) * tc::TILE_BYTES;
+                uint8_t* sb = smem + s * Cfg::kStage;
+                ptx::mbar_expect_tx(&full[s], Cfg::kTxBytes);
+                ptx::bulk_g2s(sb + Cfg::kQW, tile + tc::OFF_QW, Cfg::kMainBytes, &full[s]);
+                ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 32) * tc::U_BLOCK,
+                              Cfg::kUBytes, &full[s]);
+            };
+            int loads_issued = 0;
+            for (; loads_issued < NSTG && loads_issued < nchunks; ++loads_issued) issue_loads(loads_issued);
+            for (int it = 0; it < nchunks; ++it) {
+                const int s = it % NSTG;
+                const uint32_t sb = ptx::smem_u32(smem + s * Cfg::kStage);
+                const uint32_t d1 = tmem_base + (uint32_t)(it & 1) * NS;
+                // MMA1(it): D1 = [W ; Gamma.Q] S  -- needs this chunk's operands and the state copy
+                wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);
+                wait(sbf_ready, (uint32_t)it & 1u, 4);
+                ptx::tc_fence_after();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) x[j] = __bfloat162float(U[j]) - __uint_as_float(r[j]);
-            store_row32(vn, tid, x);
-        }
-        ptx::fence_async_smem();
-        ptx::tc_fence_before();
-        __syncthreads();
-        KDA_PHASE(hdr, 19);  // V_new
-
-        if (tid == 0) {   // MMA2: D1[64:128] += Aqk V_new,  D3 = Kt^T V_new
-            ptx::tc_fence_after();
-            // 128-row A operand whose rows 64-127 are Aqk; rows 0-63 (the tail of the Kt image) only
-            // touch accumulator rows 0-63, which are dead once V_new has been taken
-            const uint32_t aq = ptx::smem_u32(sb + Cfg::kAQ) - 8192, kt = ptx::smem_u32(sb + Cfg::kKT);
-            const uint32_t b0 = ptx::smem_u32(vn);
+                for (int k = 0; k < 8; ++k)
+                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kQW + (k >> 2) * tc::QW_HALF + (k & 3) * 32),
+                                   ptx::umma_desc_sw128_mn(sbf_a + k * 2048, 8192), idesc, k > 0);
+                ptx::umma_commit(mma1_bar);
+                // the stage of the previous chunk is free now (its readers arrived on sbf_ready)
+                if (it > 0 && loads_issued < nchunks) { issue_loads(loads_issued); ++loads_issued; }
+                // MMA2(it): D1[64:128] += Aqk V_new,  D3 = Kt^T V_new.  The 128-row A operand of the
+                // first product starts 64 rows before Aqk: those rows (the tail of the Kt image) only
+                // touch accumulator rows 0-63, which are dead once V_new has been taken.
+                wait(vn_ready, (uint32_t)it & 1u, 5);
+                ptx::tc_fence_after();
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                ptx::umma_bf16(tmem_base + d1, ptx::umma_desc_sw128(aq + k * 32),
-                               ptx::umma_desc_sw128_mn(b0 + k * 2048, 8192), idesc, 1);
+                for (int k = 0; k < 4; ++k)
+                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kAQ - 8192 + k * 32),
+                                   ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, 1);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                ptx::umma_bf16(tmem_base + d3, ptx::umma_desc_sw128(kt + k * 32),
-                               ptx::umma_desc_sw128_mn(b0 + k * 2048, 8192), idesc, k > 0);
-            ptx::umma_commit(mma_bar);
-        }
-        wait(mma_bar, mma_phase, 3);
-        KDA_PHASE(hdr, 20);  // MMA2
-        mma_phase ^= 1;
-        ptx::tc_fence_after();
-
-        {   // a8: S <- gamma^C . S + Kt^T V_new ; refresh the bf16 operand copy
-            const float gc = reinterpret_cast<const float*>(sb + Cfg::kGC)[tid];
-            uint32_t r[32];
-            ptx::tmem_ld_32x32b_x32(tmem_lane + d3, r);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) S[j] = gc * S[j] + __uint_as_float(r[j]);
-            store_row32(sbf, tid, S);
-        }
-        ptx::fence_async_smem();
-        ptx::tc_fence_before();
-        if (__syncthreads_or((int)*abort_flag)) break;
-        KDA_PHASE(hdr, 21);  // state update
-
-        if (tid == 0) {
-            if (it + 1 < nchunks) issue_mma1(it + 1);   // next chunk's first product starts now
-            KDA_PHASE(hdr, 23);
-            if (loads_issued < nchunks) { issue_loads(loads_issued); ++loads_issued; }   // stage s is free
-        }
-        if (warp >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64), overlaps MMA1
-            const int i = tid - 64;
-            const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
-            const int len = (tok_end - tok0) < kC ? (int)(tok_end - tok0) : kC;
-            __nv_bfloat16* orow = op + ((tok0 + i) * a.H + h) * kD + col0;
-            uint32_t r[32];
-            ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
-            ptx::tmem_ld_wait();
-            if (i < len) {
-#pragma unroll
-                for (int j = 0; j < 32; j += 8)
-                    *reinterpret_cast<uint4*>(orow + j) =
-                        make_uint4(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])),
-                                   pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])),
-                                   pack2(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])),
-                                   pack2(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
+                for (int k = 0; k < 4; ++k)
+                    ptx::umma_bf16(tmem_base + d3, ptx::umma_desc_sw128(sb + Cfg::kKT + k * 32),
+                                   ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, k > 0);
+                ptx::umma_commit(mma2_bar);
             }
-            ptx::tc_fence_before();
+            if (*abort_flag) {
+                // drain the bulk copies still in flight before the shared memory goes away
+                for (int j = (loads_issued > NSTG ? loads_issued - NSTG : 0); j < loads_issued; ++j)
+                    ptx::mbar_wait(&full[j % NSTG], (uint32_t)(j / NSTG) & 1u, kWaitLimitNs);
+            }
         }
-        KDA_PHASE(hdr, 22);  // issue + output
-    }
-
-    const bool aborted = *abort_flag != 0;
-    if (aborted && tid == 0) {
-        // drain the bulk copies this CTA still has in flight before its shared memory goes away
-        for (int j = (it > NSTG ? it - NSTG : 0); j < loads_issued; ++j)
-            ptx::mbar_wait(&full[j % NSTG], (uint32_t)(j / NSTG) & 1u, kWaitLimitNs);
-    }
-    if (!aborted) {
-        float* so = a.S_out + sbase;
+    } else {
+        // ================= compute warps =================
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+        // state: fp32 master in registers (thread = dk row), bf16 copy as the B operand of MMA1
+        float S[NS];
+        const size_t sbase = ((size_t)n * a.H + h) * (size_t)(kD * kD) + (size_t)tid * kD + col0;
 #pragma unroll
-        for (int j = 0; j < NS; j += 4)
-            *reinterpret_cast<float4*>(so + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
+        for (int j = 0; j < NS; j += 4) {
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (a.S_in) x = *reinterpret_cast<const float4*>(a.S_in + sbase + j);
+            S[j] = x.x; S[j + 1] = x.y; S[j + 2] = x.z; S[j + 3] = x.w;
+        }
+        store_row32(sbf, tid, S);
+        ptx::fence_async_smem();
+        ptx::mbar_arrive(sbf_ready);
+        KDA_PHASE(hdr, 16);  // set-up
+
+        for (int it = 0; it < nchunks; ++it) {
+            const int s = it % NSTG;
+            const uint8_t* sb = smem + s * Cfg::kStage;
+            const uint32_t d1 = (uint32_t)(it & 1) * NS;
+            const uint32_t par = (uint32_t)it & 1u;
+            wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);   // U and gamma^C are read with plain loads
+            if (warp < 2) {   // a6: V_new = U - W S  (token row = tid)
+                const uint4* up = reinterpret_cast<const uint4*>(sb + Cfg::kU + tid * 64);
+                uint4 uq[4] = {up[0], up[1], up[2], up[3]};
+                const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
+                wait(mma1_bar, par, 2);
+                KDA_PHASE(hdr, 18);  // MMA1
+                ptx::tc_fence_after();
+                uint32_t r[32];
+                ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
+                ptx::tmem_ld_wait();
+                float x[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[j] = __bfloat162float(U[j]) - __uint_as_float(r[j]);
+                store_row32(vn, tid, x);
+                ptx::fence_async_smem();
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(vn_ready);
+                KDA_PHASE(hdr, 19);  // V_new
+            }
+            const float gc = reinterpret_cast<const float*>(sb + Cfg::kGC)[tid];
+            wait(mma2_bar, par, 3);
+            KDA_PHASE(hdr, 20);  // MMA2
+            ptx::tc_fence_after();
+            {   // a8: S <- gamma^C . S + Kt^T V_new ; refresh the bf16 operand copy
+                uint32_t r[32];
+                ptx::tmem_ld_32x32b_x32(tmem_lane + d3, r);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) S[j] = gc * S[j] + __uint_as_float(r[j]);
+                store_row32(sbf, tid, S);
+            }
+            ptx::fence_async_smem();
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(sbf_ready);
+            KDA_PHASE(hdr, 21);  // state update
+            if (warp >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64)
+                const int i = tid - 64;
+                const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
+                const int len = (tok_end - tok0) < kC ? (int)(tok_end - tok0) : kC;
+                __nv_bfloat16* orow = op + ((tok0 + i) * a.H + h) * kD + col0;
+                uint32_t r[32];
+                ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
+                ptx::tmem_ld_wait();
+                if (i < len) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8)
+                        *reinterpret_cast<uint4*>(orow + j) =
+                            make_uint4(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])),
+                                       pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])),
+                                       pack2(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])),
+                                       pack2(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
+                }
+                ptx::tc_fence_before();
+            }
+        }
+        if (*abort_flag == 0) {
+            float* so = a.S_out + sbase;
+#pragma unroll
+            for (int j = 0; j < NS; j += 4)
+                *reinterpret_cast<float4*>(so + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
+        }
     }
     KDA_PHASE_FLUSH(hdr);
     ptx::tc_fence_before();
@@ -300,7 +296,7 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
     }
     dim3 grid(kD / NS, (unsigned)a.H, (unsigned)n_count);
     ProfScope ps(PROF_INTER, st);
-    kda_inter_tc<NS><<<grid, 128, Cfg::kSmem, st>>>(a, tiles, n_begin, hdr);
+    kda_inter_tc<NS><<<grid, 160, Cfg::kSmem, st>>>(a, tiles, n_begin, hdr);
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;

@@ -15,11 +15,11 @@ constexpr uint32_t QW_HALF = 128 * 128;
 constexpr uint32_t OFF_KT = 32768;
 // A operand of the intra-chunk output term: Aqk [64][64] (lower triangular incl. diagonal)
 constexpr uint32_t OFF_AQ = 49152;
+// gamma^C: 128 fp32 (directly after the three operand images: one bulk copy fetches all four)
+constexpr uint32_t OFF_GC = 57344;
 // U in four column blocks of [64 tokens][32 columns] bf16 (row-major inside a block)
-constexpr uint32_t OFF_U = 57344;
+constexpr uint32_t OFF_U = 57856;
 constexpr uint32_t U_BLOCK = 32 * 64 * 2;
-// gamma^C: 128 fp32
-constexpr uint32_t OFF_GC = 73728;
 constexpr uint32_t TILE_BYTES = 74240;
 static_assert(TILE_BYTES % 256 == 0, "tiles stay 256-byte aligned");
 }  // namespace tc
