@@ -12,9 +12,10 @@
 //   a2/a5  one tcgen05 MMA group  [Kg ; Qg] (128 x 128)  x  Ki^T (128 x 64)  ->  TMEM:
 //        rows 0-63  = raw key Gram matrix, rows 64-127 = raw query-key matrix
 //        L = Diag(beta) StrictTril(rows 0-63) (fp32, shared memory);  Aqk = Tril(rows 64-127)
-//   a3   T = (I + L)^-1 by blocked forward substitution in fp32: the four 16x16 diagonal blocks are
-//        inverted column by column in registers, then X = T_II L_IM for the six sub-diagonal blocks
-//        and three block levels  T_IJ = - sum_M X_IM T_MJ
+//   a3   T = (I + L)^-1 by blocked forward substitution: the four 16x16 diagonal blocks are
+//        inverted column by column in fp32 registers, then X = T_II L_IM for the six sub-diagonal
+//        blocks and three block levels  T_IJ = - sum_M X_IM T_MJ as warp-level 16x16 products
+//        (mma.sync, tf32 inputs, fp32 accumulation; T is rounded to bf16 afterwards anyway)
 //   a4   Mm = T Diag(beta) (bf16);  second MMA group  Mm (64 x 64) x [Kg | V] (64 x 256) -> TMEM;
 //        W = (Mm Kg) exp(G_m) column-wise,  U = Mm V.  Kg and V are used as MN-major B operands in
 //        the token-major layout they already have in shared memory.
@@ -22,6 +23,8 @@
 // kernel.  Tail chunks: rows past the sequence end behave as identity steps (log alpha = 0,
 // beta = 0, k = q = v = 0).
 #include <cuda.h>
+
+#include <type_traits>
 
 #include "kda_common.cuh"
 #include "kda_ptx.cuh"
@@ -65,6 +68,46 @@ __device__ __forceinline__ void ld_nc_f4(const float* p, float& a, float& b, flo
     asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
                  : "=f"(a), "=f"(b), "=f"(c), "=f"(d)
                  : "l"(p));
+}
+// 16x16 block products of the forward substitution on the legacy warp-level tensor path
+// (mma.sync m16n8k8, tf32 inputs rounded to nearest, fp32 accumulation): acc += A * B with A, B
+// 16x16 fp32 blocks in shared memory (row stride `ld` floats).
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void block16_mma(float (&acc)[2][4], const float* pa, const float* pb,
+                                            int ld, int lane) {
+    const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) {
+        const uint32_t a0 = to_tf32(pa[g * ld + ks * 8 + t4]);
+        const uint32_t a1 = to_tf32(pa[(g + 8) * ld + ks * 8 + t4]);
+        const uint32_t a2 = to_tf32(pa[g * ld + ks * 8 + t4 + 4]);
+        const uint32_t a3 = to_tf32(pa[(g + 8) * ld + ks * 8 + t4 + 4]);
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            const uint32_t b0 = to_tf32(pb[(ks * 8 + t4) * ld + nt * 8 + g]);
+            const uint32_t b1 = to_tf32(pb[(ks * 8 + t4 + 4) * ld + nt * 8 + g]);
+            asm volatile(
+                "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+                "{%8,%9}, {%0,%1,%2,%3};"
+                : "+f"(acc[nt][0]), "+f"(acc[nt][1]), "+f"(acc[nt][2]), "+f"(acc[nt][3])
+                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+        }
+    }
+}
+__device__ __forceinline__ void block16_store(float* pc, const float (&acc)[2][4], float sign, int ld,
+                                              int lane) {
+    const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+        *reinterpret_cast<float2*>(pc + g * ld + nt * 8 + 2 * t4) =
+            make_float2(sign * acc[nt][0], sign * acc[nt][1]);
+        *reinterpret_cast<float2*>(pc + (g + 8) * ld + nt * 8 + 2 * t4) =
+            make_float2(sign * acc[nt][2], sign * acc[nt][3]);
+    }
 }
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -224,58 +267,64 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     }
     const int hf = c4 >> 4;                       // K-half (channels 0-63 / 64-127)
     uint32_t ktb[4][4];                           // (K exp(G_C - G))^T: 4 channels x 8 tokens, bf16 pairs
+    auto gate_rows = [&](auto harsh_tag) {
+        constexpr bool kHarsh = decltype(harsh_tag)::value;
 #pragma unroll
-    for (int r = 0; r < 8; ++r) {
-        const int i = i0 + r;
-        const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
-        uint8_t* pk = smem + S_KQ + hf * S_KQ_HALF + off;
-        uint2 k2 = *reinterpret_cast<const uint2*>(pk);
-        uint2 q2 = *reinterpret_cast<const uint2*>(pk + 8192);
-        if (i >= L.len) k2 = q2 = make_uint2(0u, 0u);
-        if (!has_q) q2 = make_uint2(0u, 0u);
-        const float kf[4] = {__uint_as_float(k2.x << 16), __uint_as_float(k2.x & 0xffff0000u),
-                             __uint_as_float(k2.y << 16), __uint_as_float(k2.y & 0xffff0000u)};
-        const float qf[4] = {__uint_as_float(q2.x << 16), __uint_as_float(q2.x & 0xffff0000u),
-                             __uint_as_float(q2.y << 16), __uint_as_float(q2.y & 0xffff0000u)};
-        float okg[4], oqg[4], oki[4], oqt[4], okt[4];
+        for (int r = 0; r < 8; ++r) {
+            const int i = i0 + r;
+            const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
+            uint8_t* pk = smem + S_KQ + hf * S_KQ_HALF + off;
+            uint2 k2 = *reinterpret_cast<const uint2*>(pk);
+            uint2 q2 = *reinterpret_cast<const uint2*>(pk + 8192);
+            if (i >= L.len) k2 = q2 = make_uint2(0u, 0u);
+            if (!has_q) q2 = make_uint2(0u, 0u);
+            const float kf[4] = {__uint_as_float(k2.x << 16), __uint_as_float(k2.x & 0xffff0000u),
+                                 __uint_as_float(k2.y << 16), __uint_as_float(k2.y & 0xffff0000u)};
+            const float qf[4] = {__uint_as_float(q2.x << 16), __uint_as_float(q2.x & 0xffff0000u),
+                                 __uint_as_float(q2.y << 16), __uint_as_float(q2.y & 0xffff0000u)};
+            float okg[4], oqg[4], oki[4], oqt[4], okt[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float gg = G[r][e] + base[e];
-            const float x = fminf(fmaxf(gg - gref[e], -kClamp2), kClamp2);
-            const float e1 = ex2(x);                     // exp(G - G_m)
-            const float e2 = ex2(-x);                    // exp(G_m - G)
-            const float qs = a.scale * qf[e];
-            okg[e] = kf[e] * e1;
-            oqg[e] = qs * e1;
-            oki[e] = kf[e] * e2;
-            if (!harsh) {
-                oqt[e] = oqg[e] * cg[e];
-                okt[e] = oki[e] * ct[e];
+            for (int e = 0; e < 4; ++e) {
+                const float gg = G[r][e] + base[e];
+                const float x = fminf(fmaxf(gg - gref[e], -kClamp2), kClamp2);
+                const float e1 = ex2(x);                     // exp(G - G_m)
+                const float e2 = ex2(-x);                    // exp(G_m - G)
+                const float qs = a.scale * qf[e];
+                okg[e] = kf[e] * e1;
+                oqg[e] = qs * e1;
+                oki[e] = kf[e] * e2;
+                if (!kHarsh) {
+                    oqt[e] = oqg[e] * cg[e];
+                    okt[e] = oki[e] * ct[e];
+                } else {
+                    oqt[e] = qs * ex2(gg);
+                    okt[e] = kf[e] * ex2(glast[e] - gg);
+                }
+            }
+            *reinterpret_cast<uint2*>(pk) = make_uint2(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]));
+            *reinterpret_cast<uint2*>(pk + 8192) =
+                make_uint2(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]));
+            *reinterpret_cast<uint2*>(smem + S_KI + hf * S_KI_HALF + off) =
+                make_uint2(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]));
+            *reinterpret_cast<uint2*>(smem + S_QG + hf * 8192 + off) =
+                make_uint2(pack_bf16(oqt[0], oqt[1]), pack_bf16(oqt[2], oqt[3]));
+            if (r & 1) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    __nv_bfloat16 hi = __float2bfloat16_rn(okt[e]);
+                    ktb[e][r >> 1] |= (uint32_t)(*reinterpret_cast<uint16_t*>(&hi)) << 16;
+                }
             } else {
-                oqt[e] = qs * ex2(gg);
-                okt[e] = kf[e] * ex2(glast[e] - gg);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    __nv_bfloat16 lo = __float2bfloat16_rn(okt[e]);
+                    ktb[e][r >> 1] = (uint32_t)(*reinterpret_cast<uint16_t*>(&lo));
+                }
             }
         }
-        *reinterpret_cast<uint2*>(pk) = make_uint2(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]));
-        *reinterpret_cast<uint2*>(pk + 8192) = make_uint2(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]));
-        *reinterpret_cast<uint2*>(smem + S_KI + hf * S_KI_HALF + off) =
-            make_uint2(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]));
-        *reinterpret_cast<uint2*>(smem + S_QG + hf * 8192 + off) =
-            make_uint2(pack_bf16(oqt[0], oqt[1]), pack_bf16(oqt[2], oqt[3]));
-        if (r & 1) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                __nv_bfloat16 hi = __float2bfloat16_rn(okt[e]);
-                ktb[e][r >> 1] |= (uint32_t)(*reinterpret_cast<uint16_t*>(&hi)) << 16;
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                __nv_bfloat16 lo = __float2bfloat16_rn(okt[e]);
-                ktb[e][r >> 1] = (uint32_t)(*reinterpret_cast<uint16_t*>(&lo));
-            }
-        }
-    }
+    };
+    if (!harsh) gate_rows(std::false_type{});
+    else gate_rows(std::true_type{});
     // (K exp(G_C - G))^T: row = channel, this warp's 8 tokens are one 16-byte chunk
 #pragma unroll
     for (int e = 0; e < 4; ++e)
@@ -370,53 +419,25 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     }
     __syncthreads();
     KDA_PHASE(hdr, 4);   // diagonal blocks
-    {   // X_IM = T_II L_IM for the six sub-diagonal blocks (1x4 outputs per work item)
-        float xo[2][4];
-        int nitem = 0;
-        for (int item = t; item < 6 * 64; item += 256, ++nitem) {
-            const int blk = item >> 6, r = (item >> 2) & 15, cg = (item & 3) * 4;
-            const int I = blk < 1 ? 1 : (blk < 3 ? 2 : 3);
-            const int M = blk < 1 ? 0 : (blk < 3 ? blk - 1 : blk - 3);
-            const float* Tii = sT + (I * 16 + r) * LDT + I * 16;
-            const float* Lim = sA + (I * 16) * LDT + M * 16 + cg;
-            float o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
-#pragma unroll
-            for (int m = 0; m < 16; ++m) {
-                const float tv = Tii[m];
-                const float4 lv = *reinterpret_cast<const float4*>(Lim + m * LDT);
-                o0 += tv * lv.x; o1 += tv * lv.y; o2 += tv * lv.z; o3 += tv * lv.w;
-            }
-            xo[nitem][0] = o0; xo[nitem][1] = o1; xo[nitem][2] = o2; xo[nitem][3] = o3;
-        }
-        __syncthreads();
-        nitem = 0;
-        for (int item = t; item < 6 * 64; item += 256, ++nitem) {
-            const int blk = item >> 6, r = (item >> 2) & 15, cg = (item & 3) * 4;
-            const int I = blk < 1 ? 1 : (blk < 3 ? 2 : 3);
-            const int M = blk < 1 ? 0 : (blk < 3 ? blk - 1 : blk - 3);
-            *reinterpret_cast<float4*>(sA + (I * 16 + r) * LDT + M * 16 + cg) =
-                make_float4(xo[nitem][0], xo[nitem][1], xo[nitem][2], xo[nitem][3]);
-        }
+    if (warp < 6) {   // X_IM = T_II L_IM for the six sub-diagonal blocks, one warp each, in place
+        const int I = warp < 1 ? 1 : (warp < 3 ? 2 : 3);
+        const int M = warp < 1 ? 0 : (warp < 3 ? warp - 1 : warp - 3);
+        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        float* Lim = sA + (I * 16) * LDT + M * 16;
+        block16_mma(acc, sT + (I * 16) * LDT + I * 16, Lim, LDT, lane);
+        __syncwarp();   // every lane has read its part of L_IM before anyone overwrites it
+        block16_store(Lim, acc, 1.f, LDT, lane);
     }
     __syncthreads();
     KDA_PHASE(hdr, 5);   // X
 #pragma unroll
     for (int lvl = 1; lvl <= 3; ++lvl) {   // T_IJ = - sum_{M=J..I-1} X_IM T_MJ,  J = I - lvl
-        const int nblk = 4 - lvl;
-        if (t < nblk * 64) {
-            const int I = lvl + (t >> 6), J = I - lvl, r = (t >> 2) & 15, cg = (t & 3) * 4;
-            float o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
-            for (int M = J; M < I; ++M) {
-                const float* Xim = sA + (I * 16 + r) * LDT + M * 16;
-                const float* Tmj = sT + (M * 16) * LDT + J * 16 + cg;
-#pragma unroll
-                for (int m = 0; m < 16; ++m) {
-                    const float xv = Xim[m];
-                    const float4 tv = *reinterpret_cast<const float4*>(Tmj + m * LDT);
-                    o0 -= xv * tv.x; o1 -= xv * tv.y; o2 -= xv * tv.z; o3 -= xv * tv.w;
-                }
-            }
-            *reinterpret_cast<float4*>(sT + (I * 16 + r) * LDT + J * 16 + cg) = make_float4(o0, o1, o2, o3);
+        if (warp < 4 - lvl) {
+            const int I = lvl + warp, J = I - lvl;
+            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            for (int M = J; M < I; ++M)
+                block16_mma(acc, sA + (I * 16) * LDT + M * 16, sT + (M * 16) * LDT + J * 16, LDT, lane);
+            block16_store(sT + (I * 16) * LDT + J * 16, acc, -1.f, LDT, lane);
         }
         __syncthreads();
     }
