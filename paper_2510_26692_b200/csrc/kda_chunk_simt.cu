@@ -218,8 +218,8 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __re
                 const float uu[4] = {u[m].x, u[m].y, u[m].z, u[m].w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    st_bf16(tct + tc::OFF_U + ((c + e) >> 5) * tc::U_BLOCK +
-                                (i * 32 + ((c + e) & 31)) * 2, uu[e]);
+                    st_bf16(tct + tc::OFF_U + ((c + e) >> 6) * tc::U_IMAGE + ptx::sw128_off(i, (c + e) & 63),
+                            uu[e]);
             } else {
                 *reinterpret_cast<float4*>(tile + T_W + i * kD + c) = w[m];
                 *reinterpret_cast<float4*>(tile + T_U + i * kD + c) = u[m];

@@ -43,13 +43,13 @@ template <int NS> struct InterCfg {
     static constexpr uint32_t kAQ = 49152;                  // [64][64]; used as rows 64-127 of a 128-row operand
     static constexpr uint32_t kGC = 57344;                  // gamma^C, 128 fp32
     static constexpr uint32_t kMainBytes = 57856;           // QW | Kt | Aqk | gamma^C are contiguous in a tile
-    static constexpr uint32_t kU = 57856;                   // [64 tokens][NS]
-    static constexpr uint32_t kUBytes = 64 * NS * 2;
+    static constexpr uint32_t kU = 57856;                   // the [64 tokens][64 columns] image of U holding this slice
+    static constexpr uint32_t kUBytes = tc::U_IMAGE;
     static constexpr uint32_t kStage = (kU + kUBytes + 1023) / 1024 * 1024;
     static constexpr uint32_t kSbf = kStages * kStage;      // B operand of MMA1, MN-major: [128 dk rows][128 B]
     static constexpr uint32_t kVn = kSbf + 128 * 128;       // B operand of MMA2, MN-major: [64 token rows][128 B]
     static constexpr uint32_t kBars = kVn + 64 * 128;
-    static constexpr uint32_t kTotal = kBars + 64;
+    static constexpr uint32_t kTotal = kBars + 128;
     static constexpr uint32_t kSmem = kTotal + 1024;        // slack for manual 1024-byte alignment
     static constexpr uint32_t kTxBytes = kMainBytes + kUBytes;
     static constexpr uint32_t kTmemCols = 128;              // D1 (two buffers) + D3, NS columns each
@@ -86,7 +86,8 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + Cfg::kBars);        // [NSTG] operands landed
     uint64_t* mma1_bar = full + NSTG;      // MMA1 of a chunk complete
     uint64_t* mma2_bar = mma1_bar + 1;     // MMA2 of a chunk complete
-    uint64_t* sbf_ready = mma2_bar + 1;    // 128 arrivals: bf16 state copy written (and stage reads done)
+    uint64_t* out_bar = mma2_bar + 1;      // the output accumulator of a chunk is complete
+    uint64_t* sbf_ready = out_bar + 1;     // 128 arrivals: bf16 state copy written (and stage reads done)
     uint64_t* vn_ready = sbf_ready + 1;    // 64 arrivals: V_new written
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(vn_ready + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -117,6 +118,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         for (int s = 0; s < NSTG; ++s) ptx::mbar_init(&full[s], 1);
         ptx::mbar_init(mma1_bar, 1);
         ptx::mbar_init(mma2_bar, 1);
+        ptx::mbar_init(out_bar, 1);
         ptx::mbar_init(sbf_ready, 128);
         ptx::mbar_init(vn_ready, 64);
         *abort_flag = 0;
@@ -151,7 +153,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 uint8_t* sb = smem + s * Cfg::kStage;
                 ptx::mbar_expect_tx(&full[s], Cfg::kTxBytes);
                 ptx::bulk_g2s(sb + Cfg::kQW, tile + tc::OFF_QW, Cfg::kMainBytes, &full[s]);
-                ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 32) * tc::U_BLOCK,
+                ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 64) * tc::U_IMAGE,
                               Cfg::kUBytes, &full[s]);
             };
             int loads_issued = 0;
@@ -176,16 +178,19 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 // touch accumulator rows 0-63, which are dead once V_new has been taken.
                 wait(vn_ready, (uint32_t)it & 1u, 5);
                 ptx::tc_fence_after();
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kAQ - 8192 + k * 32),
-                                   ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, 1);
+                // the state product sits on the sequential chain: issue and commit it first
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     ptx::umma_bf16(tmem_base + d3, ptx::umma_desc_sw128(sb + Cfg::kKT + k * 32),
                                    ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, k > 0);
                 ptx::umma_commit(mma2_bar);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kAQ - 8192 + k * 32),
+                                   ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, 1);
+                ptx::umma_commit(out_bar);
             }
+            if (nchunks > 0) wait(out_bar, (uint32_t)(nchunks - 1) & 1u, 7);   // last output product done
             if (*abort_flag) {
                 // drain the bulk copies still in flight before the shared memory goes away
                 for (int j = (loads_issued > NSTG ? loads_issued - NSTG : 0); j < loads_issued; ++j)
@@ -216,8 +221,12 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             const uint32_t par = (uint32_t)it & 1u;
             wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);   // U and gamma^C are read with plain loads
             if (warp < 2) {   // a6: V_new = U - W S  (token row = tid)
-                const uint4* up = reinterpret_cast<const uint4*>(sb + Cfg::kU + tid * 64);
-                uint4 uq[4] = {up[0], up[1], up[2], up[3]};
+                const uint8_t* up = sb + Cfg::kU + tid * 128;   // this token's row of the swizzled image
+                const int c0 = (col0 & 63) >> 3;
+                uint4 uq[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    uq[c] = *reinterpret_cast<const uint4*>(up + (((c0 + c) ^ (tid & 7)) << 4));
                 const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
                 wait(mma1_bar, par, 2);
                 KDA_PHASE(hdr, 18);  // MMA1
@@ -255,6 +264,8 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
                 const int len = (tok_end - tok0) < kC ? (int)(tok_end - tok0) : kC;
                 __nv_bfloat16* orow = op + ((tok0 + i) * a.H + h) * kD + col0;
+                wait(out_bar, par, 6);
+                ptx::tc_fence_after();
                 uint32_t r[32];
                 ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
                 ptx::tmem_ld_wait();

@@ -16,7 +16,8 @@
 //        inverted column by column in fp32 registers, then X = T_II L_IM for the six sub-diagonal
 //        blocks and three block levels  T_IJ = - sum_M X_IM T_MJ as warp-level 16x16 products
 //        (mma.sync, tf32 inputs, fp32 accumulation; T is rounded to bf16 afterwards anyway)
-//   a4   Mm = T Diag(beta) (bf16);  second MMA group  Mm (64 x 64) x [Kg | V] (64 x 256) -> TMEM;
+//   a4   Mm = T Diag(beta) (bf16);  second MMA group  [Mm ; Mm] (128 x 64) x [Kg | V] (64 x 256) -> TMEM
+//        (the rows are held twice so that all 128 TMEM lanes, i.e. all eight warps, share the read-out);
 //        W = (Mm Kg) exp(G_m) column-wise,  U = Mm V.  Kg and V are used as MN-major B operands in
 //        the token-major layout they already have in shared memory.
 // Outputs go to the scratch tile of kda_tiles.cuh as ready-made operand images of the inter-chunk
@@ -24,6 +25,7 @@
 // beta = 0, k = q = v = 0).
 #include <cuda.h>
 
+#include <cstdlib>
 #include <type_traits>
 
 #include "kda_common.cuh"
@@ -43,20 +45,22 @@ constexpr uint32_t S_KI = 32768;      // [2 K-halves][64][64] bf16
 constexpr uint32_t S_KI_HALF = 8192;
 constexpr uint32_t S_V = 49152;       // [2 column blocks][64 tokens][64] bf16 (token-major)
 constexpr uint32_t S_V_BLOCK = 8192;
-constexpr uint32_t S_M = 65536;       // [64][64] bf16: T Diag(beta)
+constexpr uint32_t S_M = 65536;       // 8 KiB: Aqk staging; start of the 32 KiB output staging area
 constexpr uint32_t S_A = 73728;       // fp32 [64][LDT]: L, later X in its sub-diagonal blocks
 constexpr uint32_t S_T = S_A + 64 * LDT * 4;   // fp32 [64][LDT]: T
 // staging of outputs for bulk stores (aliases buffers that are dead at the time):
 constexpr uint32_t S_QG = S_M;                 // scale Q exp(G): [2 halves][64][64] bf16, 16 KiB   (phase 1)
 constexpr uint32_t S_KT = S_M + 16384;         // (K exp(G_C - G))^T: [128][64] bf16, 16 KiB        (phase 1)
 constexpr uint32_t S_TOT = S_M + 32768;        // scan exchange [8][128] fp32, 4 KiB
-constexpr uint32_t S_AQ = S_KI;                // Aqk image [64][64] bf16 (after the first MMA group)
+constexpr uint32_t S_AQ = S_M;                 // Aqk image [64][64] bf16 (after the first MMA group)
+constexpr uint32_t S_MM = S_KI;                // [128][64] bf16: T Diag(beta) twice (rows 64-127 repeat rows 0-63)
 constexpr uint32_t S_W = S_M;                  // W image [2 halves][64][64] bf16 (after the second group)
-constexpr uint32_t S_U = S_M + 16384;          // U [4 blocks][64][32] bf16
+constexpr uint32_t S_U = S_M + 16384;          // U: two [64][64] bf16 images
 constexpr uint32_t S_BETA = S_T + 64 * LDT * 4;
 constexpr uint32_t S_CG = S_BETA + 256;        // exp(G_m) per channel (undoes the Kg reference)
 constexpr uint32_t S_BAR = S_CG + 512;          // mma barrier, tma barrier, TMEM slot
 constexpr uint32_t S_TOTAL = S_BAR + 64;
+constexpr int kBulkThread = 128;   // lane 0 of warp 4 issues every bulk copy; thread 0 issues the MMAs
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kClamp2 = 80.f * 1.4426950408889634f;   // the +-80 clamp in the log2 domain
 constexpr uint32_t kIntraTcSmem = S_TOTAL + 1024;
@@ -175,7 +179,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
                 G[r][0] = G[r][1] = G[r][2] = G[r][3] = 0.f;
             }
         }
-        if (t == 0) {
+        if (t == kBulkThread) {
             ptx::mbar_expect_tx(tma_bar, 3 * 16384);
             const int x = ho * kD, y = (int)Lo.tok0;
 #pragma unroll
@@ -220,7 +224,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
 #pragma unroll
         for (int e = 0; e < 4; ++e) G[r][e] = fmaf(G[r][e], kLog2e, G[r - 1][e]);
     *reinterpret_cast<float4*>(sTot + warp * kD + d0) = make_float4(G[7][0], G[7][1], G[7][2], G[7][3]);
-    if (t == 0) ptx::bulk_wait_read0();   // the previous tile's output staging has been read out
+    if (t == kBulkThread) ptx::bulk_wait_read0();   // the previous tile's output staging has been read out
     ptx::cp_async_wait_all();             // beta
     __syncthreads();
     KDA_PHASE(hdr, 0);   // loads arrived + local scan
@@ -339,12 +343,14 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     ptx::tc_fence_after();
 
     // ---- a2 + a5: [Kg ; Qg] Ki^T ------------------------------------------------------------------------
-    if (t == 0) {
+    if (t == kBulkThread) {
         // phase-1 outputs leave through the TMA engine while the MMA runs
         ptx::bulk_s2g(tile + tc::OFF_QW + 8192, smem + S_QG, 8192);
         ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF + 8192, smem + S_QG + 8192, 8192);
         ptx::bulk_s2g(tile + tc::OFF_KT, smem + S_KT, 16384);
         ptx::bulk_commit();
+    }
+    if (t == 0) {
         const uint32_t idesc = ptx::umma_idesc_bf16(128, 64);
         const uint32_t a0 = ptx::smem_u32(smem + S_KQ), b0 = ptx::smem_u32(smem + S_KI);
 #pragma unroll
@@ -354,7 +360,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         ptx::umma_commit(mma_bar);
     }
     if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) timed_out = true;
-    if (t == 0) ptx::bulk_wait_read0();   // staging buffers are about to be reused
+    if (t == kBulkThread) ptx::bulk_wait_read0();   // staging buffers are about to be reused
     __syncthreads();
     KDA_PHASE(hdr, 2);   // first MMA group
     ptx::tc_fence_after();
@@ -396,7 +402,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     ptx::fence_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
-    if (t == 0) {
+    if (t == kBulkThread) {
         ptx::bulk_s2g(tile + tc::OFF_AQ, smem + S_AQ, 8192);
         ptx::bulk_commit();
     }
@@ -459,19 +465,23 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
             }
         }
 #pragma unroll
-        for (int c8 = 0; c8 < 2; ++c8)
-            *reinterpret_cast<uint4*>(smem + S_M + i * 128 + ((((jq * 2 + c8) ^ (i & 7))) << 4)) =
-                make_uint4(pack_bf16(x[c8 * 8], x[c8 * 8 + 1]), pack_bf16(x[c8 * 8 + 2], x[c8 * 8 + 3]),
-                           pack_bf16(x[c8 * 8 + 4], x[c8 * 8 + 5]), pack_bf16(x[c8 * 8 + 6], x[c8 * 8 + 7]));
+        for (int c8 = 0; c8 < 2; ++c8) {
+            const uint4 pk = make_uint4(pack_bf16(x[c8 * 8], x[c8 * 8 + 1]), pack_bf16(x[c8 * 8 + 2], x[c8 * 8 + 3]),
+                                        pack_bf16(x[c8 * 8 + 4], x[c8 * 8 + 5]), pack_bf16(x[c8 * 8 + 6], x[c8 * 8 + 7]));
+            uint8_t* dst = smem + S_MM + i * 128 + ((((jq * 2 + c8) ^ (i & 7))) << 4);
+            *reinterpret_cast<uint4*>(dst) = pk;
+            *reinterpret_cast<uint4*>(dst + 8192) = pk;   // rows 64-127 repeat rows 0-63
+        }
     }
+    if (t == kBulkThread) ptx::bulk_wait_read0();   // Aqk staging is reused by the W/U epilogue
     ptx::fence_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
     KDA_PHASE(hdr, 7);   // Mm
     if (t == 0) {
         ptx::tc_fence_after();
-        const uint32_t idesc = ptx::umma_idesc_bf16(64, 128) | ptx::kIdescBMajorMN;
-        const uint32_t m0 = ptx::smem_u32(smem + S_M);
+        const uint32_t idesc = ptx::umma_idesc_bf16(128, 128) | ptx::kIdescBMajorMN;
+        const uint32_t m0 = ptx::smem_u32(smem + S_MM);
         const uint32_t kg0 = ptx::smem_u32(smem + S_KQ), v0 = ptx::smem_u32(smem + S_V);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
@@ -490,45 +500,45 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     }
     KDA_PHASE(hdr, 8);   // second MMA group
     ptx::tc_fence_after();
-    {   // M = 64 accumulator: row i sits in TMEM lane 32 (i / 16) + i % 16
-        const int q4 = warp & 3, part = warp >> 2;   // part 0: W (columns 0-127), part 1: U
-        const int i = q4 * 16 + (lane & 15);
-        const bool valid = lane < 16;
+    {   // The A operand held every row twice, so TMEM lanes 0-63 and 64-127 both carry rows 0-63:
+        // warp (q4, part) converts rows 32 (q4 & 1) + lane of the 64-column block cb of [W | U].
+        const int q4 = warp & 3, cb = (warp >> 2) * 2 + (q4 >> 1);
+        const int i = (q4 & 1) * 32 + lane;
+        uint32_t r0[32], r1[32];
+        const uint32_t ta = tmem_base + ((uint32_t)(q4 * 32) << 16) + cb * 64;
+        ptx::tmem_ld_32x32b_x32(ta, r0);
+        ptx::tmem_ld_32x32b_x32(ta + 32, r1);
+        ptx::tmem_ld_wait();
+        if (cb < 2) {   // W = (Mm Kg) exp(G_m): K-half cb of the [W ; Gamma.Q] image
+            uint8_t* dst = smem + S_W + cb * 8192;
 #pragma unroll
-        for (int blk = 0; blk < 4; ++blk) {
-            uint32_t r[32];
-            ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q4 * 32) << 16) + part * 128 + blk * 32, r);
-            ptx::tmem_ld_wait();
-            if (valid) {
-                if (part == 0) {
-                    uint8_t* dst = smem + S_W + (blk >> 1) * 8192;
+            for (int j8 = 0; j8 < 64; j8 += 8) {
+                const float4 s0 = *reinterpret_cast<const float4*>(sCG + cb * 64 + j8);
+                const float4 s1 = *reinterpret_cast<const float4*>(sCG + cb * 64 + j8 + 4);
+                const uint32_t* r = j8 < 32 ? r0 + j8 : r1 + (j8 - 32);
+                *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, j8)) =
+                    make_uint4(pack_bf16(__uint_as_float(r[0]) * s0.x, __uint_as_float(r[1]) * s0.y),
+                               pack_bf16(__uint_as_float(r[2]) * s0.z, __uint_as_float(r[3]) * s0.w),
+                               pack_bf16(__uint_as_float(r[4]) * s1.x, __uint_as_float(r[5]) * s1.y),
+                               pack_bf16(__uint_as_float(r[6]) * s1.z, __uint_as_float(r[7]) * s1.w));
+            }
+        } else {        // U: image cb - 2
+            uint8_t* dst = smem + S_U + (cb - 2) * tc::U_IMAGE;
 #pragma unroll
-                    for (int j8 = 0; j8 < 32; j8 += 8) {
-                        float x[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            x[e] = __uint_as_float(r[j8 + e]) * sCG[blk * 32 + j8 + e];
-                        *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, (blk & 1) * 32 + j8)) =
-                            make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]),
-                                       pack_bf16(x[6], x[7]));
-                    }
-                } else {
-                    uint8_t* dst = smem + S_U + blk * tc::U_BLOCK + i * 64;
-#pragma unroll
-                    for (int j8 = 0; j8 < 32; j8 += 8)
-                        *reinterpret_cast<uint4*>(dst + j8 * 2) =
-                            make_uint4(pack_bf16(__uint_as_float(r[j8]), __uint_as_float(r[j8 + 1])),
-                                       pack_bf16(__uint_as_float(r[j8 + 2]), __uint_as_float(r[j8 + 3])),
-                                       pack_bf16(__uint_as_float(r[j8 + 4]), __uint_as_float(r[j8 + 5])),
-                                       pack_bf16(__uint_as_float(r[j8 + 6]), __uint_as_float(r[j8 + 7])));
-                }
+            for (int j8 = 0; j8 < 64; j8 += 8) {
+                const uint32_t* r = j8 < 32 ? r0 + j8 : r1 + (j8 - 32);
+                *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, j8)) =
+                    make_uint4(pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1])),
+                               pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3])),
+                               pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5])),
+                               pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7])));
             }
         }
     }
     ptx::fence_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
-    if (t == 0) {
+    if (t == kBulkThread) {
         ptx::bulk_s2g(tile + tc::OFF_QW, smem + S_W, 8192);
         ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF, smem + S_W + 8192, 8192);
         ptx::bulk_s2g(tile + tc::OFF_U, smem + S_U, 16384);
@@ -541,7 +551,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
 
     if (timed_out && atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = 10;
     KDA_PHASE_FLUSH(hdr);
-    if (t == 0) ptx::bulk_wait_read0();   // shared memory must outlive the reads of every bulk store
+    if (t == kBulkThread) ptx::bulk_wait_read0();   // shared memory must outlive the reads of every bulk store
     ptx::cp_async_wait_all();
     ptx::tc_fence_before();
     __syncthreads();
@@ -609,7 +619,8 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cud
     if (rc == KDA_OK) rc = make_tmap(&tm_v, a.v, a.total_tokens, a.H);
     if (rc == KDA_OK) rc = make_tmap(&tm_q, a.q ? a.q : a.k, a.total_tokens, a.H);
     if (rc != KDA_OK) return rc;
-    const int64_t resident = 2 * (int64_t)n_sm;   // two CTAs per SM
+    static const int per_sm = getenv("KDA_INTRA_CTAS_PER_SM") ? atoi(getenv("KDA_INTRA_CTAS_PER_SM")) : 2;
+    const int64_t resident = per_sm * (int64_t)n_sm;   // two CTAs per SM
     const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
     ProfScope ps(PROF_INTRA, st);
     kda_intra_tc<<<grid, 256, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, a.q ? 1 : 0);

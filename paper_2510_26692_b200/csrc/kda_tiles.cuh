@@ -17,9 +17,10 @@ constexpr uint32_t OFF_KT = 32768;
 constexpr uint32_t OFF_AQ = 49152;
 // gamma^C: 128 fp32 (directly after the three operand images: one bulk copy fetches all four)
 constexpr uint32_t OFF_GC = 57344;
-// U in four column blocks of [64 tokens][32 columns] bf16 (row-major inside a block)
+// U as two [64 tokens][64 columns] bf16 images in the same 128-byte-swizzled row layout (it is
+// read with plain loads, the swizzle only keeps the producer's stores free of bank conflicts)
 constexpr uint32_t OFF_U = 57856;
-constexpr uint32_t U_BLOCK = 32 * 64 * 2;
+constexpr uint32_t U_IMAGE = 64 * 128;
 constexpr uint32_t TILE_BYTES = 74240;
 static_assert(TILE_BYTES % 256 == 0, "tiles stay 256-byte aligned");
 }  // namespace tc
