@@ -36,6 +36,10 @@ STATE_BYTES = 2 * D * D * 4
 # decode: state read + written, q,k,v,o bf16, gates fp32, beta
 DEC_BYTES_PER_STATE = 2 * D * D * 4 + 4 * D * 2 + D * 4 + 4
 FLOPS_PER_TOKEN_HEAD = 6 * D * D + 3 * CHUNK * D + CHUNK * CHUNK   # the paper's FLOPs model
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (prefill: intra 168.7 + 98.2 MB, inter 154.2 + 19.6 MB; decode: 547.4 + 484.7 MB)
+PREFILL_DRAM_TRAFFIC = {"intra_chunk": 266.9e6, "inter_chunk": 173.8e6}
+DECODE_DRAM_TRAFFIC = 1032.1e6
 
 
 def load_peaks():
@@ -161,6 +165,60 @@ def oracle_arm(args, rank):
     return 0
 
 
+def extra_workloads(K, inputs, torch, dev, peaks):
+    """Device-resident timing of the packed varlen batch (BASELINE configs[2]) and of the 1 Mi-token
+    state-only prefill (configs[3]); inputs are far larger than L2, so no rotation is needed."""
+    out = {}
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    # varlen: 16 sequences, lengths uniform on [512, 16384]
+    lens = inputs.varlen_lengths(16, 512, 16384, seed=2)
+    d = inputs.chunk_inputs(lens, H=H, dtype=torch.bfloat16, seed=2, s0_std=0.02, device=dev)
+    T = sum(lens)
+    cu_host = d["cu_seqlens"]
+    cu_dev = cu_host.to(dev)
+    nb = K.kda_chunk_fwd_workspace_bytes(T, 16, H, D, D, CHUNK, K.KDA_BF16)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    o = torch.empty((T, H, D), dtype=torch.bfloat16, device=dev)
+    S_T = torch.empty((16, H, D, D), dtype=torch.float32, device=dev)
+    ms = timed(lambda: K.kda_chunk_fwd(d["q"], d["k"], d["v"], d["log_alpha"], d["beta"], d["S0"], o,
+                                       S_T, cu_dev, cu_host, 16, T, H, D, D, CHUNK, 1.0, K.KDA_BF16,
+                                       ws, nb, stream), 10)
+    nbytes = T * H * BYTES_PER_TOKEN_HEAD + 16 * H * STATE_BYTES
+    out["varlen_16seq"] = {"total_tokens": T, "lengths": lens, "ms": ms, "tokens_per_s": T / (ms * 1e-3),
+                           "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    del d, ws, o, S_T
+    torch.cuda.empty_cache()
+
+    # long context: 1 Mi tokens, final state only (o = NULL, q unused)
+    T = 1 << 20
+    d = inputs.chunk_inputs_slabbed(T, H, seed=3, gate_mean=6.0, s0_std=0.02, device=dev, want_q=False)
+    nb = K.kda_chunk_fwd_workspace_bytes(T, 1, H, D, D, CHUNK, K.KDA_BF16)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    S_T = torch.empty((1, H, D, D), dtype=torch.float32, device=dev)
+    ms = timed(lambda: K.kda_chunk_fwd(None, d["k"], d["v"], d["log_alpha"], d["beta"], d["S0"], None,
+                                       S_T, None, None, 1, T, H, D, D, CHUNK, 1.0, K.KDA_BF16, ws, nb,
+                                       stream), 3)
+    nbytes = T * H * 1028 + H * STATE_BYTES     # k, v, gates, beta; no q, no o
+    out["long_context_1Mi_state_only"] = {"total_tokens": T, "ms": ms, "tokens_per_s": T / (ms * 1e-3),
+                                          "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    del d, ws, S_T
+    torch.cuda.empty_cache()
+    return out
+
+
 def decode_only(args, K, inputs, torch, dev, peaks):
     """Short decode-only run (used under a profiler): one block of 64 in-place steps, timed."""
     dd = inputs.decode_inputs(DEC_SEQS, H, DEC_STEPS, seed=4)
@@ -193,6 +251,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-reps", type=int, default=5)
+    ap.add_argument("--all-workloads", action="store_true",
+                    help="also time the packed varlen batch (16 sequences) and the 1 Mi-token "
+                         "state-only prefill; needs ~70 GB of device memory")
     ap.add_argument("--prefill-only", action="store_true",
                     help="time only the device-resident prefill loop (short runs under a profiler)")
     ap.add_argument("--decode-only", action="store_true",
@@ -287,7 +348,8 @@ def main():
         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
         "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "peak_source": peaks["source"],
         "frac_of_8TBs_nominal": (achieved / 8000.0) if achieved else None,
-        "algorithmic_bytes_per_step": step_bytes, "traffic": None, "kernels": kern,
+        "algorithmic_bytes_per_step": step_bytes, "traffic": sum(PREFILL_DRAM_TRAFFIC.values()),
+        "traffic_per_kernel": PREFILL_DRAM_TRAFFIC, "kernels": kern,
         "tensor_bound_tokens_per_s": peaks["bf16_tflops"] * 1e12 / (H * FLOPS_PER_TOKEN_HEAD),
         "hbm_bound_tokens_per_s": peaks["hbm_gbs"] * 1e9 / (step_bytes / T_PREFILL),
         "note": "HBM is the slower bound at d=128, C=64; the tensor-pipe bound is above it",
@@ -360,8 +422,13 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "kda_decode_kernel", "achieved": dec_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"],
                      "peak_source": peaks["source"], "frac_of_8TBs_nominal": dec_gbs / 8000.0,
-                     "algorithmic_bytes_per_step": dec_bytes, "traffic": None},
+                     "algorithmic_bytes_per_step": dec_bytes, "traffic": DECODE_DRAM_TRAFFIC},
     }
+
+    # ---- the other prefill workloads (on request) ----------------------------------------------------
+    other = None
+    if args.all_workloads and world == 1:
+        other = extra_workloads(K, inputs, torch, dev, peaks)
 
     # ---- CPU oracle beside it (rank 0, single-GPU runs only) --------------------------------------
     cpu = None
@@ -398,6 +465,8 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
             "decode": decode, "cpu_baseline": cpu,
         }
+        if other is not None:
+            line["other_workloads"] = other
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

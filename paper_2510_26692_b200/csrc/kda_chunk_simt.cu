@@ -17,8 +17,6 @@
 // exp(G_i - G_m) * exp(G_m - G_j), with each exponent clamped to [-80, 80], so no product
 // overflows fp32; entries above the diagonal are never used (selected to zero, not multiplied).
 #include "kda_common.cuh"
-#include "kda_ptx.cuh"
-#include "kda_tiles.cuh"
 
 namespace kda {
 namespace {
@@ -44,17 +42,8 @@ constexpr size_t kInterSmem =
 
 __device__ __forceinline__ float clampf(float x) { return fminf(fmaxf(x, -kClamp), kClamp); }
 
-__device__ __forceinline__ void st_bf16x4(char* p, float a, float b, float c, float d) {
-    IO<__nv_bfloat16>::store4(reinterpret_cast<__nv_bfloat16*>(p), make_float4(a, b, c, d));
-}
-__device__ __forceinline__ void st_bf16(char* p, float a) {
-    *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(a);
-}
-
-// kTc = false: fp32 scratch tile for kda_inter_simt.  kTc = true: the bf16 operand-image tile of
-// kda_tiles.cuh for the tensor-core inter-chunk kernel (same arithmetic, different store layout).
-template <typename T, bool kTc>
-__global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __restrict__ tiles_v)
+template <typename T>
+__global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, float* __restrict__ tiles)
 {
     extern __shared__ __align__(16) float smem[];
     float* sG = smem;                    // log-decay cumsum, later V
@@ -73,9 +62,7 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __re
     const T* qp = reinterpret_cast<const T*>(a.q);
     const T* kp = reinterpret_cast<const T*>(a.k);
     const T* vp = reinterpret_cast<const T*>(a.v);
-    const size_t tile_idx = (size_t)(g - a.g0) * a.H + h;
-    float* tile = reinterpret_cast<float*>(tiles_v) + (kTc ? 0 : tile_idx * T_FLOATS);
-    char* tct = reinterpret_cast<char*>(tiles_v) + (kTc ? tile_idx * tc::TILE_BYTES : 0);
+    float* tile = tiles + ((size_t)(g - a.g0) * a.H + h) * T_FLOATS;
 
     // a1: load log alpha (identity padding past the sequence end), then scan over the tokens
     for (int idx = t; idx < kC * (kD / 4); idx += 256) {
@@ -128,15 +115,7 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __re
         *reinterpret_cast<float4*>(sKi + i * LD + c) = make_float4(oki[0], oki[1], oki[2], oki[3]);
         *reinterpret_cast<float4*>(sQg + i * LD + c) = make_float4(oqg[0], oqg[1], oqg[2], oqg[3]);
         *reinterpret_cast<float4*>(sKG + i * LD + c) = make_float4(oKG[0], oKG[1], oKG[2], oKG[3]);
-        if (kTc) {
-            st_bf16x4(tct + tc::OFF_QW + (c >> 6) * tc::QW_HALF + ptx::sw128_off(64 + i, c & 63), oQG[0],
-                      oQG[1], oQG[2], oQG[3]);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) st_bf16(tct + tc::OFF_KT + ptx::sw128_off(c + e, i), oKT[e]);
-            if (i == 0)
-                *reinterpret_cast<float4*>(tct + tc::OFF_GC + c * 4) =
-                    make_float4(ogc[0], ogc[1], ogc[2], ogc[3]);
-        } else {
+        {
             *reinterpret_cast<float4*>(tile + T_QG + i * kD + c) =
                 make_float4(oQG[0], oQG[1], oQG[2], oQG[3]);
             *reinterpret_cast<float4*>(tile + T_KT + i * kD + c) =
@@ -175,8 +154,7 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __re
                 }
             }
             sA[i * LDA + j] = (j < i) ? bi * akk : 0.f;
-            if (kTc) st_bf16(tct + tc::OFF_AQ + ptx::sw128_off(i, j), aqk);
-            else tile[T_AQK + i * kC + j] = aqk;
+            tile[T_AQK + i * kC + j] = aqk;
         }
     }
     __syncthreads();
@@ -212,15 +190,7 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, void* __re
 #pragma unroll
         for (int m = 0; m < 8; ++m) {
             const int c = cq * 4 + 16 * m;
-            if (kTc) {
-                st_bf16x4(tct + tc::OFF_QW + (c >> 6) * tc::QW_HALF + ptx::sw128_off(i, c & 63),
-                          w[m].x, w[m].y, w[m].z, w[m].w);
-                const float uu[4] = {u[m].x, u[m].y, u[m].z, u[m].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    st_bf16(tct + tc::OFF_U + ((c + e) >> 6) * tc::U_IMAGE + ptx::sw128_off(i, (c + e) & 63),
-                            uu[e]);
-            } else {
+            {
                 *reinterpret_cast<float4*>(tile + T_W + i * kD + c) = w[m];
                 *reinterpret_cast<float4*>(tile + T_U + i * kD + c) = u[m];
             }
@@ -363,7 +333,7 @@ kda_status_t launch_simt_t(const ChunkArgs& a, float* tiles, int n_begin, int n_
 {
     static bool attr_done = false;   // per dtype instantiation
     if (!attr_done) {
-        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_simt<T, false>,
+        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_simt<T>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)kIntraSmem));
         KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_simt<T>,
@@ -375,7 +345,7 @@ kda_status_t launch_simt_t(const ChunkArgs& a, float* tiles, int n_begin, int n_
     if (n_chunks > 0) {
         dim3 grid((unsigned)n_chunks, (unsigned)a.H);
         ProfScope ps(PROF_INTRA, st);
-        kda_intra_simt<T, false><<<grid, 256, kIntraSmem, st>>>(a, tiles);
+        kda_intra_simt<T><<<grid, 256, kIntraSmem, st>>>(a, tiles);
         count_launch();
         KDA_CUDA_TRY(cudaGetLastError());
     }
@@ -398,27 +368,6 @@ kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, 
 {
     if (dt == KDA_BF16) return launch_simt_t<__nv_bfloat16>(a, (float*)tiles, n_begin, n_count, st);
     return launch_simt_t<float>(a, (float*)tiles, n_begin, n_count, st);
-}
-
-// fp32-FMA intra-chunk stage writing the tensor-core tile format (bf16 storage only)
-kda_status_t launch_intra_fma_tc(const ChunkArgs& a, void* tiles, cudaStream_t st)
-{
-    using T = __nv_bfloat16;
-    static bool attr_done = false;
-    if (!attr_done) {
-        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_simt<T, true>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)kIntraSmem));
-        attr_done = true;
-    }
-    const int64_t n_chunks = a.g1 - a.g0;
-    if (n_chunks <= 0) return KDA_OK;
-    dim3 grid((unsigned)n_chunks, (unsigned)a.H);
-    ProfScope ps(PROF_INTRA, st);
-    kda_intra_simt<T, true><<<grid, 256, kIntraSmem, st>>>(a, tiles);
-    count_launch();
-    KDA_CUDA_TRY(cudaGetLastError());
-    return KDA_OK;
 }
 
 kda_status_t launch_prep(WsHeader* hdr, const int32_t* cu_seqlens, int32_t* chunk_cu, int n_seqs,

@@ -20,15 +20,12 @@
 // TMEM, read back with tcgen05.ld.
 // Every wait is bounded: on a timeout the CTA records KDA_ERR_TIMEOUT in the workspace header,
 // drains its copies, frees its TMEM and returns.
-#include <cstdlib>
-
 #include "kda_common.cuh"
 #include "kda_ptx.cuh"
 #include "kda_tiles.cuh"
 
 namespace kda {
 
-kda_status_t launch_intra_fma_tc(const ChunkArgs& a, void* tiles, cudaStream_t st);
 kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cudaStream_t st);
 
 namespace {
@@ -320,8 +317,7 @@ size_t tc_tile_bytes() { return tc::TILE_BYTES; }
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
                              WsHeader* hdr, cudaStream_t st)
 {
-    static const bool fma_intra = getenv("KDA_INTRA_FMA") != nullptr;   // debugging aid
-    kda_status_t rc = fma_intra ? launch_intra_fma_tc(a, tiles, st) : launch_intra_tc(a, tiles, hdr, st);
+    kda_status_t rc = launch_intra_tc(a, tiles, hdr, st);
     if (rc != KDA_OK) return rc;
     if (n_count <= 0) return KDA_OK;
     return launch_inter_tc_t<32>(a, (const char*)tiles, n_begin, n_count, hdr, st);

@@ -25,7 +25,6 @@
 // beta = 0, k = q = v = 0).
 #include <cuda.h>
 
-#include <cstdlib>
 #include <type_traits>
 
 #include "kda_common.cuh"
@@ -619,8 +618,7 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cud
     if (rc == KDA_OK) rc = make_tmap(&tm_v, a.v, a.total_tokens, a.H);
     if (rc == KDA_OK) rc = make_tmap(&tm_q, a.q ? a.q : a.k, a.total_tokens, a.H);
     if (rc != KDA_OK) return rc;
-    static const int per_sm = getenv("KDA_INTRA_CTAS_PER_SM") ? atoi(getenv("KDA_INTRA_CTAS_PER_SM")) : 2;
-    const int64_t resident = per_sm * (int64_t)n_sm;   // two CTAs per SM
+    const int64_t resident = 2 * (int64_t)n_sm;   // two CTAs per SM
     const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
     ProfScope ps(PROF_INTRA, st);
     kda_intra_tc<<<grid, 256, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, a.q ? 1 : 0);
