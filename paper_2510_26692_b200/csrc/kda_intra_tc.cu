@@ -59,11 +59,18 @@ constexpr uint32_t S_BETA = S_T + 64 * LDT * 4;
 constexpr uint32_t S_CG = S_BETA + 256;        // exp(G_m) per channel (undoes the Kg reference)
 constexpr uint32_t S_BAR = S_CG + 512;          // mma barrier, tma barrier, TMEM slot
 constexpr uint32_t S_TOTAL = S_BAR + 64;
-constexpr int kBulkThread = 128;   // lane 0 of warp 4 issues every bulk copy; thread 0 issues the MMAs
+#ifndef KDA_INTRA_THREADS
+#define KDA_INTRA_THREADS 256
+#endif
+constexpr int kNT = KDA_INTRA_THREADS;   // threads per CTA (256 or 512), two CTAs per SM
+constexpr int kNW = kNT / 32;            // warps
+constexpr int kRPT = kC / kNW;           // token rows per thread in the gating phase (8 or 4)
+static_assert(kNT == 256 || kNT == 512, "thread mappings below are written for 8 or 16 warps");
+constexpr int kBulkThread = kNT / 2;     // lane 0 of a middle warp issues every bulk copy; thread 0 the MMAs
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kClamp2 = 80.f * 1.4426950408889634f;   // the +-80 clamp in the log2 domain
 constexpr uint32_t kIntraTcSmem = S_TOTAL + 1024;
-static_assert(S_TOT + 8 * 128 * 4 <= S_BETA, "staging + scan exchange fit below the small arrays");
+static_assert(S_TOT + 16 * 128 * 4 <= S_BETA, "staging + scan exchange fit below the small arrays");
 constexpr uint32_t kTmemCols = 256;
 
 // loads that the compiler may not sink below their issue point (register prefetch of the next tile)
@@ -121,7 +128,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&p);
 }
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(kNT, 2)
 kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
              const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
              const __grid_constant__ CUtensorMap tm_v, int has_q)
@@ -159,9 +166,9 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     // k, q and v by 2-D tiled TMA loads straight into the swizzled operand images (k and q are then
     // gated in place), log alpha into registers (thread (w, c4) owns rows 8w..8w+7 and channels
     // 4c4..4c4+3), beta by small asynchronous copies.
-    const int c4 = lane, d0 = c4 * 4, i0 = warp * 8;
+    const int c4 = lane, d0 = c4 * 4, i0 = warp * kRPT;
     const uint32_t ntiles = (uint32_t)((a.g1 - a.g0) * a.H);
-    float G[8][4];
+    float G[kRPT][4];
     auto locate = [&](uint32_t tl, ChunkLoc& Lo, int& ho) {
         const uint32_t gl = tl / (uint32_t)a.H;
         ho = (int)(tl - gl * (uint32_t)a.H);
@@ -170,7 +177,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     auto issue_prefetch = [&](const ChunkLoc& Lo, int ho) {
         const float* gp = a.log_alpha + ((size_t)Lo.tok0 * a.H + ho) * kD + d0;
 #pragma unroll
-        for (int r = 0; r < 8; ++r) {
+        for (int r = 0; r < kRPT; ++r) {
             const int i = i0 + r;
             if (i < Lo.len) {
                 ld_nc_f4(gp + (size_t)i * a.H * kD, G[r][0], G[r][1], G[r][2], G[r][3]);
@@ -219,23 +226,23 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
 #pragma unroll
     for (int e = 0; e < 4; ++e) G[0][e] *= kLog2e;
 #pragma unroll
-    for (int r = 1; r < 8; ++r)
+    for (int r = 1; r < kRPT; ++r)
 #pragma unroll
         for (int e = 0; e < 4; ++e) G[r][e] = fmaf(G[r][e], kLog2e, G[r - 1][e]);
-    *reinterpret_cast<float4*>(sTot + warp * kD + d0) = make_float4(G[7][0], G[7][1], G[7][2], G[7][3]);
+    *reinterpret_cast<float4*>(sTot + warp * kD + d0) = make_float4(G[kRPT - 1][0], G[kRPT - 1][1], G[kRPT - 1][2], G[kRPT - 1][3]);
     if (t == kBulkThread) ptx::bulk_wait_read0();   // the previous tile's output staging has been read out
     ptx::cp_async_wait_all();             // beta
     __syncthreads();
     KDA_PHASE(hdr, 0);   // loads arrived + local scan
     float base[4] = {0.f, 0.f, 0.f, 0.f}, gref[4] = {0.f, 0.f, 0.f, 0.f}, glast[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int r2 = 0; r2 < 8; ++r2) {
+    for (int r2 = 0; r2 < kNW; ++r2) {
         const float4 x4 = *reinterpret_cast<const float4*>(sTot + r2 * kD + d0);
         const float x[4] = {x4.x, x4.y, x4.z, x4.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (r2 < warp) base[e] += x[e];
-            if (r2 < 4) gref[e] += x[e];    // rows 0..31
+            if (r2 < kNW / 2) gref[e] += x[e];    // rows 0..31
             glast[e] += x[e];
         }
     }
@@ -262,18 +269,18 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     tma_parity ^= 1;
     KDA_PHASE(hdr, 11);  // TMA wait
     if (L.len < kC) {   // short last chunk: rows past the end hold the next sequence's v; zero them
-        for (int idx = t; idx < (kC - L.len) * 16; idx += 256) {
+        for (int idx = t; idx < (kC - L.len) * 16; idx += kNT) {
             const int j = L.len + (idx >> 4), c16 = idx & 15;
             *reinterpret_cast<uint4*>(smem + S_V + (c16 >> 3) * S_V_BLOCK + j * 128 +
                                       (((c16 & 7) ^ (j & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
         }
     }
     const int hf = c4 >> 4;                       // K-half (channels 0-63 / 64-127)
-    uint32_t ktb[4][4];                           // (K exp(G_C - G))^T: 4 channels x 8 tokens, bf16 pairs
+    uint32_t ktb[4][kRPT / 2];                    // (K exp(G_C - G))^T: 4 channels x kRPT tokens, bf16 pairs
     auto gate_rows = [&](auto harsh_tag) {
         constexpr bool kHarsh = decltype(harsh_tag)::value;
 #pragma unroll
-        for (int r = 0; r < 8; ++r) {
+        for (int r = 0; r < kRPT; ++r) {
             const int i = i0 + r;
             const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
             uint8_t* pk = smem + S_KQ + hf * S_KQ_HALF + off;
@@ -328,11 +335,19 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     };
     if (!harsh) gate_rows(std::false_type{});
     else gate_rows(std::true_type{});
-    // (K exp(G_C - G))^T: row = channel, this warp's 8 tokens are one 16-byte chunk
+    // (K exp(G_C - G))^T: row = channel; this warp's tokens are one 16-byte chunk (8 warps) or half of
+    // one (16 warps)
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-        *reinterpret_cast<uint4*>(smem + S_KT + (d0 + e) * 128 + ((warp ^ ((d0 + e) & 7)) << 4)) =
-            make_uint4(ktb[e][0], ktb[e][1], ktb[e][2], ktb[e][3]);
+    for (int e = 0; e < 4; ++e) {
+        const int d = d0 + e;
+        if (kRPT == 8) {
+            *reinterpret_cast<uint4*>(smem + S_KT + d * 128 + ((warp ^ (d & 7)) << 4)) =
+                make_uint4(ktb[e][0], ktb[e][1], ktb[e][kRPT / 2 - 2], ktb[e][kRPT / 2 - 1]);
+        } else {
+            *reinterpret_cast<uint2*>(smem + S_KT + d * 128 + (((warp >> 1) ^ (d & 7)) << 4) + (warp & 1) * 8) =
+                make_uint2(ktb[e][0], ktb[e][1]);
+        }
+    }
 
     KDA_PHASE(hdr, 12);  // element loop + stores (thread 0)
     ptx::fence_async_smem();
@@ -364,35 +379,37 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     KDA_PHASE(hdr, 2);   // first MMA group
     ptx::tc_fence_after();
     {
-        const int q4 = warp & 3, ch = warp >> 2;
+        constexpr int NCA = 64 / (kNW / 4);   // accumulator columns per warp: 32 (8 warps) or 16 (16 warps)
+        const int q4 = warp & 3, c0 = (warp >> 2) * NCA;
         const int R = q4 * 32 + lane;
-        uint32_t r[32];
-        ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q4 * 32) << 16) + ch * 32, r);
+        uint32_t r[NCA];
+        if (NCA == 32) ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q4 * 32) << 16) + c0, reinterpret_cast<uint32_t(&)[32]>(r));
+        else ptx::tmem_ld_32x32b_x16(tmem_base + ((uint32_t)(q4 * 32) << 16) + c0, reinterpret_cast<uint32_t(&)[16]>(r));
         ptx::tmem_ld_wait();
         if (R < 64) {
             const int i = R;
             const float bi = sBeta[i];
 #pragma unroll
-            for (int j4 = 0; j4 < 32; j4 += 4) {
+            for (int j4 = 0; j4 < NCA; j4 += 4) {
                 float x[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int j = ch * 32 + j4 + e;
+                    const int j = c0 + j4 + e;
                     x[e] = (j < i) ? bi * __uint_as_float(r[j4 + e]) : 0.f;
                 }
-                *reinterpret_cast<float4*>(sA + i * LDT + ch * 32 + j4) = make_float4(x[0], x[1], x[2], x[3]);
+                *reinterpret_cast<float4*>(sA + i * LDT + c0 + j4) = make_float4(x[0], x[1], x[2], x[3]);
             }
         } else {
             const int i = R - 64;
 #pragma unroll
-            for (int j8 = 0; j8 < 32; j8 += 8) {
+            for (int j8 = 0; j8 < NCA; j8 += 8) {
                 float x[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const int j = ch * 32 + j8 + e;
+                    const int j = c0 + j8 + e;
                     x[e] = (j <= i) ? __uint_as_float(r[j8 + e]) : 0.f;
                 }
-                *reinterpret_cast<uint4*>(smem + S_AQ + ptx::sw128_off(i, ch * 32 + j8)) =
+                *reinterpret_cast<uint4*>(smem + S_AQ + ptx::sw128_off(i, c0 + j8)) =
                     make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]),
                                pack_bf16(x[6], x[7]));
             }
@@ -450,24 +467,26 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     KDA_PHASE(hdr, 6);   // block levels
     // ---- a4: Mm = T Diag(beta) as the A operand; [W | U] = Mm [Kg | V] ---------------------------------
     {
-        const int i = t >> 2, jq = t & 3;
-        float x[16];
-        if (jq > (i >> 4)) {
+        constexpr int NCM = 64 / (kNT / 64);   // columns per thread: 16 (256 threads) or 8 (512 threads)
+        const int i = t / (kNT / 64), jq = t % (kNT / 64);
+        const int j0 = jq * NCM;
+        float x[NCM];
+        if ((j0 >> 4) > (i >> 4)) {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) x[e] = 0.f;
+            for (int e = 0; e < NCM; ++e) x[e] = 0.f;
         } else {
 #pragma unroll
-            for (int e4 = 0; e4 < 16; e4 += 4) {
-                const float4 tv = *reinterpret_cast<const float4*>(sT + i * LDT + jq * 16 + e4);
-                const float4 bv = *reinterpret_cast<const float4*>(sBeta + jq * 16 + e4);
+            for (int e4 = 0; e4 < NCM; e4 += 4) {
+                const float4 tv = *reinterpret_cast<const float4*>(sT + i * LDT + j0 + e4);
+                const float4 bv = *reinterpret_cast<const float4*>(sBeta + j0 + e4);
                 x[e4] = tv.x * bv.x; x[e4 + 1] = tv.y * bv.y; x[e4 + 2] = tv.z * bv.z; x[e4 + 3] = tv.w * bv.w;
             }
         }
 #pragma unroll
-        for (int c8 = 0; c8 < 2; ++c8) {
+        for (int c8 = 0; c8 < NCM / 8; ++c8) {
             const uint4 pk = make_uint4(pack_bf16(x[c8 * 8], x[c8 * 8 + 1]), pack_bf16(x[c8 * 8 + 2], x[c8 * 8 + 3]),
                                         pack_bf16(x[c8 * 8 + 4], x[c8 * 8 + 5]), pack_bf16(x[c8 * 8 + 6], x[c8 * 8 + 7]));
-            uint8_t* dst = smem + S_MM + i * 128 + ((((jq * 2 + c8) ^ (i & 7))) << 4);
+            uint8_t* dst = smem + S_MM + i * 128 + ((((j0 >> 3) + c8) ^ (i & 7)) << 4);
             *reinterpret_cast<uint4*>(dst) = pk;
             *reinterpret_cast<uint4*>(dst + 8192) = pk;   // rows 64-127 repeat rows 0-63
         }
@@ -500,38 +519,38 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     KDA_PHASE(hdr, 8);   // second MMA group
     ptx::tc_fence_after();
     {   // The A operand held every row twice, so TMEM lanes 0-63 and 64-127 both carry rows 0-63:
-        // warp (q4, part) converts rows 32 (q4 & 1) + lane of the 64-column block cb of [W | U].
-        const int q4 = warp & 3, cb = (warp >> 2) * 2 + (q4 >> 1);
+        // each warp converts rows 32 (q4 & 1) + lane of one NCE-column block of [W | U].
+        constexpr int NCE = 256 / (kNW / 2);   // 64 columns per warp (8 warps) or 32 (16 warps)
+        const int q4 = warp & 3, cbk = (warp >> 2) * 2 + (q4 >> 1);
+        const int col0 = cbk * NCE;            // first column inside [W | U]
         const int i = (q4 & 1) * 32 + lane;
-        uint32_t r0[32], r1[32];
-        const uint32_t ta = tmem_base + ((uint32_t)(q4 * 32) << 16) + cb * 64;
-        ptx::tmem_ld_32x32b_x32(ta, r0);
-        ptx::tmem_ld_32x32b_x32(ta + 32, r1);
+        uint32_t r[NCE];
+        const uint32_t ta = tmem_base + ((uint32_t)(q4 * 32) << 16) + col0;
+#pragma unroll
+        for (int b = 0; b < NCE / 32; ++b)
+            ptx::tmem_ld_32x32b_x32(ta + b * 32, reinterpret_cast<uint32_t(&)[32]>(r[b * 32]));
         ptx::tmem_ld_wait();
-        if (cb < 2) {   // W = (Mm Kg) exp(G_m): K-half cb of the [W ; Gamma.Q] image
-            uint8_t* dst = smem + S_W + cb * 8192;
+        if (col0 < 128) {   // W = (Mm Kg) exp(G_m): K-half col0 / 64 of the [W ; Gamma.Q] image
+            uint8_t* dst = smem + S_W + (col0 >> 6) * 8192;
 #pragma unroll
-            for (int j8 = 0; j8 < 64; j8 += 8) {
-                const float4 s0 = *reinterpret_cast<const float4*>(sCG + cb * 64 + j8);
-                const float4 s1 = *reinterpret_cast<const float4*>(sCG + cb * 64 + j8 + 4);
-                const uint32_t* r = j8 < 32 ? r0 + j8 : r1 + (j8 - 32);
-                *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, j8)) =
-                    make_uint4(pack_bf16(__uint_as_float(r[0]) * s0.x, __uint_as_float(r[1]) * s0.y),
-                               pack_bf16(__uint_as_float(r[2]) * s0.z, __uint_as_float(r[3]) * s0.w),
-                               pack_bf16(__uint_as_float(r[4]) * s1.x, __uint_as_float(r[5]) * s1.y),
-                               pack_bf16(__uint_as_float(r[6]) * s1.z, __uint_as_float(r[7]) * s1.w));
+            for (int j8 = 0; j8 < NCE; j8 += 8) {
+                const float4 s0 = *reinterpret_cast<const float4*>(sCG + col0 + j8);
+                const float4 s1 = *reinterpret_cast<const float4*>(sCG + col0 + j8 + 4);
+                *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, (col0 & 63) + j8)) =
+                    make_uint4(pack_bf16(__uint_as_float(r[j8]) * s0.x, __uint_as_float(r[j8 + 1]) * s0.y),
+                               pack_bf16(__uint_as_float(r[j8 + 2]) * s0.z, __uint_as_float(r[j8 + 3]) * s0.w),
+                               pack_bf16(__uint_as_float(r[j8 + 4]) * s1.x, __uint_as_float(r[j8 + 5]) * s1.y),
+                               pack_bf16(__uint_as_float(r[j8 + 6]) * s1.z, __uint_as_float(r[j8 + 7]) * s1.w));
             }
-        } else {        // U: image cb - 2
-            uint8_t* dst = smem + S_U + (cb - 2) * tc::U_IMAGE;
+        } else {            // U: image (col0 - 128) / 64
+            uint8_t* dst = smem + S_U + ((col0 - 128) >> 6) * tc::U_IMAGE;
 #pragma unroll
-            for (int j8 = 0; j8 < 64; j8 += 8) {
-                const uint32_t* r = j8 < 32 ? r0 + j8 : r1 + (j8 - 32);
-                *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, j8)) =
-                    make_uint4(pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1])),
-                               pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3])),
-                               pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5])),
-                               pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7])));
-            }
+            for (int j8 = 0; j8 < NCE; j8 += 8)
+                *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, (col0 & 63) + j8)) =
+                    make_uint4(pack_bf16(__uint_as_float(r[j8]), __uint_as_float(r[j8 + 1])),
+                               pack_bf16(__uint_as_float(r[j8 + 2]), __uint_as_float(r[j8 + 3])),
+                               pack_bf16(__uint_as_float(r[j8 + 4]), __uint_as_float(r[j8 + 5])),
+                               pack_bf16(__uint_as_float(r[j8 + 6]), __uint_as_float(r[j8 + 7])));
         }
     }
     ptx::fence_async_smem();
@@ -621,7 +640,7 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cud
     const int64_t resident = 2 * (int64_t)n_sm;   // two CTAs per SM
     const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
     ProfScope ps(PROF_INTRA, st);
-    kda_intra_tc<<<grid, 256, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, a.q ? 1 : 0);
+    kda_intra_tc<<<grid, kNT, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, a.q ? 1 : 0);
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;
