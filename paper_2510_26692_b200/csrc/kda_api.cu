@@ -192,7 +192,11 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
     int32_t* chunk_cu_dev = reinterpret_cast<int32_t*>(ws + L.off_table);
-    kda_status_t rc = launch_prep(hdr, cu_seqlens_dev, chunk_cu_dev, n_seqs, st);
+    // The prologue kernel clears the status word and builds the chunk table of a packed batch.  An
+    // equal-length bf16 call with work to do skips it: its first intra-chunk kernel clears the word.
+    const bool tc_clears = dt == KDA_BF16 && !cu_seqlens_dev && total_chunks > 0 && (o || S_T);
+    kda_status_t rc = KDA_OK;
+    if (!tc_clears) rc = launch_prep(hdr, cu_seqlens_dev, chunk_cu_dev, n_seqs, st);
     if (rc != KDA_OK) return rc;
     if (!o && !S_T) return KDA_OK;   // nothing observable to produce
 
@@ -219,7 +223,7 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
             n_count = n_end - n_begin;
         }
         if (dt == KDA_BF16)
-            rc = launch_chunk_tc(a, ws + L.off_tiles, n_begin, n_count, hdr, st);
+            rc = launch_chunk_tc(a, ws + L.off_tiles, n_begin, n_count, hdr, tc_clears && first, st);
         else
             rc = launch_chunk_simt(a, dt, ws + L.off_tiles, n_begin, n_count, st);
         if (rc != KDA_OK) return rc;

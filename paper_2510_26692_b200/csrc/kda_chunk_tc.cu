@@ -26,7 +26,8 @@
 
 namespace kda {
 
-kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cudaStream_t st);
+kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, bool clear_status,
+                             cudaStream_t st);
 
 namespace {
 
@@ -153,6 +154,9 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 64) * tc::U_IMAGE,
                               Cfg::kUBytes, &full[s]);
             };
+            // the tiles come from the intra-chunk kernel launched just before this one; everything
+            // above (barriers, TMEM, reading the state) may overlap that kernel's tail
+            ptx::grid_dep_wait();
             int loads_issued = 0;
             for (; loads_issued < NSTG && loads_issued < nchunks; ++loads_issued) issue_loads(loads_issued);
             for (int it = 0; it < nchunks; ++it) {
@@ -293,7 +297,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
 
 template <int NS>
 kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begin, int n_count,
-                               WsHeader* hdr, cudaStream_t st)
+                               WsHeader* hdr, bool after_intra, cudaStream_t st)
 {
     using Cfg = InterCfg<NS>;
     static bool attr_done = false;
@@ -302,11 +306,21 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
                                           (int)Cfg::kSmem));
         attr_done = true;
     }
-    dim3 grid(kD / NS, (unsigned)a.H, (unsigned)n_count);
     ProfScope ps(PROF_INTER, st);
-    kda_inter_tc<NS><<<grid, 160, Cfg::kSmem, st>>>(a, tiles, n_begin, hdr);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kD / NS, (unsigned)a.H, (unsigned)n_count);
+    cfg.blockDim = dim3(160);
+    cfg.dynamicSmemBytes = Cfg::kSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    // only overlap with this library's own intra-chunk kernel, never with a caller's kernel that may
+    // still be producing S0
+    cfg.numAttrs = after_intra ? 1 : 0;
+    KDA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kda_inter_tc<NS>, a, tiles, n_begin, hdr));
     count_launch();
-    KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;
 }
 
@@ -315,12 +329,12 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
 size_t tc_tile_bytes() { return tc::TILE_BYTES; }
 
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
-                             WsHeader* hdr, cudaStream_t st)
+                             WsHeader* hdr, bool clear_status, cudaStream_t st)
 {
-    kda_status_t rc = launch_intra_tc(a, tiles, hdr, st);
+    kda_status_t rc = launch_intra_tc(a, tiles, hdr, clear_status, st);
     if (rc != KDA_OK) return rc;
     if (n_count <= 0) return KDA_OK;
-    return launch_inter_tc_t<32>(a, (const char*)tiles, n_begin, n_count, hdr, st);
+    return launch_inter_tc_t<32>(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);
 }
 
 }  // namespace kda

@@ -162,7 +162,7 @@ kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, 
 // bf16 tensor-core path (tcgen05 + bulk copies): per-tile scratch size and pass launcher
 size_t tc_tile_bytes();
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
-                             WsHeader* hdr, cudaStream_t st);
+                             WsHeader* hdr, bool clear_status, cudaStream_t st);
 
 // clears the status word and (packed batches) builds chunk_cu[n_seqs+1] from cu_seqlens
 kda_status_t launch_prep(WsHeader* hdr, const int32_t* cu_seqlens, int32_t* chunk_cu, int n_seqs,

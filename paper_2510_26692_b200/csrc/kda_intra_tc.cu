@@ -131,7 +131,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 __global__ void __launch_bounds__(kNT, 2)
 kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
              const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
-             const __grid_constant__ CUtensorMap tm_v, int has_q)
+             const __grid_constant__ CUtensorMap tm_v, int has_q, int clear_status)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(
@@ -148,6 +148,11 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
 
     KDA_PHASE_DECL;
+    ptx::grid_dep_launch();   // the inter-chunk kernel may set itself up while this one drains
+    if (clear_status && blockIdx.x == 0 && t == 0) {
+        hdr->status = 0;      // (an equal-length call has no prologue kernel to do this)
+        hdr->where = 0;
+    }
     if (t == 0) {
         ptx::mbar_init(mma_bar, 1);
         ptx::mbar_init(tma_bar, 1);
@@ -614,7 +619,8 @@ kda_status_t make_tmap(CUtensorMap* tm, const void* base, int64_t total_tokens, 
 }
 }  // namespace
 
-kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cudaStream_t st)
+kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, bool clear_status,
+                             cudaStream_t st)
 {
     static bool attr_done = false;
     if (!attr_done) {
@@ -640,7 +646,8 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, cud
     const int64_t resident = 2 * (int64_t)n_sm;   // two CTAs per SM
     const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
     ProfScope ps(PROF_INTRA, st);
-    kda_intra_tc<<<grid, kNT, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, a.q ? 1 : 0);
+    kda_intra_tc<<<grid, kNT, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, a.q ? 1 : 0,
+                                                     clear_status ? 1 : 0);
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;

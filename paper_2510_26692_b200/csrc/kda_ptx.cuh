@@ -125,6 +125,13 @@ __device__ __forceinline__ void cp_async4(void* dst_smem, const void* src_gmem, 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
+// programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
+// attribute may begin before its predecessor in the stream has finished; grid_dep_wait() blocks
+// until the predecessor has completed and its writes are visible.  grid_dep_launch() in the
+// predecessor allows the dependent grid to be scheduled as soon as resources free up.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA / tcgen05 operand reads)
 __device__ __forceinline__ void fence_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
