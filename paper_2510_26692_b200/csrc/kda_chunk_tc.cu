@@ -41,8 +41,8 @@ template <int NS> struct InterCfg {
     static constexpr uint32_t kAQ = 49152;                  // [64][64]; used as rows 64-127 of a 128-row operand
     static constexpr uint32_t kGC = 57344;                  // gamma^C, 128 fp32
     static constexpr uint32_t kMainBytes = 57856;           // QW | Kt | Aqk | gamma^C are contiguous in a tile
-    static constexpr uint32_t kU = 57856;                   // the [64 tokens][64 columns] image of U holding this slice
-    static constexpr uint32_t kUBytes = tc::U_IMAGE;
+    static constexpr uint32_t kU = 57856;                   // [64 tokens][NS] block of U
+    static constexpr uint32_t kUBytes = tc::U_BLOCK;
     static constexpr uint32_t kStage = (kU + kUBytes + 1023) / 1024 * 1024;
     static constexpr uint32_t kSbf = kStages * kStage;      // B operand of MMA1, MN-major: [128 dk rows][128 B]
     static constexpr uint32_t kVn = kSbf + 128 * 128;       // B operand of MMA2, MN-major: [64 token rows][128 B]
@@ -151,7 +151,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 uint8_t* sb = smem + s * Cfg::kStage;
                 ptx::mbar_expect_tx(&full[s], Cfg::kTxBytes);
                 ptx::bulk_g2s(sb + Cfg::kQW, tile + tc::OFF_QW, Cfg::kMainBytes, &full[s]);
-                ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 64) * tc::U_IMAGE,
+                ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 32) * tc::U_BLOCK,
                               Cfg::kUBytes, &full[s]);
             };
             // the tiles come from the intra-chunk kernel launched just before this one; everything
@@ -222,12 +222,10 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             const uint32_t par = (uint32_t)it & 1u;
             wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);   // U and gamma^C are read with plain loads
             if (warp < 2) {   // a6: V_new = U - W S  (token row = tid)
-                const uint8_t* up = sb + Cfg::kU + tid * 128;   // this token's row of the swizzled image
-                const int c0 = (col0 & 63) >> 3;
-                uint4 uq[4];
+                uint4 uq[4];   // this token's 32 values of U
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                    uq[c] = *reinterpret_cast<const uint4*>(up + (((c0 + c) ^ (tid & 7)) << 4));
+                    uq[c] = *reinterpret_cast<const uint4*>(sb + Cfg::kU + tc::u_off(tid, c));
                 const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
                 wait(mma1_bar, par, 2);
                 KDA_PHASE(hdr, 18);  // MMA1

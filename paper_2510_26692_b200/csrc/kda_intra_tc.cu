@@ -54,7 +54,7 @@ constexpr uint32_t S_TOT = S_M + 32768;        // scan exchange [8][128] fp32, 4
 constexpr uint32_t S_AQ = S_M;                 // Aqk image [64][64] bf16 (after the first MMA group)
 constexpr uint32_t S_MM = S_KI;                // [128][64] bf16: T Diag(beta) twice (rows 64-127 repeat rows 0-63)
 constexpr uint32_t S_W = S_M;                  // W image [2 halves][64][64] bf16 (after the second group)
-constexpr uint32_t S_U = S_M + 16384;          // U: two [64][64] bf16 images
+constexpr uint32_t S_U = S_M + 16384;          // U: four [64][32] bf16 blocks
 constexpr uint32_t S_BETA = S_T + 64 * LDT * 4;
 constexpr uint32_t S_CG = S_BETA + 256;        // exp(G_m) per channel (undoes the Kg reference)
 constexpr uint32_t S_BAR = S_CG + 512;          // mma barrier, tma barrier, TMEM slot
@@ -547,15 +547,16 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
                                pack_bf16(__uint_as_float(r[j8 + 4]) * s1.x, __uint_as_float(r[j8 + 5]) * s1.y),
                                pack_bf16(__uint_as_float(r[j8 + 6]) * s1.z, __uint_as_float(r[j8 + 7]) * s1.w));
             }
-        } else {            // U: image (col0 - 128) / 64
-            uint8_t* dst = smem + S_U + ((col0 - 128) >> 6) * tc::U_IMAGE;
+        } else {            // U: 32-column blocks (col0 - 128) / 32 ...
 #pragma unroll
-            for (int j8 = 0; j8 < NCE; j8 += 8)
-                *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, (col0 & 63) + j8)) =
+            for (int j8 = 0; j8 < NCE; j8 += 8) {
+                const int cu = col0 - 128 + j8;
+                *reinterpret_cast<uint4*>(smem + S_U + (cu >> 5) * tc::U_BLOCK + tc::u_off(i, (cu & 31) >> 3)) =
                     make_uint4(pack_bf16(__uint_as_float(r[j8]), __uint_as_float(r[j8 + 1])),
                                pack_bf16(__uint_as_float(r[j8 + 2]), __uint_as_float(r[j8 + 3])),
                                pack_bf16(__uint_as_float(r[j8 + 4]), __uint_as_float(r[j8 + 5])),
                                pack_bf16(__uint_as_float(r[j8 + 6]), __uint_as_float(r[j8 + 7])));
+            }
         }
     }
     ptx::fence_async_smem();

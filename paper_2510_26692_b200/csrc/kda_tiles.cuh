@@ -17,10 +17,14 @@ constexpr uint32_t OFF_KT = 32768;
 constexpr uint32_t OFF_AQ = 49152;
 // gamma^C: 128 fp32 (directly after the three operand images: one bulk copy fetches all four)
 constexpr uint32_t OFF_GC = 57344;
-// U as two [64 tokens][64 columns] bf16 images in the same 128-byte-swizzled row layout (it is
-// read with plain loads, the swizzle only keeps the producer's stores free of bank conflicts)
+// U in four column blocks of [64 tokens][32 columns] bf16 (64-byte rows).  It is read with plain
+// loads; the 16-byte chunks of a row are XOR-swizzled with (row >> 1) & 3 only to keep the
+// producer's row-per-thread stores free of shared-memory bank conflicts (see u_off).
 constexpr uint32_t OFF_U = 57856;
-constexpr uint32_t U_IMAGE = 64 * 128;
+constexpr uint32_t U_BLOCK = 64 * 64;
+__host__ __device__ __forceinline__ constexpr uint32_t u_off(uint32_t row, uint32_t chunk) {
+    return row * 64u + ((chunk ^ ((row >> 1) & 3u)) << 4);
+}
 constexpr uint32_t TILE_BYTES = 74240;
 static_assert(TILE_BYTES % 256 == 0, "tiles stay 256-byte aligned");
 }  // namespace tc
