@@ -84,8 +84,10 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + Cfg::kBars);        // [NSTG] operands landed
     uint64_t* mma1_bar = full + NSTG;      // MMA1 of a chunk complete
     uint64_t* mma2_bar = mma1_bar + 1;     // MMA2 of a chunk complete
-    uint64_t* out_bar = mma2_bar + 1;      // the output accumulator of a chunk is complete
-    uint64_t* sbf_ready = out_bar + 1;     // 128 arrivals: bf16 state copy written (and stage reads done)
+    // out_bar is waited on by warps that the rest of the pipeline could, in principle, overtake by a
+    // whole chunk; two barriers used alternately keep a parity wait from ever being lapped
+    uint64_t* out_bar = mma2_bar + 1;      // [2] the output accumulator of a chunk is complete
+    uint64_t* sbf_ready = out_bar + 2;     // 128 arrivals: bf16 state copy written (and stage reads done)
     uint64_t* vn_ready = sbf_ready + 1;    // 64 arrivals: V_new written
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(vn_ready + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -116,7 +118,8 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         for (int s = 0; s < NSTG; ++s) ptx::mbar_init(&full[s], 1);
         ptx::mbar_init(mma1_bar, 1);
         ptx::mbar_init(mma2_bar, 1);
-        ptx::mbar_init(out_bar, 1);
+        ptx::mbar_init(&out_bar[0], 1);
+        ptx::mbar_init(&out_bar[1], 1);
         ptx::mbar_init(sbf_ready, 128);
         ptx::mbar_init(vn_ready, 64);
         *abort_flag = 0;
@@ -189,9 +192,9 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 for (int k = 0; k < 4; ++k)
                     ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kAQ - 8192 + k * 32),
                                    ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, 1);
-                ptx::umma_commit(out_bar);
+                ptx::umma_commit(&out_bar[it & 1]);
             }
-            if (nchunks > 0) wait(out_bar, (uint32_t)(nchunks - 1) & 1u, 7);   // last output product done
+            if (nchunks > 0) wait(&out_bar[(nchunks - 1) & 1], (uint32_t)((nchunks - 1) >> 1) & 1u, 7);   // last output product done
             if (*abort_flag) {
                 // drain the bulk copies still in flight before the shared memory goes away
                 for (int j = (loads_issued > NSTG ? loads_issued - NSTG : 0); j < loads_issued; ++j)
@@ -263,7 +266,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
                 const int len = (tok_end - tok0) < kC ? (int)(tok_end - tok0) : kC;
                 __nv_bfloat16* orow = op + ((tok0 + i) * a.H + h) * kD + col0;
-                wait(out_bar, par, 6);
+                wait(&out_bar[it & 1], (uint32_t)(it >> 1) & 1u, 6);
                 ptx::tc_fence_after();
                 uint32_t r[32];
                 ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
