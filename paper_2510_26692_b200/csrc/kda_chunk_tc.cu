@@ -50,7 +50,7 @@ template <int NS> struct InterCfg {
     static constexpr uint32_t kTotal = kBars + 128;
     static constexpr uint32_t kSmem = kTotal + 1024;        // slack for manual 1024-byte alignment
     static constexpr uint32_t kTxBytes = kMainBytes + kUBytes;
-    static constexpr uint32_t kTmemCols = 128;              // D1 (two buffers) + D3, NS columns each
+    static constexpr uint32_t kTmemCols = 256;              // 4 x D1 + 2 x D3, NS columns each
 };
 
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
@@ -69,11 +69,12 @@ __device__ __forceinline__ void store_row32(uint8_t* img, int row, const float (
 }
 
 // Thread roles: warps 0-3 compute (TMEM lane quadrant = warp index; thread = token row for
-// V_new / O, thread = dk row for the state), warp 4 is the control warp whose lane 0 issues every
-// bulk copy and every MMA.  The roles meet only on mbarriers, so issue latencies never sit on the
-// compute warps' path and the output conversion overlaps the next chunk's first MMA.
+// V_new / O, thread = dk row for the state), warps 4 and 5 are control warps whose lane 0 issues
+// the MMAs (and, in warp 4, the bulk copies).  The roles meet only on mbarriers, so issue
+// latencies never sit on the compute warps' path and the output conversion overlaps the next
+// chunk's first MMA.
 template <int NS>
-__global__ void __launch_bounds__(160, 1)
+__global__ void __launch_bounds__(192, 1)
 kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader* hdr)
 {
     using Cfg = InterCfg<NS>;
@@ -116,8 +117,8 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < NSTG; ++s) ptx::mbar_init(&full[s], 1);
-        ptx::mbar_init(mma1_bar, 1);
-        ptx::mbar_init(mma2_bar, 1);
+        ptx::mbar_init(mma1_bar, 2);   // one commit from each control thread
+        ptx::mbar_init(mma2_bar, 2);
         ptx::mbar_init(&out_bar[0], 1);
         ptx::mbar_init(&out_bar[1], 1);
         ptx::mbar_init(sbf_ready, 128);
@@ -133,7 +134,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t d3 = 2 * NS;   // TMEM column offsets: D1 buffers at 0 and NS, D3 at 2 NS
+    const uint32_t d3 = 4 * NS;   // TMEM columns: D1 {parity 0,1} x {half 0,1} at 0..4 NS, D3 halves at 4 NS, 5 NS
 
     auto wait = [&](uint64_t* bar, uint32_t parity, int where) {
         if (*abort_flag) return;
@@ -143,9 +144,14 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         }
     };
 
-    if (warp == 4) {
-        // ================= control warp: lane 0 issues all copies and MMAs =================
-        if (tid == 128) {
+    if (warp >= 4) {
+        // ================= two control warps: lane 0 of each issues MMAs =================
+        // Issuing one tcgen05.mma costs the issuing thread several tens of cycles whatever the tile
+        // size, and both products on the sequential chain are tiny, so each is split along its
+        // summation index between the two threads, into two accumulators that are added when they
+        // are read back.  Thread A (warp 4) also issues the bulk copies and the output product.
+        const int half = warp - 4;
+        if ((tid & 31) == 0) {
             const uint32_t idesc = ptx::umma_idesc_bf16(128, NS) | ptx::kIdescBMajorMN;
             const uint32_t sbf_a = ptx::smem_u32(sbf), vn_a = ptx::smem_u32(vn);
             auto issue_loads = [&](int it) {
@@ -157,48 +163,57 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::bulk_g2s(sb + Cfg::kU, tile + tc::OFF_U + (size_t)(col0 / 32) * tc::U_BLOCK,
                               Cfg::kUBytes, &full[s]);
             };
-            // the tiles come from the intra-chunk kernel launched just before this one; everything
-            // above (barriers, TMEM, reading the state) may overlap that kernel's tail
-            ptx::grid_dep_wait();
             int loads_issued = 0;
-            for (; loads_issued < NSTG && loads_issued < nchunks; ++loads_issued) issue_loads(loads_issued);
+            if (half == 0) {
+                // the tiles come from the intra-chunk kernel launched just before this one; everything
+                // above (barriers, TMEM, reading the state) may overlap that kernel's tail
+                ptx::grid_dep_wait();
+                for (; loads_issued < NSTG && loads_issued < nchunks; ++loads_issued) issue_loads(loads_issued);
+            }
             for (int it = 0; it < nchunks; ++it) {
                 const int s = it % NSTG;
                 const uint32_t sb = ptx::smem_u32(smem + s * Cfg::kStage);
-                const uint32_t d1 = tmem_base + (uint32_t)(it & 1) * NS;
-                // MMA1(it): D1 = [W ; Gamma.Q] S  -- needs this chunk's operands and the state copy
+                // accumulators of this chunk: D1 (two parities x two halves), D3 (two halves)
+                const uint32_t d1 = tmem_base + (uint32_t)((it & 1) * 2 + half) * NS;
+                // MMA1(it): D1 = [W ; Gamma.Q] S, this thread's half of the sum over dk
                 wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);
                 wait(sbf_ready, (uint32_t)it & 1u, 4);
                 ptx::tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kQW + (k >> 2) * tc::QW_HALF + (k & 3) * 32),
-                                   ptx::umma_desc_sw128_mn(sbf_a + k * 2048, 8192), idesc, k > 0);
+                for (int k = 0; k < 4; ++k)
+                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kQW + half * tc::QW_HALF + k * 32),
+                                   ptx::umma_desc_sw128_mn(sbf_a + (half * 4 + k) * 2048, 8192), idesc, k > 0);
                 ptx::umma_commit(mma1_bar);
                 // the stage of the previous chunk is free now (its readers arrived on sbf_ready)
-                if (it > 0 && loads_issued < nchunks) { issue_loads(loads_issued); ++loads_issued; }
-                // MMA2(it): D1[64:128] += Aqk V_new,  D3 = Kt^T V_new.  The 128-row A operand of the
-                // first product starts 64 rows before Aqk: those rows (the tail of the Kt image) only
-                // touch accumulator rows 0-63, which are dead once V_new has been taken.
+                if (half == 0 && it > 0 && loads_issued < nchunks) { issue_loads(loads_issued); ++loads_issued; }
+                // MMA2(it): D3 = Kt^T V_new, this thread's half of the sum over the chunk's tokens.
+                // The state product sits on the sequential chain: it is issued and committed first.
                 wait(vn_ready, (uint32_t)it & 1u, 5);
                 ptx::tc_fence_after();
-                // the state product sits on the sequential chain: issue and commit it first
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    ptx::umma_bf16(tmem_base + d3, ptx::umma_desc_sw128(sb + Cfg::kKT + k * 32),
-                                   ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, k > 0);
+                for (int k = 0; k < 2; ++k)
+                    ptx::umma_bf16(tmem_base + d3 + half * NS,
+                                   ptx::umma_desc_sw128(sb + Cfg::kKT + (half * 2 + k) * 32),
+                                   ptx::umma_desc_sw128_mn(vn_a + (half * 2 + k) * 2048, 8192), idesc, k > 0);
                 ptx::umma_commit(mma2_bar);
+                if (half == 0) {
+                    // D1[64:128] += Aqk V_new.  The 128-row A operand starts 64 rows before Aqk: those
+                    // rows (the tail of the Kt image) only touch accumulator rows 0-63, which are dead
+                    // once V_new has been taken.
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kAQ - 8192 + k * 32),
-                                   ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, 1);
-                ptx::umma_commit(&out_bar[it & 1]);
+                    for (int k = 0; k < 4; ++k)
+                        ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kAQ - 8192 + k * 32),
+                                       ptx::umma_desc_sw128_mn(vn_a + k * 2048, 8192), idesc, 1);
+                    ptx::umma_commit(&out_bar[it & 1]);
+                }
             }
-            if (nchunks > 0) wait(&out_bar[(nchunks - 1) & 1], (uint32_t)((nchunks - 1) >> 1) & 1u, 7);   // last output product done
-            if (*abort_flag) {
-                // drain the bulk copies still in flight before the shared memory goes away
-                for (int j = (loads_issued > NSTG ? loads_issued - NSTG : 0); j < loads_issued; ++j)
-                    ptx::mbar_wait(&full[j % NSTG], (uint32_t)(j / NSTG) & 1u, kWaitLimitNs);
+            if (half == 0) {
+                if (nchunks > 0) wait(&out_bar[(nchunks - 1) & 1], (uint32_t)((nchunks - 1) >> 1) & 1u, 7);   // last output product done
+                if (*abort_flag) {
+                    // drain the bulk copies still in flight before the shared memory goes away
+                    for (int j = (loads_issued > NSTG ? loads_issued - NSTG : 0); j < loads_issued; ++j)
+                        ptx::mbar_wait(&full[j % NSTG], (uint32_t)(j / NSTG) & 1u, kWaitLimitNs);
+                }
             }
         }
     } else {
@@ -221,7 +236,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         for (int it = 0; it < nchunks; ++it) {
             const int s = it % NSTG;
             const uint8_t* sb = smem + s * Cfg::kStage;
-            const uint32_t d1 = (uint32_t)(it & 1) * NS;
+            const uint32_t d1 = (uint32_t)(it & 1) * 2 * NS;   // first of this chunk's two D1 halves
             const uint32_t par = (uint32_t)it & 1u;
             wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);   // U and gamma^C are read with plain loads
             if (warp < 2) {   // a6: V_new = U - W S  (token row = tid)
@@ -233,12 +248,14 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 wait(mma1_bar, par, 2);
                 KDA_PHASE(hdr, 18);  // MMA1
                 ptx::tc_fence_after();
-                uint32_t r[32];
+                uint32_t r[32], r2[32];
                 ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
+                ptx::tmem_ld_32x32b_x32(tmem_lane + d1 + NS, r2);
                 ptx::tmem_ld_wait();
                 float x[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) x[j] = __bfloat162float(U[j]) - __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j)
+                    x[j] = __bfloat162float(U[j]) - (__uint_as_float(r[j]) + __uint_as_float(r2[j]));
                 store_row32(vn, tid, x);
                 ptx::fence_async_smem();
                 ptx::tc_fence_before();
@@ -250,11 +267,12 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             KDA_PHASE(hdr, 20);  // MMA2
             ptx::tc_fence_after();
             {   // a8: S <- gamma^C . S + Kt^T V_new ; refresh the bf16 operand copy
-                uint32_t r[32];
+                uint32_t r[32], r2[32];
                 ptx::tmem_ld_32x32b_x32(tmem_lane + d3, r);
+                ptx::tmem_ld_32x32b_x32(tmem_lane + d3 + NS, r2);
                 ptx::tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) S[j] = gc * S[j] + __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) S[j] = gc * S[j] + (__uint_as_float(r[j]) + __uint_as_float(r2[j]));
                 store_row32(sbf, tid, S);
             }
             ptx::fence_async_smem();
@@ -269,8 +287,14 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 wait(&out_bar[it & 1], (uint32_t)(it >> 1) & 1u, 6);
                 ptx::tc_fence_after();
                 uint32_t r[32];
-                ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
-                ptx::tmem_ld_wait();
+                {
+                    uint32_t r2[32];
+                    ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
+                    ptx::tmem_ld_32x32b_x32(tmem_lane + d1 + NS, r2);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                }
                 if (i < len) {
 #pragma unroll
                     for (int j = 0; j < 32; j += 8)
@@ -310,7 +334,7 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
     ProfScope ps(PROF_INTER, st);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kD / NS, (unsigned)a.H, (unsigned)n_count);
-    cfg.blockDim = dim3(160);
+    cfg.blockDim = dim3(192);
     cfg.dynamicSmemBytes = Cfg::kSmem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
