@@ -32,6 +32,7 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, boo
 namespace {
 
 constexpr uint64_t kWaitLimitNs = 1000000000ull;   // 1 s per wait
+constexpr int kNCtrl = 2;                          // MMA-issuing threads (one per control warp): 2 or 4
 
 template <int NS> struct InterCfg {
     static_assert(NS == 32, "one 32-column accumulator block per matrix");
@@ -50,9 +51,25 @@ template <int NS> struct InterCfg {
     static constexpr uint32_t kTotal = kBars + 128;
     static constexpr uint32_t kSmem = kTotal + 1024;        // slack for manual 1024-byte alignment
     static constexpr uint32_t kTxBytes = kMainBytes + kUBytes;
-    static constexpr uint32_t kTmemCols = 256;              // 4 x D1 + 2 x D3, NS columns each
+    static constexpr uint32_t kTmemCols = kNCtrl == 2 ? 256 : 512;   // 2 kNCtrl x D1 + kNCtrl x D3, NS columns each
 };
 
+// sum of the kNCtrl partial accumulators (NS columns each, side by side in TMEM) of one matrix
+__device__ __forceinline__ void tmem_ld_sum(uint32_t taddr, float (&acc)[32]) {
+    uint32_t r[32], r2[32];
+    ptx::tmem_ld_32x32b_x32(taddr, r);
+    ptx::tmem_ld_32x32b_x32(taddr + 32, r2);
+    ptx::tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(r[j]) + __uint_as_float(r2[j]);
+    if (kNCtrl == 4) {
+        ptx::tmem_ld_32x32b_x32(taddr + 64, r);
+        ptx::tmem_ld_32x32b_x32(taddr + 96, r2);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[j] += __uint_as_float(r[j]) + __uint_as_float(r2[j]);
+    }
+}
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
     __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&p);
@@ -74,7 +91,7 @@ __device__ __forceinline__ void store_row32(uint8_t* img, int row, const float (
 // latencies never sit on the compute warps' path and the output conversion overlaps the next
 // chunk's first MMA.
 template <int NS>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(128 + 32 * kNCtrl, 1)
 kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader* hdr)
 {
     using Cfg = InterCfg<NS>;
@@ -117,8 +134,8 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < NSTG; ++s) ptx::mbar_init(&full[s], 1);
-        ptx::mbar_init(mma1_bar, 2);   // one commit from each control thread
-        ptx::mbar_init(mma2_bar, 2);
+        ptx::mbar_init(mma1_bar, kNCtrl);   // one commit from each control thread
+        ptx::mbar_init(mma2_bar, kNCtrl);
         ptx::mbar_init(&out_bar[0], 1);
         ptx::mbar_init(&out_bar[1], 1);
         ptx::mbar_init(sbf_ready, 128);
@@ -134,7 +151,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t d3 = 4 * NS;   // TMEM columns: D1 {parity 0,1} x {half 0,1} at 0..4 NS, D3 halves at 4 NS, 5 NS
+    const uint32_t d3 = 2 * kNCtrl * NS;   // TMEM columns: D1 {parity 0,1} x {part} first, then the D3 parts
 
     auto wait = [&](uint64_t* bar, uint32_t parity, int where) {
         if (*abort_flag) return;
@@ -145,11 +162,12 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     };
 
     if (warp >= 4) {
-        // ================= two control warps: lane 0 of each issues MMAs =================
+        // ================= control warps: lane 0 of each issues MMAs =================
         // Issuing one tcgen05.mma costs the issuing thread several tens of cycles whatever the tile
         // size, and both products on the sequential chain are tiny, so each is split along its
-        // summation index between the two threads, into two accumulators that are added when they
-        // are read back.  Thread A (warp 4) also issues the bulk copies and the output product.
+        // summation index between the control threads, into one accumulator each; the accumulators
+        // are added when they are read back.  Warp 4's thread also issues the bulk copies and the
+        // output product.
         const int half = warp - 4;
         if ((tid & 31) == 0) {
             const uint32_t idesc = ptx::umma_idesc_bf16(128, NS) | ptx::kIdescBMajorMN;
@@ -174,15 +192,17 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 const int s = it % NSTG;
                 const uint32_t sb = ptx::smem_u32(smem + s * Cfg::kStage);
                 // accumulators of this chunk: D1 (two parities x two halves), D3 (two halves)
-                const uint32_t d1 = tmem_base + (uint32_t)((it & 1) * 2 + half) * NS;
+                const uint32_t d1 = tmem_base + (uint32_t)((it & 1) * kNCtrl + half) * NS;
                 // MMA1(it): D1 = [W ; Gamma.Q] S, this thread's half of the sum over dk
                 wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);
                 wait(sbf_ready, (uint32_t)it & 1u, 4);
                 ptx::tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kQW + half * tc::QW_HALF + k * 32),
-                                   ptx::umma_desc_sw128_mn(sbf_a + (half * 4 + k) * 2048, 8192), idesc, k > 0);
+                for (int k = 0; k < 8 / kNCtrl; ++k) {
+                    const int kk = half * (8 / kNCtrl) + k;   // 16-wide step of the sum over dk
+                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sb + Cfg::kQW + (kk >> 2) * tc::QW_HALF + (kk & 3) * 32),
+                                   ptx::umma_desc_sw128_mn(sbf_a + kk * 2048, 8192), idesc, k > 0);
+                }
                 ptx::umma_commit(mma1_bar);
                 // the stage of the previous chunk is free now (its readers arrived on sbf_ready)
                 if (half == 0 && it > 0 && loads_issued < nchunks) { issue_loads(loads_issued); ++loads_issued; }
@@ -191,10 +211,11 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 wait(vn_ready, (uint32_t)it & 1u, 5);
                 ptx::tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < 2; ++k)
-                    ptx::umma_bf16(tmem_base + d3 + half * NS,
-                                   ptx::umma_desc_sw128(sb + Cfg::kKT + (half * 2 + k) * 32),
-                                   ptx::umma_desc_sw128_mn(vn_a + (half * 2 + k) * 2048, 8192), idesc, k > 0);
+                for (int k = 0; k < 4 / kNCtrl; ++k) {
+                    const int kk = half * (4 / kNCtrl) + k;   // 16-wide step of the sum over tokens
+                    ptx::umma_bf16(tmem_base + d3 + half * NS, ptx::umma_desc_sw128(sb + Cfg::kKT + kk * 32),
+                                   ptx::umma_desc_sw128_mn(vn_a + kk * 2048, 8192), idesc, k > 0);
+                }
                 ptx::umma_commit(mma2_bar);
                 if (half == 0) {
                     // D1[64:128] += Aqk V_new.  The 128-row A operand starts 64 rows before Aqk: those
@@ -236,7 +257,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         for (int it = 0; it < nchunks; ++it) {
             const int s = it % NSTG;
             const uint8_t* sb = smem + s * Cfg::kStage;
-            const uint32_t d1 = (uint32_t)(it & 1) * 2 * NS;   // first of this chunk's two D1 halves
+            const uint32_t d1 = (uint32_t)(it & 1) * kNCtrl * NS;   // first of this chunk's D1 parts
             const uint32_t par = (uint32_t)it & 1u;
             wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);   // U and gamma^C are read with plain loads
             if (warp < 2) {   // a6: V_new = U - W S  (token row = tid)
@@ -248,14 +269,10 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 wait(mma1_bar, par, 2);
                 KDA_PHASE(hdr, 18);  // MMA1
                 ptx::tc_fence_after();
-                uint32_t r[32], r2[32];
-                ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
-                ptx::tmem_ld_32x32b_x32(tmem_lane + d1 + NS, r2);
-                ptx::tmem_ld_wait();
                 float x[32];
+                tmem_ld_sum(tmem_lane + d1, x);
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    x[j] = __bfloat162float(U[j]) - (__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                for (int j = 0; j < 32; ++j) x[j] = __bfloat162float(U[j]) - x[j];
                 store_row32(vn, tid, x);
                 ptx::fence_async_smem();
                 ptx::tc_fence_before();
@@ -267,12 +284,10 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             KDA_PHASE(hdr, 20);  // MMA2
             ptx::tc_fence_after();
             {   // a8: S <- gamma^C . S + Kt^T V_new ; refresh the bf16 operand copy
-                uint32_t r[32], r2[32];
-                ptx::tmem_ld_32x32b_x32(tmem_lane + d3, r);
-                ptx::tmem_ld_32x32b_x32(tmem_lane + d3 + NS, r2);
-                ptx::tmem_ld_wait();
+                float ds[32];
+                tmem_ld_sum(tmem_lane + d3, ds);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) S[j] = gc * S[j] + (__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                for (int j = 0; j < 32; ++j) S[j] = gc * S[j] + ds[j];
                 store_row32(sbf, tid, S);
             }
             ptx::fence_async_smem();
@@ -288,12 +303,10 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::tc_fence_after();
                 uint32_t r[32];
                 {
-                    uint32_t r2[32];
-                    ptx::tmem_ld_32x32b_x32(tmem_lane + d1, r);
-                    ptx::tmem_ld_32x32b_x32(tmem_lane + d1 + NS, r2);
-                    ptx::tmem_ld_wait();
+                    float ov[32];
+                    tmem_ld_sum(tmem_lane + d1, ov);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(ov[j]);
                 }
                 if (i < len) {
 #pragma unroll
@@ -334,7 +347,7 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
     ProfScope ps(PROF_INTER, st);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kD / NS, (unsigned)a.H, (unsigned)n_count);
-    cfg.blockDim = dim3(192);
+    cfg.blockDim = dim3(128 + 32 * kNCtrl);
     cfg.dynamicSmemBytes = Cfg::kSmem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
