@@ -176,6 +176,15 @@ kda_status_t kda_decode_step_host(const void *q_host, const void *k_host, const 
 kda_status_t kda_check_status(void *workspace, void *cuda_stream);
 
 /*
+ * Self-test of the bounded-wait mechanism every tensor-core kernel of this library relies on (no
+ * counterpart in the paper).  Launches one warp that waits, for at most limit_ms (1..1000), on a
+ * barrier that nothing ever completes; the wait must give up and record KDA_ERR_TIMEOUT in the
+ * status word at the start of `workspace` (>= 256 bytes, device), which kda_check_status then
+ * reports.  The CUDA context stays usable.
+ */
+kda_status_t kda_selftest_wait_timeout(void *workspace, int limit_ms, void *cuda_stream);
+
+/*
  * Optional per-kernel timing for benchmarks.  While enabled, every kernel launch of this library
  * is bracketed by CUDA events on the launching stream (at most 8192 launches are recorded; enabling
  * resets the record).  kda_profile_read synchronises the device and returns the summed duration and

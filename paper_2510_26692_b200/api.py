@@ -71,6 +71,8 @@ def load():
                                          i32, vp, sz, vp]
     lib.kda_check_status.restype = i32
     lib.kda_check_status.argtypes = [vp, vp]
+    lib.kda_selftest_wait_timeout.restype = i32
+    lib.kda_selftest_wait_timeout.argtypes = [vp, i32, vp]
     lib.kda_profile_enable.restype = None
     lib.kda_profile_enable.argtypes = [i32]
     lib.kda_profile_read.restype = i32
@@ -236,6 +238,13 @@ def kda_decode_step_host(q, k, v, log_alpha, beta, S_dev, state_slot_host, o, n_
         _ptr(o, False, et, "o"), int(n_seqs), int(H), int(dk), int(dv), float(scale), int(dt),
         _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
     _check(rc)
+
+
+def kda_selftest_wait_timeout(workspace, limit_ms: int = 20, stream=None):
+    """``kda_selftest_wait_timeout``: makes one bounded device-side wait run out; afterwards
+    ``kda_check_status(workspace)`` raises ``KdaError`` with KDA_ERR_TIMEOUT."""
+    _check(load().kda_selftest_wait_timeout(_ptr(workspace, True, None, "workspace"), int(limit_ms),
+                                            _stream(stream)))
 
 
 def kda_profile_enable(on: bool):

@@ -387,6 +387,15 @@ kda_status_t kda_decode_step_host(const void* q_host, const void* k_host, const 
     return KDA_OK;
 }
 
+kda_status_t kda_selftest_wait_timeout(void* workspace, int limit_ms, void* cuda_stream)
+{
+    if (!workspace || limit_ms <= 0 || limit_ms > 1000)
+        return fail(KDA_ERR_INVALID_ARG, "kda_selftest_wait_timeout: workspace NULL or limit outside 1..1000 ms");
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    KDA_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st));
+    return launch_wait_selftest(reinterpret_cast<WsHeader*>(workspace), (uint64_t)limit_ms * 1000000ull, st);
+}
+
 void kda_profile_enable(int on)
 {
     std::lock_guard<std::mutex> lk(g_prof.mu);

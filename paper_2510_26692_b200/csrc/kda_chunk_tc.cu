@@ -364,6 +364,29 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
 
 }  // namespace
 
+// Self-test of the bounded-wait path: one CTA waits on an mbarrier that nothing ever arrives on,
+// with a short limit, and must come back with KDA_ERR_TIMEOUT in the status word.
+__global__ void kda_wait_selftest_kernel(WsHeader* hdr, uint64_t limit_ns)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (!ptx::mbar_wait(&bar, 0, limit_ns)) {
+        if (atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = 99;
+    }
+}
+
+kda_status_t launch_wait_selftest(WsHeader* hdr, uint64_t limit_ns, cudaStream_t st)
+{
+    kda_wait_selftest_kernel<<<1, 32, 0, st>>>(hdr, limit_ns);
+    count_launch();
+    KDA_CUDA_TRY(cudaGetLastError());
+    return KDA_OK;
+}
+
 size_t tc_tile_bytes() { return tc::TILE_BYTES; }
 
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,

@@ -177,6 +177,8 @@ size_t tc_tile_bytes();
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
                              WsHeader* hdr, bool clear_status, cudaStream_t st);
 
+kda_status_t launch_wait_selftest(WsHeader* hdr, uint64_t limit_ns, cudaStream_t st);
+
 // clears the status word and (packed batches) builds chunk_cu[n_seqs+1] from cu_seqlens
 kda_status_t launch_prep(WsHeader* hdr, const int32_t* cu_seqlens, int32_t* chunk_cu, int n_seqs,
                          cudaStream_t st);

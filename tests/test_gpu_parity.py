@@ -296,3 +296,16 @@ def test_status_word_clean(oracle_mod):
     K.kda_chunk_fwd(g["q"], g["k"], g["v"], g["log_alpha"], g["beta"], None, o, None, None, None,
                     1, 128, 2, 128, 128, 64, 1.0, K.KDA_BF16, ws)
     K.kda_check_status(ws)   # raises KdaError on a device-side timeout
+
+
+def test_bounded_wait_reports_timeout(oracle_mod):
+    """A device-side wait that nothing completes gives up after its limit, records KDA_ERR_TIMEOUT
+    in the status word, and leaves the context usable (the next prefill still matches the oracle)."""
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda:0")
+    K.kda_selftest_wait_timeout(ws, 20)
+    with pytest.raises(K.KdaError) as ei:
+        K.kda_check_status(ws)
+    assert ei.value.code == 5
+    K.kda_check_status(ws)    # the word was cleared by the failed check
+    d = inputs.chunk_inputs([130], H=2, dtype=torch.bfloat16, seed=35, s0_std=0.02)
+    check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
