@@ -4,12 +4,14 @@
 // One CTA owns one (sequence, head, 32-column slice of dv) -- the columns of the state are
 // independent under  S <- Diag(gamma^C) S + Kt^T (U - W S) -- and walks the sequence's chunks in
 // order.  Per chunk:
-//   MMA1  D1[128 x 32]  = [W ; Gamma.Q] (128 x 128, bf16)  x  S (128 x 32, bf16 copy of the state)
+//   MMA1  D1[128 x 32]  = [W' ; Q'] (128 x 128, bf16)  x  bf16(exp(G_m) . S) (128 x 32)
+//         (the tile holds W, Gamma.Q and K relative to the chunk's middle row m; the true scales
+//         exp(G_m), exp(G_C - G_m) are applied to the state here, in fp32)
 //         rows 0-63 of D1 = W S, rows 64-127 = (Gamma.Q) S  (inter-chunk output term)
 //   a6    V_new = U - W S            TMEM -> registers, rounded to bf16 into shared memory
 //   MMA2  D1[64:128] += Aqk V_new    (a7, intra-chunk output term)
-//         D3[128 x 32] = Kt^T V_new  (a8, Kt = (gamma^C/Gamma).K)
-//   a8    S <- gamma^C . S + D3      fp32 master copy of the state lives in registers (thread = dk
+//         D3[128 x 32] = K'^T V_new  (a8; (gamma^C/Gamma).K = exp(G_C - G_m) . K')
+//   a8    S <- gamma^C . S + exp(G_C - G_m) . D3      fp32 master copy of the state lives in registers (thread = dk
 //                                    row), refreshed bf16 copy goes back to shared memory
 //   MMA1 of the next chunk is issued (D1 is double-buffered), and while it runs:
 //   a7    O = rows 64-127 of D1 -> bf16 -> global
@@ -38,11 +40,11 @@ template <int NS> struct InterCfg {
     static_assert(NS == 32, "one 32-column accumulator block per matrix");
     static constexpr int kStages = 3;
     static constexpr uint32_t kQW = 0;                      // [2 K-halves][128][64]: rows 0-63 W, 64-127 Gamma.Q
-    static constexpr uint32_t kKT = 32768;                  // [128 dk][64 tokens]
+    static constexpr uint32_t kKT = 32768;                  // K': [2 dk-halves][64 tokens][64], MN-major A operand
     static constexpr uint32_t kAQ = 49152;                  // [64][64]; used as rows 64-127 of a 128-row operand
-    static constexpr uint32_t kGC = 57344;                  // gamma^C, 128 fp32
-    static constexpr uint32_t kMainBytes = 57856;           // QW | Kt | Aqk | gamma^C are contiguous in a tile
-    static constexpr uint32_t kU = 57856;                   // [64 tokens][NS] block of U
+    static constexpr uint32_t kGC = 57344;                  // gamma^C | exp(G_m) | exp(G_C - G_m), 128 fp32 each
+    static constexpr uint32_t kMainBytes = tc::OFF_U;       // the images and the three vectors are contiguous in a tile
+    static constexpr uint32_t kU = tc::OFF_U;               // [64 tokens][NS] block of U
     static constexpr uint32_t kUBytes = tc::U_BLOCK;
     static constexpr uint32_t kStage = (kU + kUBytes + 1023) / 1024 * 1024;
     static constexpr uint32_t kSbf = kStages * kStage;      // B operand of MMA1, MN-major: [128 dk rows][128 B]
@@ -206,15 +208,18 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::umma_commit(mma1_bar);
                 // the stage of the previous chunk is free now (its readers arrived on sbf_ready)
                 if (half == 0 && it > 0 && loads_issued < nchunks) { issue_loads(loads_issued); ++loads_issued; }
-                // MMA2(it): D3 = Kt^T V_new, this thread's half of the sum over the chunk's tokens.
+                // MMA2(it): D3 = K'^T V_new (K' token-major = MN-major A operand), this thread's half of the
+                // sum over the chunk's tokens.
                 // The state product sits on the sequential chain: it is issued and committed first.
                 wait(vn_ready, (uint32_t)it & 1u, 5);
                 ptx::tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < 4 / kNCtrl; ++k) {
                     const int kk = half * (4 / kNCtrl) + k;   // 16-wide step of the sum over tokens
-                    ptx::umma_bf16(tmem_base + d3 + half * NS, ptx::umma_desc_sw128(sb + Cfg::kKT + kk * 32),
-                                   ptx::umma_desc_sw128_mn(vn_a + kk * 2048, 8192), idesc, k > 0);
+                    ptx::umma_bf16(tmem_base + d3 + half * NS,
+                                   ptx::umma_desc_sw128_mn(sb + Cfg::kKT + kk * 2048, tc::KI_HALF),
+                                   ptx::umma_desc_sw128_mn(vn_a + kk * 2048, 8192), idesc | ptx::kIdescAMajorMN,
+                                   k > 0);
                 }
                 ptx::umma_commit(mma2_bar);
                 if (half == 0) {
@@ -249,7 +254,20 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             if (a.S_in) x = *reinterpret_cast<const float4*>(a.S_in + sbase + j);
             S[j] = x.x; S[j + 1] = x.y; S[j + 2] = x.z; S[j + 3] = x.w;
         }
-        store_row32(sbf, tid, S);
+        // the operand copy carries the next chunk's reference scale: bf16(exp(G_m) . S)
+        auto ref_scale_of = [&](int it_next) {   // exp(G_m) of a chunk (0 past the last one)
+            if (it_next >= nchunks) return 0.f;
+            const int sn = it_next % NSTG;
+            wait(&full[sn], (uint32_t)(it_next / NSTG) & 1u, 8);
+            return reinterpret_cast<const float*>(smem + sn * Cfg::kStage + Cfg::kGC + 512)[tid];
+        };
+        auto store_scaled = [&](float cgn) {
+            float z[NS];
+#pragma unroll
+            for (int j = 0; j < NS; ++j) z[j] = cgn * S[j];
+            store_row32(sbf, tid, z);
+        };
+        store_scaled(ref_scale_of(0));
         ptx::fence_async_smem();
         ptx::mbar_arrive(sbf_ready);
         KDA_PHASE(hdr, 16);  // set-up
@@ -279,20 +297,34 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::mbar_arrive(vn_ready);
                 KDA_PHASE(hdr, 19);  // V_new
             }
-            const float gc = reinterpret_cast<const float*>(sb + Cfg::kGC)[tid];
+            const float gc = reinterpret_cast<const float*>(sb + Cfg::kGC)[tid];          // gamma^C
+            const float ct = reinterpret_cast<const float*>(sb + Cfg::kGC + 1024)[tid];   // exp(G_C - G_m)
+            const float cgn = ref_scale_of(it + 1);   // fetched off the chain, before the wait below
+            // the next operand copy is exp(G_m') . S_new = (cgn gc) . S + (cgn ct) . D3: everything that
+            // does not need D3 is formed before the wait
+            float zpre[NS];
+            const float zb = cgn * ct;
+            {
+                const float za = cgn * gc;
+#pragma unroll
+                for (int j = 0; j < NS; ++j) zpre[j] = za * S[j];
+            }
             wait(mma2_bar, par, 3);
             KDA_PHASE(hdr, 20);  // MMA2
             ptx::tc_fence_after();
-            {   // a8: S <- gamma^C . S + Kt^T V_new ; refresh the bf16 operand copy
+            {   // a8: S <- gamma^C . S + exp(G_C - G_m) . (K'^T V_new) ; refresh the bf16 operand copy
                 float ds[32];
                 tmem_ld_sum(tmem_lane + d3, ds);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) S[j] = gc * S[j] + ds[j];
-                store_row32(sbf, tid, S);
+                for (int j = 0; j < 32; ++j) zpre[j] = fmaf(zb, ds[j], zpre[j]);
+                store_row32(sbf, tid, zpre);
+                ptx::fence_async_smem();
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(sbf_ready);
+                // the fp32 master copy itself is not on the chain
+#pragma unroll
+                for (int j = 0; j < 32; ++j) S[j] = fmaf(ct, ds[j], gc * S[j]);
             }
-            ptx::fence_async_smem();
-            ptx::tc_fence_before();
-            ptx::mbar_arrive(sbf_ready);
             KDA_PHASE(hdr, 21);  // state update
             if (warp >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64)
                 const int i = tid - 64;

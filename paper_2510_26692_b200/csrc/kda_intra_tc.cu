@@ -7,8 +7,8 @@
 //        gated operands, all bf16:  Kg = K exp(G - G_m),  Qg = scale Q exp(G - G_m),
 //        Ki = K exp(G_m - G)   (m = row 31, the middle of the chunk, so that neither factor of
 //        exp(G_i - G_j) = exp(G_i - G_m) exp(G_m - G_j) leaves the bf16/fp32 range; exponents are
-//        clamped to +-80),
-//        and for the inter-chunk stage  scale Q exp(G)  and  (K exp(G_C - G))^T
+//        clamped to +-80).  The same three images serve the inter-chunk stage, which restores the
+//        true scales exp(G_m), exp(G_C - G_m) in fp32 on its side
 //   a2/a5  one tcgen05 MMA group  [Kg ; Qg] (128 x 128)  x  Ki^T (128 x 64)  ->  TMEM:
 //        rows 0-63  = raw key Gram matrix, rows 64-127 = raw query-key matrix
 //        L = Diag(beta) StrictTril(rows 0-63) (fp32, shared memory);  Aqk = Tril(rows 64-127)
@@ -18,14 +18,12 @@
 //        (mma.sync, tf32 inputs, fp32 accumulation; T is rounded to bf16 afterwards anyway)
 //   a4   Mm = T Diag(beta) (bf16);  second MMA group  [Mm ; Mm] (128 x 64) x [Kg | V] (64 x 256) -> TMEM
 //        (the rows are held twice so that all 128 TMEM lanes, i.e. all eight warps, share the read-out);
-//        W = (Mm Kg) exp(G_m) column-wise,  U = Mm V.  Kg and V are used as MN-major B operands in
+//        W' = Mm Kg (= W / exp(G_m) column-wise),  U = Mm V.  Kg and V are used as MN-major B operands in
 //        the token-major layout they already have in shared memory.
 // Outputs go to the scratch tile of kda_tiles.cuh as ready-made operand images of the inter-chunk
 // kernel.  Tail chunks: rows past the sequence end behave as identity steps (log alpha = 0,
 // beta = 0, k = q = v = 0).
 #include <cuda.h>
-
-#include <type_traits>
 
 #include "kda_common.cuh"
 #include "kda_ptx.cuh"
@@ -48,16 +46,13 @@ constexpr uint32_t S_M = 65536;       // 8 KiB: Aqk staging; start of the 32 KiB
 constexpr uint32_t S_A = 73728;       // fp32 [64][LDT]: L, later X in its sub-diagonal blocks
 constexpr uint32_t S_T = S_A + 64 * LDT * 4;   // fp32 [64][LDT]: T
 // staging of outputs for bulk stores (aliases buffers that are dead at the time):
-constexpr uint32_t S_QG = S_M;                 // scale Q exp(G): [2 halves][64][64] bf16, 16 KiB   (phase 1)
-constexpr uint32_t S_KT = S_M + 16384;         // (K exp(G_C - G))^T: [128][64] bf16, 16 KiB        (phase 1)
-constexpr uint32_t S_TOT = S_M + 32768;        // scan exchange [8][128] fp32, 4 KiB
+constexpr uint32_t S_TOT = S_M + 32768;        // scan exchange [8..16][128] fp32, <= 8 KiB
 constexpr uint32_t S_AQ = S_M;                 // Aqk image [64][64] bf16 (after the first MMA group)
 constexpr uint32_t S_MM = S_KI;                // [128][64] bf16: T Diag(beta) twice (rows 64-127 repeat rows 0-63)
 constexpr uint32_t S_W = S_M;                  // W image [2 halves][64][64] bf16 (after the second group)
 constexpr uint32_t S_U = S_M + 16384;          // U: four [64][32] bf16 blocks
 constexpr uint32_t S_BETA = S_T + 64 * LDT * 4;
-constexpr uint32_t S_CG = S_BETA + 256;        // exp(G_m) per channel (undoes the Kg reference)
-constexpr uint32_t S_BAR = S_CG + 512;          // mma barrier, tma barrier, TMEM slot
+constexpr uint32_t S_BAR = S_BETA + 256;        // mma barrier, tma barrier, TMEM slot
 constexpr uint32_t S_TOTAL = S_BAR + 64;
 #ifndef KDA_INTRA_THREADS
 #define KDA_INTRA_THREADS 256
@@ -140,7 +135,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     float* sT = reinterpret_cast<float*>(smem + S_T);
     float* sTot = reinterpret_cast<float*>(smem + S_TOT);   // [16][128] during the scan
     float* sBeta = reinterpret_cast<float*>(smem + S_BETA);
-    float* sCG = reinterpret_cast<float*>(smem + S_CG);
     uint64_t* mma_bar = reinterpret_cast<uint64_t*>(smem + S_BAR);
     uint64_t* tma_bar = mma_bar + 1;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_bar + 2);
@@ -253,21 +247,16 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     }
 
     // ---- gated operands ---------------------------------------------------------------------------------
-    // exp(G) = exp(G - G_m) exp(G_m) and exp(G_C - G) = exp(G_m - G) exp(G_C - G_m) reuse the two
-    // exponentials of the intra-chunk operands unless a channel decays by more than e^-80 on one
-    // side of the middle row, in which case they are evaluated directly (no underflow of the factor)
-    float cg[4], ct[4];
-    bool harsh = false;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        cg[e] = ex2(gref[e]);               // exp(G_m)
-        ct[e] = ex2(glast[e] - gref[e]);    // exp(G_C - G_m)
-        harsh = harsh || (gref[e] < -kClamp2) || (glast[e] - gref[e] < -kClamp2);
-    }
+    // the true scales exp(G_m), exp(G_C - G_m) and gamma^C go to the tile as fp32 vectors; the
+    // inter-chunk kernel applies them to the state in fp32
     if (warp == 0) {
-        *reinterpret_cast<float4*>(tile + tc::OFF_GC + d0 * 4) =
+        *reinterpret_cast<float4*>(tile + tc::OFF_GV + d0 * 4) =
             make_float4(ex2(glast[0]), ex2(glast[1]), ex2(glast[2]), ex2(glast[3]));
-        *reinterpret_cast<float4*>(sCG + d0) = make_float4(cg[0], cg[1], cg[2], cg[3]);
+        *reinterpret_cast<float4*>(tile + tc::OFF_GV + 512 + d0 * 4) =
+            make_float4(ex2(gref[0]), ex2(gref[1]), ex2(gref[2]), ex2(gref[3]));
+        *reinterpret_cast<float4*>(tile + tc::OFF_GV + 1024 + d0 * 4) =
+            make_float4(ex2(glast[0] - gref[0]), ex2(glast[1] - gref[1]), ex2(glast[2] - gref[2]),
+                        ex2(glast[3] - gref[3]));
     }
     KDA_PHASE(hdr, 10);  // prefix + per-channel factors
     if (!ptx::mbar_wait(tma_bar, tma_parity, kWaitLimitNs)) timed_out = true;   // k, q, v have landed
@@ -281,77 +270,33 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         }
     }
     const int hf = c4 >> 4;                       // K-half (channels 0-63 / 64-127)
-    uint32_t ktb[4][kRPT / 2];                    // (K exp(G_C - G))^T: 4 channels x kRPT tokens, bf16 pairs
-    auto gate_rows = [&](auto harsh_tag) {
-        constexpr bool kHarsh = decltype(harsh_tag)::value;
 #pragma unroll
-        for (int r = 0; r < kRPT; ++r) {
-            const int i = i0 + r;
-            const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
-            uint8_t* pk = smem + S_KQ + hf * S_KQ_HALF + off;
-            uint2 k2 = *reinterpret_cast<const uint2*>(pk);
-            uint2 q2 = *reinterpret_cast<const uint2*>(pk + 8192);
-            if (i >= L.len) k2 = q2 = make_uint2(0u, 0u);
-            if (!has_q) q2 = make_uint2(0u, 0u);
-            const float kf[4] = {__uint_as_float(k2.x << 16), __uint_as_float(k2.x & 0xffff0000u),
-                                 __uint_as_float(k2.y << 16), __uint_as_float(k2.y & 0xffff0000u)};
-            const float qf[4] = {__uint_as_float(q2.x << 16), __uint_as_float(q2.x & 0xffff0000u),
-                                 __uint_as_float(q2.y << 16), __uint_as_float(q2.y & 0xffff0000u)};
-            float okg[4], oqg[4], oki[4], oqt[4], okt[4];
+    for (int r = 0; r < kRPT; ++r) {
+        const int i = i0 + r;
+        const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
+        uint8_t* pk = smem + S_KQ + hf * S_KQ_HALF + off;
+        uint2 k2 = *reinterpret_cast<const uint2*>(pk);
+        uint2 q2 = *reinterpret_cast<const uint2*>(pk + 8192);
+        if (i >= L.len) k2 = q2 = make_uint2(0u, 0u);
+        if (!has_q) q2 = make_uint2(0u, 0u);
+        const float kf[4] = {__uint_as_float(k2.x << 16), __uint_as_float(k2.x & 0xffff0000u),
+                             __uint_as_float(k2.y << 16), __uint_as_float(k2.y & 0xffff0000u)};
+        const float qf[4] = {__uint_as_float(q2.x << 16), __uint_as_float(q2.x & 0xffff0000u),
+                             __uint_as_float(q2.y << 16), __uint_as_float(q2.y & 0xffff0000u)};
+        float okg[4], oqg[4], oki[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float gg = G[r][e] + base[e];
-                const float x = fminf(fmaxf(gg - gref[e], -kClamp2), kClamp2);
-                const float e1 = ex2(x);                     // exp(G - G_m)
-                const float e2 = ex2(-x);                    // exp(G_m - G)
-                const float qs = a.scale * qf[e];
-                okg[e] = kf[e] * e1;
-                oqg[e] = qs * e1;
-                oki[e] = kf[e] * e2;
-                if (!kHarsh) {
-                    oqt[e] = oqg[e] * cg[e];
-                    okt[e] = oki[e] * ct[e];
-                } else {
-                    oqt[e] = qs * ex2(gg);
-                    okt[e] = kf[e] * ex2(glast[e] - gg);
-                }
-            }
-            *reinterpret_cast<uint2*>(pk) = make_uint2(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]));
-            *reinterpret_cast<uint2*>(pk + 8192) =
-                make_uint2(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]));
-            *reinterpret_cast<uint2*>(smem + S_KI + hf * S_KI_HALF + off) =
-                make_uint2(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]));
-            *reinterpret_cast<uint2*>(smem + S_QG + hf * 8192 + off) =
-                make_uint2(pack_bf16(oqt[0], oqt[1]), pack_bf16(oqt[2], oqt[3]));
-            if (r & 1) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    __nv_bfloat16 hi = __float2bfloat16_rn(okt[e]);
-                    ktb[e][r >> 1] |= (uint32_t)(*reinterpret_cast<uint16_t*>(&hi)) << 16;
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    __nv_bfloat16 lo = __float2bfloat16_rn(okt[e]);
-                    ktb[e][r >> 1] = (uint32_t)(*reinterpret_cast<uint16_t*>(&lo));
-                }
-            }
+        for (int e = 0; e < 4; ++e) {
+            const float x = fminf(fmaxf(G[r][e] + base[e] - gref[e], -kClamp2), kClamp2);
+            const float e1 = ex2(x);                     // exp(G - G_m)
+            const float e2 = ex2(-x);                    // exp(G_m - G)
+            okg[e] = kf[e] * e1;
+            oqg[e] = a.scale * qf[e] * e1;
+            oki[e] = kf[e] * e2;
         }
-    };
-    if (!harsh) gate_rows(std::false_type{});
-    else gate_rows(std::true_type{});
-    // (K exp(G_C - G))^T: row = channel; this warp's tokens are one 16-byte chunk (8 warps) or half of
-    // one (16 warps)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int d = d0 + e;
-        if (kRPT == 8) {
-            *reinterpret_cast<uint4*>(smem + S_KT + d * 128 + ((warp ^ (d & 7)) << 4)) =
-                make_uint4(ktb[e][0], ktb[e][1], ktb[e][kRPT / 2 - 2], ktb[e][kRPT / 2 - 1]);
-        } else {
-            *reinterpret_cast<uint2*>(smem + S_KT + d * 128 + (((warp >> 1) ^ (d & 7)) << 4) + (warp & 1) * 8) =
-                make_uint2(ktb[e][0], ktb[e][1]);
-        }
+        *reinterpret_cast<uint2*>(pk) = make_uint2(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]));
+        *reinterpret_cast<uint2*>(pk + 8192) = make_uint2(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]));
+        *reinterpret_cast<uint2*>(smem + S_KI + hf * S_KI_HALF + off) =
+            make_uint2(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]));
     }
 
     KDA_PHASE(hdr, 12);  // element loop + stores (thread 0)
@@ -364,9 +309,10 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     // ---- a2 + a5: [Kg ; Qg] Ki^T ------------------------------------------------------------------------
     if (t == kBulkThread) {
         // phase-1 outputs leave through the TMA engine while the MMA runs
-        ptx::bulk_s2g(tile + tc::OFF_QW + 8192, smem + S_QG, 8192);
-        ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF + 8192, smem + S_QG + 8192, 8192);
-        ptx::bulk_s2g(tile + tc::OFF_KT, smem + S_KT, 16384);
+        // Q' (rows 64-127 of both K-halves of the operand image) and K' are tile contents as they are
+        ptx::bulk_s2g(tile + tc::OFF_QW + 8192, smem + S_KQ + 8192, 8192);
+        ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF + 8192, smem + S_KQ + S_KQ_HALF + 8192, 8192);
+        ptx::bulk_s2g(tile + tc::OFF_KI, smem + S_KI, 16384);
         ptx::bulk_commit();
     }
     if (t == 0) {
@@ -379,7 +325,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         ptx::umma_commit(mma_bar);
     }
     if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) timed_out = true;
-    if (t == kBulkThread) ptx::bulk_wait_read0();   // staging buffers are about to be reused
     __syncthreads();
     KDA_PHASE(hdr, 2);   // first MMA group
     ptx::tc_fence_after();
@@ -496,7 +441,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
             *reinterpret_cast<uint4*>(dst + 8192) = pk;   // rows 64-127 repeat rows 0-63
         }
     }
-    if (t == kBulkThread) ptx::bulk_wait_read0();   // Aqk staging is reused by the W/U epilogue
+    if (t == kBulkThread) ptx::bulk_wait_read0();   // K' (overwritten by the Mm image) and the Aqk staging (reused by the W/U epilogue) have been read out
     ptx::fence_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
@@ -535,18 +480,15 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         for (int b = 0; b < NCE / 32; ++b)
             ptx::tmem_ld_32x32b_x32(ta + b * 32, reinterpret_cast<uint32_t(&)[32]>(r[b * 32]));
         ptx::tmem_ld_wait();
-        if (col0 < 128) {   // W = (Mm Kg) exp(G_m): K-half col0 / 64 of the [W ; Gamma.Q] image
+        if (col0 < 128) {   // W' = Mm Kg: K-half col0 / 64 of the [W' ; Q'] image
             uint8_t* dst = smem + S_W + (col0 >> 6) * 8192;
 #pragma unroll
-            for (int j8 = 0; j8 < NCE; j8 += 8) {
-                const float4 s0 = *reinterpret_cast<const float4*>(sCG + col0 + j8);
-                const float4 s1 = *reinterpret_cast<const float4*>(sCG + col0 + j8 + 4);
+            for (int j8 = 0; j8 < NCE; j8 += 8)
                 *reinterpret_cast<uint4*>(dst + ptx::sw128_off(i, (col0 & 63) + j8)) =
-                    make_uint4(pack_bf16(__uint_as_float(r[j8]) * s0.x, __uint_as_float(r[j8 + 1]) * s0.y),
-                               pack_bf16(__uint_as_float(r[j8 + 2]) * s0.z, __uint_as_float(r[j8 + 3]) * s0.w),
-                               pack_bf16(__uint_as_float(r[j8 + 4]) * s1.x, __uint_as_float(r[j8 + 5]) * s1.y),
-                               pack_bf16(__uint_as_float(r[j8 + 6]) * s1.z, __uint_as_float(r[j8 + 7]) * s1.w));
-            }
+                    make_uint4(pack_bf16(__uint_as_float(r[j8]), __uint_as_float(r[j8 + 1])),
+                               pack_bf16(__uint_as_float(r[j8 + 2]), __uint_as_float(r[j8 + 3])),
+                               pack_bf16(__uint_as_float(r[j8 + 4]), __uint_as_float(r[j8 + 5])),
+                               pack_bf16(__uint_as_float(r[j8 + 6]), __uint_as_float(r[j8 + 7])));
         } else {            // U: 32-column blocks (col0 - 128) / 32 ...
 #pragma unroll
             for (int j8 = 0; j8 < NCE; j8 += 8) {

@@ -186,6 +186,7 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t smem_addr, uint3
     return d;
 }
 constexpr uint32_t kIdescBMajorMN = 1u << 16;   // OR into the instruction descriptor: B is MN-major
+constexpr uint32_t kIdescAMajorMN = 1u << 15;   // A is MN-major
 // Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, both operands K-major.
 __device__ __forceinline__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
