@@ -173,7 +173,8 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         ho = (int)(tl - gl * (uint32_t)a.H);
         Lo = locate_chunk(a, a.g0 + gl);
     };
-    auto issue_prefetch = [&](const ChunkLoc& Lo, int ho) {
+    // log alpha -> registers (may be issued while the second MMA group still runs)
+    auto prefetch_regs = [&](const ChunkLoc& Lo, int ho) {
         const float* gp = a.log_alpha + ((size_t)Lo.tok0 * a.H + ho) * kD + d0;
 #pragma unroll
         for (int r = 0; r < kRPT; ++r) {
@@ -184,6 +185,9 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
                 G[r][0] = G[r][1] = G[r][2] = G[r][3] = 0.f;
             }
         }
+    };
+    // k, q, v, beta -> shared memory (only once the second MMA group has finished reading Kg and V)
+    auto prefetch_bufs = [&](const ChunkLoc& Lo, int ho) {
         if (t == kBulkThread) {
             ptx::mbar_expect_tx(tma_bar, 3 * 16384);
             const int x = ho * kD, y = (int)Lo.tok0;
@@ -213,7 +217,8 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     int h = 0;
     if (cur < ntiles) {
         locate(cur, L, h);
-        issue_prefetch(L, h);
+        prefetch_regs(L, h);
+        prefetch_bufs(L, h);
     }
     for (; cur < ntiles; cur += gridDim.x) {
     char* tile = tiles + (size_t)cur * tc::TILE_BYTES;
@@ -229,7 +234,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
 #pragma unroll
         for (int e = 0; e < 4; ++e) G[r][e] = fmaf(G[r][e], kLog2e, G[r - 1][e]);
     *reinterpret_cast<float4*>(sTot + warp * kD + d0) = make_float4(G[kRPT - 1][0], G[kRPT - 1][1], G[kRPT - 1][2], G[kRPT - 1][3]);
-    if (t == kBulkThread) ptx::bulk_wait_read0();   // the previous tile's output staging has been read out
     ptx::cp_async_wait_all();             // beta
     __syncthreads();
     KDA_PHASE(hdr, 0);   // loads arrived + local scan
@@ -325,6 +329,9 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         ptx::umma_commit(mma_bar);
     }
     if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) timed_out = true;
+    // the previous tile's W/U staging (and this tile's Q', K' stores) have been read out by now; the
+    // staging area is written next (L, Aqk)
+    if (t == kBulkThread) ptx::bulk_wait_read0();
     __syncthreads();
     KDA_PHASE(hdr, 2);   // first MMA group
     ptx::tc_fence_after();
@@ -461,11 +468,12 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
                            ptx::umma_desc_sw128_mn(v0 + k * 2048, S_V_BLOCK), idesc, k > 0);
         ptx::umma_commit(mma_bar);
     }
-    if (!ptx::mbar_wait(mma_bar, 1, kWaitLimitNs)) timed_out = true;
-    if (nxt < ntiles) {   // every input buffer is free again: request the next tile
+    if (nxt < ntiles) {   // request the next tile: registers now, buffers once the MMAs are done with them
         locate(nxt, Ln, hn);
-        issue_prefetch(Ln, hn);
+        prefetch_regs(Ln, hn);
     }
+    if (!ptx::mbar_wait(mma_bar, 1, kWaitLimitNs)) timed_out = true;
+    if (nxt < ntiles) prefetch_bufs(Ln, hn);
     KDA_PHASE(hdr, 8);   // second MMA group
     ptx::tc_fence_after();
     {   // The A operand held every row twice, so TMEM lanes 0-63 and 64-127 both carry rows 0-63:
