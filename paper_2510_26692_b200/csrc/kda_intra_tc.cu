@@ -14,7 +14,7 @@
 //        L = Diag(beta) StrictTril(rows 0-63) (fp32, shared memory);  Aqk = Tril(rows 64-127)
 //   a3   T = (I + L)^-1 by blocked forward substitution: the four 16x16 diagonal blocks are
 //        inverted column by column in fp32 registers, then X = T_II L_IM for the six sub-diagonal
-//        blocks and three block levels  T_IJ = - sum_M X_IM T_MJ as warp-level 16x16 products
+//        blocks and  T_IJ = - sum_M X_IM T_MJ  in three dependency stages, as warp-level 16x16 products
 //        (mma.sync, tf32 inputs, fp32 accumulation; T is rounded to bf16 afterwards anyway)
 //   a4   Mm = T Diag(beta) (bf16);  second MMA group  [Mm ; Mm] (128 x 64) x [Kg | V] (64 x 256) -> TMEM
 //        (the rows are held twice so that all 128 TMEM lanes, i.e. all eight warps, share the read-out);
@@ -101,6 +101,15 @@ __device__ __forceinline__ void block16_mma(float (&acc)[2][4], const float* pa,
                 : "+f"(acc[nt][0]), "+f"(acc[nt][1]), "+f"(acc[nt][2]), "+f"(acc[nt][3])
                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
         }
+    }
+}
+__device__ __forceinline__ void block16_load(float (&acc)[2][4], const float* pc, int ld, int lane) {
+    const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+        const float2 lo = *reinterpret_cast<const float2*>(pc + g * ld + nt * 8 + 2 * t4);
+        const float2 hi = *reinterpret_cast<const float2*>(pc + (g + 8) * ld + nt * 8 + 2 * t4);
+        acc[nt][0] = lo.x; acc[nt][1] = lo.y; acc[nt][2] = hi.x; acc[nt][3] = hi.y;
     }
 }
 __device__ __forceinline__ void block16_store(float* pc, const float (&acc)[2][4], float sign, int ld,
@@ -409,17 +418,36 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     }
     __syncthreads();
     KDA_PHASE(hdr, 5);   // X
-#pragma unroll
-    for (int lvl = 1; lvl <= 3; ++lvl) {   // T_IJ = - sum_{M=J..I-1} X_IM T_MJ,  J = I - lvl
-        if (warp < 4 - lvl) {
-            const int I = lvl + warp, J = I - lvl;
-            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-            for (int M = J; M < I; ++M)
-                block16_mma(acc, sA + (I * 16) * LDT + M * 16, sT + (M * 16) * LDT + J * 16, LDT, lane);
-            block16_store(sT + (I * 16) * LDT + J * 16, acc, -1.f, LDT, lane);
-        }
-        __syncthreads();
+    // T_IJ = - sum_{M=J..I-1} X_IM T_MJ in three dependency stages; the terms of a sum that do not
+    // depend on blocks still being computed are taken early (kept, un-negated, in the block's place).
+    //   stage A: T10, T21, T32 final;  P20 = X20 T00,  P31 = X31 T11,  P30 = X30 T00
+    //   stage B: T20 = -(P20 + X21 T10),  T31 = -(P31 + X32 T21),  P30 += X31 T10
+    //   stage C: T30 = -(P30 + X32 T20)
+    auto blk = [&](float* base, int I, int J) { return base + (I * 16) * LDT + J * 16; };
+    if (warp < 6) {
+        const int I = warp < 3 ? warp + 1 : (warp == 3 ? 2 : 3);
+        const int J = warp < 3 ? warp : (warp == 4 ? 1 : 0);
+        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        block16_mma(acc, blk(sA, I, J), blk(sT, J, J), LDT, lane);
+        block16_store(blk(sT, I, J), acc, warp < 3 ? -1.f : 1.f, LDT, lane);
     }
+    __syncthreads();
+    if (warp < 3) {
+        // warp 0: T20 (M = 1), warp 1: T31 (M = 2), warp 2: P30 += X31 T10
+        const int I = warp == 0 ? 2 : 3, J = warp == 1 ? 1 : 0, M = warp == 1 ? 2 : 1;
+        float acc[2][4];
+        block16_load(acc, blk(sT, I, J), LDT, lane);
+        block16_mma(acc, blk(sA, I, M), blk(sT, M, J), LDT, lane);
+        block16_store(blk(sT, I, J), acc, warp < 2 ? -1.f : 1.f, LDT, lane);
+    }
+    __syncthreads();
+    if (warp == 0) {
+        float acc[2][4];
+        block16_load(acc, blk(sT, 3, 0), LDT, lane);
+        block16_mma(acc, blk(sA, 3, 2), blk(sT, 2, 0), LDT, lane);
+        block16_store(blk(sT, 3, 0), acc, -1.f, LDT, lane);
+    }
+    __syncthreads();
 
     KDA_PHASE(hdr, 6);   // block levels
     // ---- a4: Mm = T Diag(beta) as the A operand; [W | U] = Mm [Kg | V] ---------------------------------
