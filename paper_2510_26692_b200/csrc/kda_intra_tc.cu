@@ -407,31 +407,28 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     }
     __syncthreads();
     KDA_PHASE(hdr, 4);   // diagonal blocks
-    if (warp < 6) {   // X_IM = T_II L_IM for the six sub-diagonal blocks, one warp each, in place
-        const int I = warp < 1 ? 1 : (warp < 3 ? 2 : 3);
-        const int M = warp < 1 ? 0 : (warp < 3 ? warp - 1 : warp - 3);
-        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        float* Lim = sA + (I * 16) * LDT + M * 16;
-        block16_mma(acc, sT + (I * 16) * LDT + I * 16, Lim, LDT, lane);
-        __syncwarp();   // every lane has read its part of L_IM before anyone overwrites it
-        block16_store(Lim, acc, 1.f, LDT, lane);
-    }
-    __syncthreads();
-    KDA_PHASE(hdr, 5);   // X
+    // X_IM = T_II L_IM for the six sub-diagonal blocks (one warp each, in place), then
     // T_IJ = - sum_{M=J..I-1} X_IM T_MJ in three dependency stages; the terms of a sum that do not
     // depend on blocks still being computed are taken early (kept, un-negated, in the block's place).
     //   stage A: T10, T21, T32 final;  P20 = X20 T00,  P31 = X31 T11,  P30 = X30 T00
+    //            (each uses only the X block its own warp has just formed)
     //   stage B: T20 = -(P20 + X21 T10),  T31 = -(P31 + X32 T21),  P30 += X31 T10
     //   stage C: T30 = -(P30 + X32 T20)
     auto blk = [&](float* base, int I, int J) { return base + (I * 16) * LDT + J * 16; };
     if (warp < 6) {
-        const int I = warp < 3 ? warp + 1 : (warp == 3 ? 2 : 3);
-        const int J = warp < 3 ? warp : (warp == 4 ? 1 : 0);
+        const int I = warp < 1 ? 1 : (warp < 3 ? 2 : 3);
+        const int M = warp < 1 ? 0 : (warp < 3 ? warp - 1 : warp - 3);
         float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        block16_mma(acc, blk(sA, I, J), blk(sT, J, J), LDT, lane);
-        block16_store(blk(sT, I, J), acc, warp < 3 ? -1.f : 1.f, LDT, lane);
+        block16_mma(acc, blk(sT, I, I), blk(sA, I, M), LDT, lane);
+        __syncwarp();   // every lane has read its part of L_IM before anyone overwrites it
+        block16_store(blk(sA, I, M), acc, 1.f, LDT, lane);
+        __syncwarp();
+        float acc2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        block16_mma(acc2, blk(sA, I, M), blk(sT, M, M), LDT, lane);
+        block16_store(blk(sT, I, M), acc2, (I - M == 1) ? -1.f : 1.f, LDT, lane);
     }
     __syncthreads();
+    KDA_PHASE(hdr, 5);   // X + stage A
     if (warp < 3) {
         // warp 0: T20 (M = 1), warp 1: T31 (M = 2), warp 2: P30 += X31 T10
         const int I = warp == 0 ? 2 : 3, J = warp == 1 ? 1 : 0, M = warp == 1 ? 2 : 1;
