@@ -419,7 +419,30 @@ def main():
     dec_ms = max_over_ranks(e0.elapsed_time(e1)) / (args.decode_reps * DEC_STEPS)
     dec_bytes = DEC_SEQS * H * DEC_BYTES_PER_STATE
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
+    # multi-token decode (4 tokens per sequence and call): the state crosses HBM once per call
+    MT = 4
+    mq, mk, mv, mg, mb = (gd[n][:MT].transpose(0, 1).contiguous() for n in ("q", "k", "v", "log_alpha", "beta"))
+    mo = torch.empty((DEC_SEQS, MT, H, D), dtype=torch.bfloat16, device=dev)
+
+    def multi_block():
+        for _ in range(16):
+            K.kda_decode_multi(mq, mk, mv, mg, mb, S, None, mo, DEC_SEQS, MT, H, D, D, 1.0, dt, stream)
+
+    multi_block()
+    barrier()
+    e0.record(stream)
+    for _ in range(args.decode_reps):
+        multi_block()
+    e1.record(stream)
+    barrier()
+    mt_ms = max_over_ranks(e0.elapsed_time(e1)) / (args.decode_reps * 16)
+    mt_bytes = DEC_SEQS * H * (2 * D * D * 4 + MT * (4 * D * 2 + D * 4 + 4))
+    multi = {"tokens_per_call_and_sequence": MT, "ms_per_call": mt_ms,
+             "value": world * DEC_SEQS * MT / (mt_ms * 1e-3), "unit": "tokens/s",
+             "achieved_gbs": mt_bytes / (mt_ms * 1e-3) / 1e9,
+             "frac": mt_bytes / (mt_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     decode = {
+        "multi_token": multi,
         "metric": "KDA decode tokens/s (256 seqs x 32 heads, 64 in-place steps)",
         "value": world * DEC_SEQS / (dec_ms * 1e-3), "unit": "tokens/s", "ms_per_step": dec_ms,
         "roofline": {"bound": "hbm", "kernel": "kda_decode_kernel", "achieved": dec_gbs,

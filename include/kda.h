@@ -146,6 +146,22 @@ kda_status_t kda_decode_step(const void *q, const void *k, const void *v, const 
                              void *cuda_stream);
 
 /*
+ * Multi-token decode: Eq. 1 for n_tokens (1..64) consecutive tokens of every sequence in one call,
+ * e.g. the verification step of speculative decoding or a few tokens appended to a prefill
+ * (Section 6.3: generation uses the recurrent kernel; the paper's serving integration is the use
+ * case).  The state is read and written once per call, not once per token.
+ *
+ *   q, k, log_alpha  [n_seqs, n_tokens, H, dk]   v, o  [n_seqs, n_tokens, H, dv]
+ *   beta             [n_seqs, n_tokens, H]
+ *   S, state_slot    as in kda_decode_step
+ * Equivalent to n_tokens calls of kda_decode_step on the tokens in order.
+ */
+kda_status_t kda_decode_multi(const void *q, const void *k, const void *v, const float *log_alpha,
+                              const float *beta, float *S, const int32_t *state_slot, void *o,
+                              int n_seqs, int n_tokens, int H, int dk, int dv, float scale,
+                              kda_dtype_t dt, void *cuda_stream);
+
+/*
  * Host-buffer variants: same operations with q, k, v, log_alpha, beta, S0 (chunk) and o, S_T read
  * from / written to HOST memory (pinned memory makes the copies asynchronous).  The device copies
  * live in the caller's device workspace, so these allocate nothing either.  cu_seqlens is given on

@@ -59,6 +59,8 @@ def load():
                                          i32, i32, f32, i32, vp]
     lib.kda_decode_step.restype = i32
     lib.kda_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp]
+    lib.kda_decode_multi.restype = i32
+    lib.kda_decode_multi.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, i32, vp]
     lib.kda_chunk_fwd_host_workspace_bytes.restype = sz
     lib.kda_chunk_fwd_host_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32, i32]
     lib.kda_chunk_fwd_host.restype = i32
@@ -203,6 +205,20 @@ def kda_decode_step(q, k, v, log_alpha, beta, S, state_slot, o, n_seqs, H, dk, d
         _ptr(S, True, f32, "S"), _ptr(state_slot, True, torch.int32, "state_slot"),
         _ptr(o, True, et, "o"), int(n_seqs), int(H), int(dk), int(dv), float(scale), int(dt),
         _stream(stream))
+    _check(rc)
+
+
+def kda_decode_multi(q, k, v, log_alpha, beta, S, state_slot, o, n_seqs, n_tokens, H, dk, dv, scale,
+                     dt, stream=None):
+    """``kda_decode_multi`` of ``include/kda.h``: ``n_tokens`` tokens per sequence, ``S`` in place."""
+    f32 = torch.float32
+    et = torch.bfloat16 if dt == KDA_BF16 else torch.float32
+    rc = load().kda_decode_multi(
+        _ptr(q, True, et, "q"), _ptr(k, True, et, "k"), _ptr(v, True, et, "v"),
+        _ptr(log_alpha, True, f32, "log_alpha"), _ptr(beta, True, f32, "beta"),
+        _ptr(S, True, f32, "S"), _ptr(state_slot, True, torch.int32, "state_slot"),
+        _ptr(o, True, et, "o"), int(n_seqs), int(n_tokens), int(H), int(dk), int(dv), float(scale),
+        int(dt), _stream(stream))
     _check(rc)
 
 

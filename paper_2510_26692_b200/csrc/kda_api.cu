@@ -254,6 +254,28 @@ kda_status_t kda_decode_step(const void* q, const void* k, const void* v, const 
                          static_cast<cudaStream_t>(cuda_stream));
 }
 
+kda_status_t kda_decode_multi(const void* q, const void* k, const void* v, const float* log_alpha,
+                              const float* beta, float* S, const int32_t* state_slot, void* o,
+                              int n_seqs, int n_tokens, int H, int dk, int dv, float scale,
+                              kda_dtype_t dt, void* cuda_stream)
+{
+    if (dk != kD || dv != kD || (dt != KDA_F32 && dt != KDA_BF16))
+        return fail(KDA_ERR_UNSUPPORTED, "kda_decode_multi: only dk=dv=128, dt in {f32,bf16} are "
+                    "supported (got dk=%d dv=%d dt=%d)", dk, dv, (int)dt);
+    if (n_seqs < 0 || H <= 0 || n_tokens < 0 || n_tokens > 64 || (int64_t)n_seqs * H > 0x7fffffff)
+        return fail(KDA_ERR_INVALID_ARG, "kda_decode_multi: bad sizes n_seqs=%d n_tokens=%d H=%d "
+                    "(n_tokens must be 0..64)", n_seqs, n_tokens, H);
+    if (n_seqs == 0 || n_tokens == 0) return KDA_OK;
+    if (!q || !k || !v || !log_alpha || !beta || !S || !o)
+        return fail(KDA_ERR_INVALID_ARG, "kda_decode_multi: NULL pointer argument");
+    const void* ptrs[] = {q, k, v, log_alpha, beta, S, o, state_slot};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return fail(KDA_ERR_INVALID_ARG, "kda_decode_multi: pointer %p is not "
+                                       "16-byte aligned", p);
+    return launch_decode_multi(q, k, v, log_alpha, beta, S, state_slot, o, n_seqs, n_tokens, H, scale, dt,
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+
 // ---- host-buffer variants -------------------------------------------------------------------------
 
 namespace {

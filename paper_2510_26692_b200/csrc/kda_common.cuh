@@ -167,6 +167,10 @@ kda_status_t launch_decode(const void* q, const void* k, const void* v, const fl
                            const float* beta, float* S, const int32_t* slot, void* o, int n_seqs,
                            int H, float scale, kda_dtype_t dt, cudaStream_t st);
 
+kda_status_t launch_decode_multi(const void* q, const void* k, const void* v, const float* log_alpha,
+                                 const float* beta, float* S, const int32_t* slot, void* o, int n_seqs,
+                                 int n_tok, int H, float scale, kda_dtype_t dt, cudaStream_t st);
+
 // fp32 FMA path (also accepts bf16 storage): per-tile scratch size and pass launcher
 size_t simt_tile_bytes();
 kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, int n_begin,

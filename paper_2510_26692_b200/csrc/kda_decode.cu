@@ -103,6 +103,104 @@ kda_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
     }
 }
 
+// Multi-token decode: the same recurrence for T consecutive tokens of each sequence (speculative
+// decoding, continuation of a chunked prefill by a few tokens) with the state held in registers
+// across the tokens: it crosses HBM once in each direction per call instead of once per token.
+// Layout: q, k, log_alpha [n_seqs, T, H, 128], v, o [n_seqs, T, H, 128], beta [n_seqs, T, H].
+template <typename T>
+__global__ void __launch_bounds__(256, 2)
+kda_decode_multi_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                        const float* __restrict__ log_alpha, const float* __restrict__ beta, float* S,
+                        const int32_t* __restrict__ slot, T* __restrict__ o, int H, int n_tok, float scale)
+{
+    __shared__ float s_a[2][kD], s_k[2][kD], s_q[2][kD];
+    __shared__ float4 s_red[2][2][8][32];
+    const int item = blockIdx.x;
+    const int n = item / H, h = item - n * H;
+    const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
+    const size_t sl = slot ? (size_t)slot[n] : (size_t)n;
+    float* Sp = S + (sl * H + h) * (size_t)(kD * kD) + lane * 4;
+
+    float4 x[16];
+#pragma unroll
+    for (int m = 0; m < 16; ++m) x[m] = ld_stream(Sp + (size_t)(warp + 8 * m) * kD);
+
+    auto vec_of = [&](int tt) { return ((size_t)(n * n_tok + tt) * H + h) * kD; };
+    // the per-token vectors are fetched one token ahead (threads 0-127: one channel each)
+    float pa = 0.f, pk = 0.f, pq = 0.f;
+    if (t < kD) {
+        const size_t vec = vec_of(0);
+        pa = log_alpha[vec + t];
+        pk = to_f<T>(k[vec + t]);
+        pq = to_f<T>(q[vec + t]);
+    }
+    float bt_next = beta[(size_t)(n * n_tok) * H + h];
+    float4 vv_next = IO<T>::load4(v + vec_of(0) + lane * 4);
+    for (int tt = 0; tt < n_tok; ++tt) {
+        const int b = tt & 1;
+        if (t < kD) {
+            s_a[b][t] = expf(pa);
+            s_k[b][t] = pk;
+            s_q[b][t] = pq;
+            if (tt + 1 < n_tok) {
+                const size_t vec = vec_of(tt + 1);
+                pa = log_alpha[vec + t];
+                pk = to_f<T>(k[vec + t]);
+                pq = to_f<T>(q[vec + t]);
+            }
+        }
+        const size_t vec = vec_of(tt);
+        const float bt = bt_next;
+        const float4 vv = vv_next;
+        if (tt + 1 < n_tok) {
+            bt_next = beta[(size_t)(n * n_tok + tt + 1) * H + h];
+            vv_next = IO<T>::load4(v + vec_of(tt + 1) + lane * 4);
+        }
+        __syncthreads();
+
+        float qk = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) qk += s_q[b][lane * 4 + i] * s_k[b][lane * 4 + i];
+#pragma unroll
+        for (int ofs = 16; ofs > 0; ofs >>= 1) qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
+
+        float4 p = make_float4(0.f, 0.f, 0.f, 0.f), s = p;
+#pragma unroll
+        for (int m = 0; m < 16; ++m) {
+            const int row = warp + 8 * m;
+            const float a = s_a[b][row], kk = s_k[b][row], qq = s_q[b][row];
+            x[m].x *= a; x[m].y *= a; x[m].z *= a; x[m].w *= a;
+            p.x += kk * x[m].x; p.y += kk * x[m].y; p.z += kk * x[m].z; p.w += kk * x[m].w;
+            s.x += qq * x[m].x; s.y += qq * x[m].y; s.z += qq * x[m].z; s.w += qq * x[m].w;
+        }
+        s_red[b][0][warp][lane] = p;
+        s_red[b][1][warp][lane] = s;
+        __syncthreads();
+        p = s_red[b][0][0][lane];
+        s = s_red[b][1][0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) {   // fixed order: bitwise reproducible
+            float4 a4 = s_red[b][0][w][lane], b4 = s_red[b][1][w][lane];
+            p.x += a4.x; p.y += a4.y; p.z += a4.z; p.w += a4.w;
+            s.x += b4.x; s.y += b4.y; s.z += b4.z; s.w += b4.w;
+        }
+        const float4 r = make_float4(vv.x - p.x, vv.y - p.y, vv.z - p.z, vv.w - p.w);
+        if (warp == 0) {
+            const float c = bt * qk;
+            IO<T>::store4(o + vec + lane * 4,
+                          make_float4(scale * (s.x + c * r.x), scale * (s.y + c * r.y),
+                                      scale * (s.z + c * r.z), scale * (s.w + c * r.w)));
+        }
+#pragma unroll
+        for (int m = 0; m < 16; ++m) {
+            const float c = bt * s_k[b][warp + 8 * m];
+            x[m].x += c * r.x; x[m].y += c * r.y; x[m].z += c * r.z; x[m].w += c * r.w;
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < 16; ++m) st_stream(Sp + (size_t)(warp + 8 * m) * kD, x[m]);
+}
+
 }  // namespace
 
 kda_status_t launch_decode(const void* q, const void* k, const void* v, const float* log_alpha,
@@ -120,6 +218,27 @@ kda_status_t launch_decode(const void* q, const void* k, const void* v, const fl
         kda_decode_kernel<float><<<grid, 256, 0, st>>>((const float*)q, (const float*)k,
                                                        (const float*)v, log_alpha, beta, S, slot,
                                                        (float*)o, H, scale);
+    }
+    count_launch();
+    KDA_CUDA_TRY(cudaGetLastError());
+    return KDA_OK;
+}
+
+kda_status_t launch_decode_multi(const void* q, const void* k, const void* v, const float* log_alpha,
+                                 const float* beta, float* S, const int32_t* slot, void* o, int n_seqs,
+                                 int n_tok, int H, float scale, kda_dtype_t dt, cudaStream_t st)
+{
+    if (n_seqs == 0 || n_tok == 0) return KDA_OK;
+    const unsigned grid = (unsigned)((size_t)n_seqs * H);
+    ProfScope ps(PROF_DECODE, st);
+    if (dt == KDA_BF16) {
+        using T = __nv_bfloat16;
+        kda_decode_multi_kernel<T><<<grid, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v, log_alpha,
+                                                         beta, S, slot, (T*)o, H, n_tok, scale);
+    } else {
+        kda_decode_multi_kernel<float><<<grid, 256, 0, st>>>((const float*)q, (const float*)k,
+                                                             (const float*)v, log_alpha, beta, S, slot,
+                                                             (float*)o, H, n_tok, scale);
     }
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());

@@ -309,3 +309,42 @@ def test_bounded_wait_reports_timeout(oracle_mod):
     K.kda_check_status(ws)    # the word was cleared by the failed check
     d = inputs.chunk_inputs([130], H=2, dtype=torch.bfloat16, seed=35, s0_std=0.02)
     check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
+
+
+@pytest.mark.parametrize("dtype,n_tok", [(torch.bfloat16, 4), (torch.float32, 7), (torch.bfloat16, 16)])
+def test_decode_multi_token(oracle_mod, dtype, n_tok):
+    """n_tok tokens per sequence in one call: equals the recurrence over those tokens from the
+    slot's state (oracle), and equals n_tok single-token decode calls bit for bit."""
+    N, H = 6, 3
+    d = inputs.decode_inputs(N, H, n_tok, dtype=dtype, seed=36)       # [n_tok, N, H, .]
+    dev = "cuda:0"
+    perm = lambda t: t.transpose(0, 1).contiguous()                    # -> [N, n_tok, H, .]
+    q, k, v, la, be = (perm(d[x]) for x in ("q", "k", "v", "log_alpha", "beta"))
+    slots = torch.tensor([4, 0, 7, 2, 6, 1], dtype=torch.int32)
+    S0 = torch.randn((8, H, 128, 128), generator=torch.Generator().manual_seed(6)) * 0.05
+    dt = K.KDA_BF16 if dtype == torch.bfloat16 else K.KDA_F32
+    S = S0.to(dev)
+    o = torch.empty((N, n_tok, H, 128), dtype=dtype, device=dev)
+    K.kda_decode_multi(q.to(dev), k.to(dev), v.to(dev), la.to(dev), be.to(dev), S, slots.to(dev), o,
+                       N, n_tok, H, 128, 128, 0.7, dt)
+    # single-token calls
+    S1 = S0.to(dev)
+    o1 = torch.empty_like(o)
+    for t in range(n_tok):
+        ot = torch.empty((N, H, 128), dtype=dtype, device=dev)
+        K.kda_decode_step(d["q"][t].to(dev), d["k"][t].to(dev), d["v"][t].to(dev),
+                          d["log_alpha"][t].to(dev), d["beta"][t].to(dev), S1, slots.to(dev), ot,
+                          N, H, 128, 128, 0.7, dt)
+        o1[:, t] = ot
+    torch.cuda.synchronize()
+    assert torch.equal(o, o1) and torch.equal(S, S1)
+    # oracle: each sequence is n_tok tokens starting from its slot's state
+    flat = lambda t: to_np32(t.reshape((N * n_tok,) + tuple(t.shape[2:])))
+    cu = np.arange(N + 1, dtype=np.int64) * n_tok
+    o_ref, S_ref = oracle_mod.recurrence(flat(q), flat(k), flat(v), flat(la), flat(be),
+                                         S0=S0[slots.long()].double().numpy(), cu_seqlens=cu, scale=0.7)
+    tol = TOL[dt] if dtype == torch.bfloat16 else 1e-5
+    assert rel_l2(to_np32(o).reshape(o_ref.shape), o_ref) <= tol
+    assert rel_l2(to_np32(S[slots.long()]), S_ref) <= 1e-5
+    untouched = [3, 5]
+    assert torch.equal(S[untouched].cpu(), S0[untouched])
