@@ -115,15 +115,10 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, float* __r
         *reinterpret_cast<float4*>(sKi + i * LD + c) = make_float4(oki[0], oki[1], oki[2], oki[3]);
         *reinterpret_cast<float4*>(sQg + i * LD + c) = make_float4(oqg[0], oqg[1], oqg[2], oqg[3]);
         *reinterpret_cast<float4*>(sKG + i * LD + c) = make_float4(oKG[0], oKG[1], oKG[2], oKG[3]);
-        {
-            *reinterpret_cast<float4*>(tile + T_QG + i * kD + c) =
-                make_float4(oQG[0], oQG[1], oQG[2], oQG[3]);
-            *reinterpret_cast<float4*>(tile + T_KT + i * kD + c) =
-                make_float4(oKT[0], oKT[1], oKT[2], oKT[3]);
-            if (i == 0)
-                *reinterpret_cast<float4*>(tile + T_GC + c) =
-                    make_float4(ogc[0], ogc[1], ogc[2], ogc[3]);
-        }
+        *reinterpret_cast<float4*>(tile + T_QG + i * kD + c) = make_float4(oQG[0], oQG[1], oQG[2], oQG[3]);
+        *reinterpret_cast<float4*>(tile + T_KT + i * kD + c) = make_float4(oKT[0], oKT[1], oKT[2], oKT[3]);
+        if (i == 0)
+            *reinterpret_cast<float4*>(tile + T_GC + c) = make_float4(ogc[0], ogc[1], ogc[2], ogc[3]);
     }
     __syncthreads();
 
@@ -190,10 +185,8 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, float* __r
 #pragma unroll
         for (int m = 0; m < 8; ++m) {
             const int c = cq * 4 + 16 * m;
-            {
-                *reinterpret_cast<float4*>(tile + T_W + i * kD + c) = w[m];
-                *reinterpret_cast<float4*>(tile + T_U + i * kD + c) = u[m];
-            }
+            *reinterpret_cast<float4*>(tile + T_W + i * kD + c) = w[m];
+            *reinterpret_cast<float4*>(tile + T_U + i * kD + c) = u[m];
         }
     }
 }

@@ -104,17 +104,6 @@ template <> struct IO<__nv_bfloat16> {
             kda_phase_last_ = now_;                                           \
         }                                                                     \
     } while (0)
-#define KDA_PHASE_ANY(slot)                                                   \
-    do {                                                                      \
-        const long long now_ = clock64();                                     \
-        kda_phase_acc_[slot] += (int)(now_ - kda_phase_last_);                \
-        kda_phase_last_ = now_;                                               \
-    } while (0)
-#define KDA_PHASE_FLUSH_ANY(hdr)                                              \
-    do {                                                                      \
-        _Pragma("unroll") for (int s_ = 0; s_ < 24; ++s_)                     \
-            if (kda_phase_acc_[s_]) atomicAdd(&(hdr)->pad[s_ + 24], kda_phase_acc_[s_] >> 4); \
-    } while (0)
 #define KDA_PHASE_FLUSH(hdr)                                                  \
     do {                                                                      \
         if (threadIdx.x == 0) {                                               \
@@ -126,8 +115,6 @@ template <> struct IO<__nv_bfloat16> {
 #define KDA_PHASE_DECL do {} while (0)
 #define KDA_PHASE(hdr, slot) do {} while (0)
 #define KDA_PHASE_FLUSH(hdr) do {} while (0)
-#define KDA_PHASE_ANY(slot) do {} while (0)
-#define KDA_PHASE_FLUSH_ANY(hdr) do {} while (0)
 #endif
 
 // Locate global chunk g: sequence index, first token, number of valid tokens (1..64).
