@@ -37,7 +37,7 @@ constexpr uint64_t kWaitLimitNs = 1000000000ull;   // 1 s per wait
 constexpr int kNCtrl = 2;                          // MMA-issuing threads (one per control warp): 2 or 4
 
 template <int NS> struct InterCfg {
-    static_assert(NS == 32, "one 32-column accumulator block per matrix");
+    static_assert(NS == 32 || NS == 64, "state columns per CTA: one or two 32-column blocks");
     static constexpr int kStages = 3;
     static constexpr uint32_t kQW = 0;                      // [2 K-halves][128][64]: rows 0-63 W, 64-127 Gamma.Q
     static constexpr uint32_t kKT = 32768;                  // K': [2 dk-halves][64 tokens][64], MN-major A operand
@@ -45,7 +45,7 @@ template <int NS> struct InterCfg {
     static constexpr uint32_t kGC = 57344;                  // gamma^C | exp(G_m) | exp(G_C - G_m), 128 fp32 each
     static constexpr uint32_t kMainBytes = tc::OFF_U;       // the images and the three vectors are contiguous in a tile
     static constexpr uint32_t kU = tc::OFF_U;               // [64 tokens][NS] block of U
-    static constexpr uint32_t kUBytes = tc::U_BLOCK;
+    static constexpr uint32_t kUBytes = (NS / 32) * tc::U_BLOCK;
     static constexpr uint32_t kStage = (kU + kUBytes + 1023) / 1024 * 1024;
     static constexpr uint32_t kSbf = kStages * kStage;      // B operand of MMA1, MN-major: [128 dk rows][128 B]
     static constexpr uint32_t kVn = kSbf + 128 * 128;       // B operand of MMA2, MN-major: [64 token rows][128 B]
@@ -53,23 +53,28 @@ template <int NS> struct InterCfg {
     static constexpr uint32_t kTotal = kBars + 128;
     static constexpr uint32_t kSmem = kTotal + 1024;        // slack for manual 1024-byte alignment
     static constexpr uint32_t kTxBytes = kMainBytes + kUBytes;
-    static constexpr uint32_t kTmemCols = kNCtrl == 2 ? 256 : 512;   // 2 kNCtrl x D1 + kNCtrl x D3, NS columns each
+    static constexpr uint32_t kTmemCols = 3 * kNCtrl * NS <= 256 ? 256 : 512;   // 2 kNCtrl x D1 + kNCtrl x D3, NS columns each
+    static_assert(3 * kNCtrl * NS <= 512 && kSmem <= 232448, "fits TMEM and the shared memory of one SM");
 };
 
 // sum of the kNCtrl partial accumulators (NS columns each, side by side in TMEM) of one matrix
-__device__ __forceinline__ void tmem_ld_sum(uint32_t taddr, float (&acc)[32]) {
-    uint32_t r[32], r2[32];
-    ptx::tmem_ld_32x32b_x32(taddr, r);
-    ptx::tmem_ld_32x32b_x32(taddr + 32, r2);
-    ptx::tmem_ld_wait();
+template <int NS>
+__device__ __forceinline__ void tmem_ld_sum(uint32_t taddr, float (&acc)[NS]) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(r[j]) + __uint_as_float(r2[j]);
-    if (kNCtrl == 4) {
-        ptx::tmem_ld_32x32b_x32(taddr + 64, r);
-        ptx::tmem_ld_32x32b_x32(taddr + 96, r2);
+    for (int blk = 0; blk < NS / 32; ++blk) {
+        uint32_t r[32], r2[32];
+        ptx::tmem_ld_32x32b_x32(taddr + blk * 32, r);
+        ptx::tmem_ld_32x32b_x32(taddr + NS + blk * 32, r2);
         ptx::tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc[j] += __uint_as_float(r[j]) + __uint_as_float(r2[j]);
+        for (int j = 0; j < 32; ++j) acc[blk * 32 + j] = __uint_as_float(r[j]) + __uint_as_float(r2[j]);
+        if (kNCtrl == 4) {
+            ptx::tmem_ld_32x32b_x32(taddr + 2 * NS + blk * 32, r);
+            ptx::tmem_ld_32x32b_x32(taddr + 3 * NS + blk * 32, r2);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc[blk * 32 + j] += __uint_as_float(r[j]) + __uint_as_float(r2[j]);
+        }
     }
 }
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
@@ -77,11 +82,12 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&p);
 }
 
-// Writes 32 fp32 values as one 64-byte bf16 row (four 16-byte chunks) of an MN-major operand image
-// with 128-byte rows and 128-byte swizzle.
-__device__ __forceinline__ void store_row32(uint8_t* img, int row, const float (&x)[32]) {
+// Writes NS fp32 values as one bf16 row (NS / 8 16-byte chunks) of an MN-major operand image with
+// 128-byte rows and 128-byte swizzle.
+template <int NS>
+__device__ __forceinline__ void store_row(uint8_t* img, int row, const float (&x)[NS]) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
+    for (int c = 0; c < NS / 8; ++c)
         *reinterpret_cast<uint4*>(img + row * 128 + ((c ^ (row & 7)) << 4)) =
             make_uint4(pack2(x[8 * c], x[8 * c + 1]), pack2(x[8 * c + 2], x[8 * c + 3]),
                        pack2(x[8 * c + 4], x[8 * c + 5]), pack2(x[8 * c + 6], x[8 * c + 7]));
@@ -265,7 +271,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             float z[NS];
 #pragma unroll
             for (int j = 0; j < NS; ++j) z[j] = cgn * S[j];
-            store_row32(sbf, tid, z);
+            store_row<NS>(sbf, tid, z);
         };
         store_scaled(ref_scale_of(0));
         ptx::fence_async_smem();
@@ -279,19 +285,19 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             const uint32_t par = (uint32_t)it & 1u;
             wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);   // U and gamma^C are read with plain loads
             if (warp < 2) {   // a6: V_new = U - W S  (token row = tid)
-                uint4 uq[4];   // this token's 32 values of U
+                uint4 uq[NS / 8];   // this token's NS values of U
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    uq[c] = *reinterpret_cast<const uint4*>(sb + Cfg::kU + tc::u_off(tid, c));
+                for (int c = 0; c < NS / 8; ++c)
+                    uq[c] = *reinterpret_cast<const uint4*>(sb + Cfg::kU + (c >> 2) * tc::U_BLOCK + tc::u_off(tid, c & 3));
                 const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
                 wait(mma1_bar, par, 2);
                 KDA_PHASE(hdr, 18);  // MMA1
                 ptx::tc_fence_after();
-                float x[32];
-                tmem_ld_sum(tmem_lane + d1, x);
+                float x[NS];
+                tmem_ld_sum<NS>(tmem_lane + d1, x);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) x[j] = __bfloat162float(U[j]) - x[j];
-                store_row32(vn, tid, x);
+                for (int j = 0; j < NS; ++j) x[j] = __bfloat162float(U[j]) - x[j];
+                store_row<NS>(vn, tid, x);
                 ptx::fence_async_smem();
                 ptx::tc_fence_before();
                 ptx::mbar_arrive(vn_ready);
@@ -313,17 +319,17 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             KDA_PHASE(hdr, 20);  // MMA2
             ptx::tc_fence_after();
             {   // a8: S <- gamma^C . S + exp(G_C - G_m) . (K'^T V_new) ; refresh the bf16 operand copy
-                float ds[32];
-                tmem_ld_sum(tmem_lane + d3, ds);
+                float ds[NS];
+                tmem_ld_sum<NS>(tmem_lane + d3, ds);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) zpre[j] = fmaf(zb, ds[j], zpre[j]);
-                store_row32(sbf, tid, zpre);
+                for (int j = 0; j < NS; ++j) zpre[j] = fmaf(zb, ds[j], zpre[j]);
+                store_row<NS>(sbf, tid, zpre);
                 ptx::fence_async_smem();
                 ptx::tc_fence_before();
                 ptx::mbar_arrive(sbf_ready);
                 // the fp32 master copy itself is not on the chain
 #pragma unroll
-                for (int j = 0; j < 32; ++j) S[j] = fmaf(ct, ds[j], gc * S[j]);
+                for (int j = 0; j < NS; ++j) S[j] = fmaf(ct, ds[j], gc * S[j]);
             }
             KDA_PHASE(hdr, 21);  // state update
             if (warp >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64)
@@ -333,21 +339,14 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 __nv_bfloat16* orow = op + ((tok0 + i) * a.H + h) * kD + col0;
                 wait(&out_bar[it & 1], (uint32_t)(it >> 1) & 1u, 6);
                 ptx::tc_fence_after();
-                uint32_t r[32];
-                {
-                    float ov[32];
-                    tmem_ld_sum(tmem_lane + d1, ov);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(ov[j]);
-                }
+                float ov[NS];
+                tmem_ld_sum<NS>(tmem_lane + d1, ov);
                 if (i < len) {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 8)
+                    for (int j = 0; j < NS; j += 8)
                         *reinterpret_cast<uint4*>(orow + j) =
-                            make_uint4(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])),
-                                       pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])),
-                                       pack2(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])),
-                                       pack2(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
+                            make_uint4(pack2(ov[j], ov[j + 1]), pack2(ov[j + 2], ov[j + 3]),
+                                       pack2(ov[j + 4], ov[j + 5]), pack2(ov[j + 6], ov[j + 7]));
                 }
                 ptx::tc_fence_before();
             }
@@ -427,6 +426,17 @@ kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n
     kda_status_t rc = launch_intra_tc(a, tiles, hdr, clear_status, st);
     if (rc != KDA_OK) return rc;
     if (n_count <= 0) return KDA_OK;
+    // 32 state columns per CTA give the most CTAs (the chains are latency-bound); once there are
+    // more chains than the GPU can hold at one CTA per SM, 64 columns per CTA do twice the work per
+    // MMA issue and halve the operand traffic from L2.
+    static int n_sm = 0;
+    if (n_sm == 0) {
+        int dev = 0;
+        KDA_CUDA_TRY(cudaGetDevice(&dev));
+        KDA_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    }
+    if ((int64_t)n_count * a.H * 4 > 2 * (int64_t)n_sm)
+        return launch_inter_tc_t<64>(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);
     return launch_inter_tc_t<32>(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);
 }
 
