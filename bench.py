@@ -37,8 +37,8 @@ STATE_BYTES = 2 * D * D * 4
 DEC_BYTES_PER_STATE = 2 * D * D * 4 + 4 * D * 2 + D * 4 + 4
 FLOPS_PER_TOKEN_HEAD = 6 * D * D + 3 * CHUNK * D + CHUNK * CHUNK   # the paper's FLOPs model
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (prefill: intra 168.4 + 97.7 MB, inter 154.2 + 20.3 MB; decode: 547.4 + 484.7 MB)
-PREFILL_DRAM_TRAFFIC = {"intra_chunk": 266.1e6, "inter_chunk": 174.4e6}
+# profiles/ (prefill: intra 168.4 + 99.7 MB, inter 156.3 + 20.1 MB; decode: 547.4 + 484.7 MB)
+PREFILL_DRAM_TRAFFIC = {"intra_chunk": 268.1e6, "inter_chunk": 176.4e6}
 DECODE_DRAM_TRAFFIC = 1032.1e6
 
 
