@@ -348,3 +348,20 @@ def test_decode_multi_token(oracle_mod, dtype, n_tok):
     assert rel_l2(to_np32(S[slots.long()]), S_ref) <= 1e-5
     untouched = [3, 5]
     assert torch.equal(S[untouched].cpu(), S0[untouched])
+
+
+@pytest.mark.parametrize("seed", [101, 102, 103, 104])
+def test_random_packed_batches(oracle_mod, seed):
+    """Randomly drawn packed batches (number of sequences, lengths incl. 0 and non-multiples of the
+    chunk, head count, dtype, with and without S0): every sequence's o and S_T against the oracle."""
+    g = torch.Generator().manual_seed(seed)
+    n = int(torch.randint(1, 7, (1,), generator=g))
+    lens = [int(x) for x in torch.randint(0, 400, (n,), generator=g)]
+    if sum(lens) == 0:
+        lens[0] = 65
+    H = int(torch.randint(1, 6, (1,), generator=g))
+    bf16 = bool(torch.randint(0, 2, (1,), generator=g))
+    d = inputs.chunk_inputs(lens, H=H, dtype=torch.bfloat16 if bf16 else torch.float32, seed=seed,
+                            s0_std=0.02 if seed % 2 else 0.0, gate_mean=float(torch.randint(0, 6, (1,), generator=g)))
+    d["force_varlen"] = True
+    check_chunk(oracle_mod, d, TOL[K.KDA_BF16 if bf16 else K.KDA_F32])
