@@ -113,8 +113,8 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     // out_bar is waited on by warps that the rest of the pipeline could, in principle, overtake by a
     // whole chunk; two barriers used alternately keep a parity wait from ever being lapped
     uint64_t* out_bar = mma2_bar + 1;      // [2] the output accumulator of a chunk is complete
-    uint64_t* sbf_ready = out_bar + 2;     // 128 arrivals: bf16 state copy written (and stage reads done)
-    uint64_t* vn_ready = sbf_ready + 1;    // 64 arrivals: V_new written
+    uint64_t* sbf_ready = out_bar + 2;     // 4 warp arrivals: bf16 state copy written (and stage reads done)
+    uint64_t* vn_ready = sbf_ready + 1;    // 2 warp arrivals: V_new written
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(vn_ready + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     uint8_t* sbf = smem + Cfg::kSbf;
@@ -146,8 +146,8 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         ptx::mbar_init(mma2_bar, kNCtrl);
         ptx::mbar_init(&out_bar[0], 1);
         ptx::mbar_init(&out_bar[1], 1);
-        ptx::mbar_init(sbf_ready, 128);
-        ptx::mbar_init(vn_ready, 64);
+        ptx::mbar_init(sbf_ready, 4);    // one arrival per compute warp (after a warp-level sync)
+        ptx::mbar_init(vn_ready, 2);
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -251,6 +251,12 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     } else {
         // ================= compute warps =================
         const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+        // one barrier arrival per warp: every lane has fenced its own writes, the warp-level sync
+        // orders them before lane 0's (releasing) arrive -- 32x fewer serialised arrivals per hop
+        auto warp_arrive = [&](uint64_t* bar) {
+            __syncwarp();
+            if ((tid & 31) == 0) ptx::mbar_arrive(bar);
+        };
         // state: fp32 master in registers (thread = dk row), bf16 copy as the B operand of MMA1
         float S[NS];
         const size_t sbase = ((size_t)n * a.H + h) * (size_t)(kD * kD) + (size_t)tid * kD + col0;
@@ -275,7 +281,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         };
         store_scaled(ref_scale_of(0));
         ptx::fence_async_smem();
-        ptx::mbar_arrive(sbf_ready);
+        warp_arrive(sbf_ready);
         KDA_PHASE(hdr, 16);  // set-up
 
         for (int it = 0; it < nchunks; ++it) {
@@ -300,7 +306,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 store_row<NS>(vn, tid, x);
                 ptx::fence_async_smem();
                 ptx::tc_fence_before();
-                ptx::mbar_arrive(vn_ready);
+                warp_arrive(vn_ready);
                 KDA_PHASE(hdr, 19);  // V_new
             }
             const float gc = reinterpret_cast<const float*>(sb + Cfg::kGC)[tid];          // gamma^C
@@ -326,7 +332,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 store_row<NS>(sbf, tid, zpre);
                 ptx::fence_async_smem();
                 ptx::tc_fence_before();
-                ptx::mbar_arrive(sbf_ready);
+                warp_arrive(sbf_ready);
                 // the fp32 master copy itself is not on the chain
 #pragma unroll
                 for (int j = 0; j < NS; ++j) S[j] = fmaf(ct, ds[j], gc * S[j]);
