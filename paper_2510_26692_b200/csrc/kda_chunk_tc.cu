@@ -228,7 +228,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                                    k > 0);
                 }
                 ptx::umma_commit(mma2_bar);
-                if (half == 0) {
+                if (half == 0 && op) {
                     // D1[64:128] += Aqk V_new.  The 128-row A operand starts 64 rows before Aqk: those
                     // rows (the tail of the Kt image) only touch accumulator rows 0-63, which are dead
                     // once V_new has been taken.
@@ -240,7 +240,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 }
             }
             if (half == 0) {
-                if (nchunks > 0) wait(&out_bar[(nchunks - 1) & 1], (uint32_t)((nchunks - 1) >> 1) & 1u, 7);   // last output product done
+                if (nchunks > 0 && op) wait(&out_bar[(nchunks - 1) & 1], (uint32_t)((nchunks - 1) >> 1) & 1u, 7);   // last output product done
                 if (*abort_flag) {
                     // drain the bulk copies still in flight before the shared memory goes away
                     for (int j = (loads_issued > NSTG ? loads_issued - NSTG : 0); j < loads_issued; ++j)

@@ -25,6 +25,8 @@
 // beta = 0, k = q = v = 0).
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "kda_common.cuh"
 #include "kda_ptx.cuh"
 #include "kda_tiles.cuh"
@@ -132,11 +134,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&p);
 }
+// kHasQ = false: state-only call (no output requested): the query half of the work is compiled out.
+template <bool kHasQ>
 __global__ void __launch_bounds__(kNT, 2)
 kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
              const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
-             const __grid_constant__ CUtensorMap tm_v, int has_q, int clear_status)
+             const __grid_constant__ CUtensorMap tm_v, int clear_status)
 {
+    constexpr bool has_q = kHasQ;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -198,12 +203,13 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     // k, q, v, beta -> shared memory (only once the second MMA group has finished reading Kg and V)
     auto prefetch_bufs = [&](const ChunkLoc& Lo, int ho) {
         if (t == kBulkThread) {
-            ptx::mbar_expect_tx(tma_bar, 3 * 16384);
+            ptx::mbar_expect_tx(tma_bar, (has_q ? 3 : 2) * 16384);
             const int x = ho * kD, y = (int)Lo.tok0;
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 ptx::tma_load_2d(smem + S_KQ + hf * S_KQ_HALF, &tm_k, x + hf * 64, y, tma_bar);
-                ptx::tma_load_2d(smem + S_KQ + hf * S_KQ_HALF + 8192, &tm_q, x + hf * 64, y, tma_bar);
+                if (has_q)
+                    ptx::tma_load_2d(smem + S_KQ + hf * S_KQ_HALF + 8192, &tm_q, x + hf * 64, y, tma_bar);
                 ptx::tma_load_2d(smem + S_V + hf * S_V_BLOCK, &tm_v, x + hf * 64, y, tma_bar);
             }
         }
@@ -283,34 +289,42 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         }
     }
     const int hf = c4 >> 4;                       // K-half (channels 0-63 / 64-127)
+    // (state-only calls produce no output: the query half is skipped altogether; the choice is made
+    // outside the loop so that each version stays branch-free)
+    auto gate_rows = [&](auto with_q) {
+        constexpr bool kQ = decltype(with_q)::value;
 #pragma unroll
-    for (int r = 0; r < kRPT; ++r) {
-        const int i = i0 + r;
-        const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
-        uint8_t* pk = smem + S_KQ + hf * S_KQ_HALF + off;
-        uint2 k2 = *reinterpret_cast<const uint2*>(pk);
-        uint2 q2 = *reinterpret_cast<const uint2*>(pk + 8192);
-        if (i >= L.len) k2 = q2 = make_uint2(0u, 0u);
-        if (!has_q) q2 = make_uint2(0u, 0u);
-        const float kf[4] = {__uint_as_float(k2.x << 16), __uint_as_float(k2.x & 0xffff0000u),
-                             __uint_as_float(k2.y << 16), __uint_as_float(k2.y & 0xffff0000u)};
-        const float qf[4] = {__uint_as_float(q2.x << 16), __uint_as_float(q2.x & 0xffff0000u),
-                             __uint_as_float(q2.y << 16), __uint_as_float(q2.y & 0xffff0000u)};
-        float okg[4], oqg[4], oki[4];
+        for (int r = 0; r < kRPT; ++r) {
+            const int i = i0 + r;
+            const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
+            uint8_t* pk = smem + S_KQ + hf * S_KQ_HALF + off;
+            uint2 k2 = *reinterpret_cast<const uint2*>(pk);
+            uint2 q2 = make_uint2(0u, 0u);
+            if (kQ) q2 = *reinterpret_cast<const uint2*>(pk + 8192);
+            if (i >= L.len) k2 = q2 = make_uint2(0u, 0u);
+            const float kf[4] = {__uint_as_float(k2.x << 16), __uint_as_float(k2.x & 0xffff0000u),
+                                 __uint_as_float(k2.y << 16), __uint_as_float(k2.y & 0xffff0000u)};
+            const float qf[4] = {__uint_as_float(q2.x << 16), __uint_as_float(q2.x & 0xffff0000u),
+                                 __uint_as_float(q2.y << 16), __uint_as_float(q2.y & 0xffff0000u)};
+            float okg[4], oqg[4], oki[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float x = fminf(fmaxf(G[r][e] + base[e] - gref[e], -kClamp2), kClamp2);
-            const float e1 = ex2(x);                     // exp(G - G_m)
-            const float e2 = ex2(-x);                    // exp(G_m - G)
-            okg[e] = kf[e] * e1;
-            oqg[e] = a.scale * qf[e] * e1;
-            oki[e] = kf[e] * e2;
+            for (int e = 0; e < 4; ++e) {
+                const float x = fminf(fmaxf(G[r][e] + base[e] - gref[e], -kClamp2), kClamp2);
+                const float e1 = ex2(x);                     // exp(G - G_m)
+                const float e2 = ex2(-x);                    // exp(G_m - G)
+                okg[e] = kf[e] * e1;
+                oqg[e] = a.scale * qf[e] * e1;
+                oki[e] = kf[e] * e2;
+            }
+            *reinterpret_cast<uint2*>(pk) = make_uint2(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]));
+            if (kQ)
+                *reinterpret_cast<uint2*>(pk + 8192) =
+                    make_uint2(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]));
+            *reinterpret_cast<uint2*>(smem + S_KI + hf * S_KI_HALF + off) =
+                make_uint2(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]));
         }
-        *reinterpret_cast<uint2*>(pk) = make_uint2(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]));
-        *reinterpret_cast<uint2*>(pk + 8192) = make_uint2(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]));
-        *reinterpret_cast<uint2*>(smem + S_KI + hf * S_KI_HALF + off) =
-            make_uint2(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]));
-    }
+    };
+    gate_rows(std::integral_constant<bool, kHasQ>{});
 
     KDA_PHASE(hdr, 12);  // element loop + stores (thread 0)
     ptx::fence_async_smem();
@@ -323,8 +337,10 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     if (t == kBulkThread) {
         // phase-1 outputs leave through the TMA engine while the MMA runs
         // Q' (rows 64-127 of both K-halves of the operand image) and K' are tile contents as they are
-        ptx::bulk_s2g(tile + tc::OFF_QW + 8192, smem + S_KQ + 8192, 8192);
-        ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF + 8192, smem + S_KQ + S_KQ_HALF + 8192, 8192);
+        if (has_q) {
+            ptx::bulk_s2g(tile + tc::OFF_QW + 8192, smem + S_KQ + 8192, 8192);
+            ptx::bulk_s2g(tile + tc::OFF_QW + tc::QW_HALF + 8192, smem + S_KQ + S_KQ_HALF + 8192, 8192);
+        }
         ptx::bulk_s2g(tile + tc::OFF_KI, smem + S_KI, 16384);
         ptx::bulk_commit();
     }
@@ -365,7 +381,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
                 }
                 *reinterpret_cast<float4*>(sA + i * LDT + c0 + j4) = make_float4(x[0], x[1], x[2], x[3]);
             }
-        } else {
+        } else if (has_q) {
             const int i = R - 64;
 #pragma unroll
             for (int j8 = 0; j8 < NCA; j8 += 8) {
@@ -384,7 +400,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     ptx::fence_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
-    if (t == kBulkThread) {
+    if (t == kBulkThread && has_q) {
         ptx::bulk_s2g(tile + tc::OFF_AQ, smem + S_AQ, 8192);
         ptx::bulk_commit();
     }
@@ -600,7 +616,9 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, boo
 {
     static bool attr_done = false;
     if (!attr_done) {
-        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)kIntraTcSmem));
+        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)kIntraTcSmem));
         attr_done = true;
     }
@@ -622,8 +640,10 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, boo
     const int64_t resident = 2 * (int64_t)n_sm;   // two CTAs per SM
     const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
     ProfScope ps(PROF_INTRA, st);
-    kda_intra_tc<<<grid, kNT, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, a.q ? 1 : 0,
-                                                     clear_status ? 1 : 0);
+    if (a.q && a.o)
+        kda_intra_tc<true><<<grid, kNT, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
+    else
+        kda_intra_tc<false><<<grid, kNT, kIntraTcSmem, st>>>(a, (char*)tiles, hdr, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;
