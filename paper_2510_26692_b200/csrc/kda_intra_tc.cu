@@ -242,6 +242,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     int hn = h;
 
     // ---- a1: cumulative log-decay, in the log2 domain (exponentials below are bare ex2) -------
+    KDA_PHASE(hdr, 13);  // loop overhead
 #pragma unroll
     for (int e = 0; e < 4; ++e) G[0][e] *= kLog2e;
 #pragma unroll
@@ -249,7 +250,9 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
 #pragma unroll
         for (int e = 0; e < 4; ++e) G[r][e] = fmaf(G[r][e], kLog2e, G[r - 1][e]);
     *reinterpret_cast<float4*>(sTot + warp * kD + d0) = make_float4(G[kRPT - 1][0], G[kRPT - 1][1], G[kRPT - 1][2], G[kRPT - 1][3]);
+    KDA_PHASE(hdr, 14);  // G arrived + local scan
     ptx::cp_async_wait_all();             // beta
+    KDA_PHASE(hdr, 15);  // beta wait
     __syncthreads();
     KDA_PHASE(hdr, 0);   // loads arrived + local scan
     float base[4] = {0.f, 0.f, 0.f, 0.f}, gref[4] = {0.f, 0.f, 0.f, 0.f}, glast[4] = {0.f, 0.f, 0.f, 0.f};
@@ -352,6 +355,10 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
             ptx::umma_bf16(tmem_base, ptx::umma_desc_sw128(a0 + (k >> 2) * S_KQ_HALF + (k & 3) * 32),
                            ptx::umma_desc_sw128(b0 + (k >> 2) * S_KI_HALF + (k & 3) * 32), idesc, k > 0);
         ptx::umma_commit(mma_bar);
+    }
+    if (nxt < ntiles) {   // the next tile's log alpha: a whole tile ahead (its registers are free since the gating loop)
+        locate(nxt, Ln, hn);
+        prefetch_regs(Ln, hn);
     }
     if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) timed_out = true;
     // the previous tile's W/U staging (and this tile's Q', K' stores) have been read out by now; the
@@ -508,10 +515,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
             ptx::umma_bf16(tmem_base + 128, ptx::umma_desc_sw128(m0 + k * 32),
                            ptx::umma_desc_sw128_mn(v0 + k * 2048, S_V_BLOCK), idesc, k > 0);
         ptx::umma_commit(mma_bar);
-    }
-    if (nxt < ntiles) {   // request the next tile: registers now, buffers once the MMAs are done with them
-        locate(nxt, Ln, hn);
-        prefetch_regs(Ln, hn);
     }
     if (!ptx::mbar_wait(mma_bar, 1, kWaitLimitNs)) timed_out = true;
     if (nxt < ntiles) prefetch_bufs(Ln, hn);
