@@ -26,6 +26,19 @@ __device__ __forceinline__ void st_stream(float* p, float4 x) {
                  "f"(x.y), "f"(x.z), "f"(x.w)
                  : "memory");
 }
+// packed fp32 arithmetic (two independent round-to-nearest operations per instruction on sm_100):
+// the multi-token kernel is bound by instruction issue, not by HBM
+__device__ __forceinline__ void mul4(float4& x, float a) {
+    const float2 aa = make_float2(a, a);
+    const float2 lo = __fmul2_rn(make_float2(x.x, x.y), aa), hi = __fmul2_rn(make_float2(x.z, x.w), aa);
+    x = make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ void fma4(float4& acc, float a, const float4& x) {   // acc += a * x
+    const float2 aa = make_float2(a, a);
+    const float2 lo = __ffma2_rn(aa, make_float2(x.x, x.y), make_float2(acc.x, acc.y));
+    const float2 hi = __ffma2_rn(aa, make_float2(x.z, x.w), make_float2(acc.z, acc.w));
+    acc = make_float4(lo.x, lo.y, hi.x, hi.y);
+}
 template <typename T> __device__ __forceinline__ float to_f(T x);
 template <> __device__ __forceinline__ float to_f<float>(float x) { return x; }
 template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 x) {
@@ -113,7 +126,9 @@ kda_decode_multi_kernel(const T* __restrict__ q, const T* __restrict__ k, const 
                         const float* __restrict__ log_alpha, const float* __restrict__ beta, float* S,
                         const int32_t* __restrict__ slot, T* __restrict__ o, int H, int n_tok, float scale)
 {
-    __shared__ float s_a[2][kD], s_k[2][kD], s_q[2][kD];
+    constexpr int GT = 8;   // tokens whose vectors are staged together: one memory latency per group
+    __shared__ float s_a[GT][kD], s_k[GT][kD], s_q[GT][kD], s_v[GT][kD];
+    __shared__ float s_b[GT];
     __shared__ float4 s_red[2][2][8][32];
     const int item = blockIdx.x;
     const int n = item / H, h = item - n * H;
@@ -126,75 +141,74 @@ kda_decode_multi_kernel(const T* __restrict__ q, const T* __restrict__ k, const 
     for (int m = 0; m < 16; ++m) x[m] = ld_stream(Sp + (size_t)(warp + 8 * m) * kD);
 
     auto vec_of = [&](int tt) { return ((size_t)(n * n_tok + tt) * H + h) * kD; };
-    // the per-token vectors are fetched one token ahead (threads 0-127: one channel each)
-    float pa = 0.f, pk = 0.f, pq = 0.f;
-    if (t < kD) {
-        const size_t vec = vec_of(0);
-        pa = log_alpha[vec + t];
-        pk = to_f<T>(k[vec + t]);
-        pq = to_f<T>(q[vec + t]);
-    }
-    float bt_next = beta[(size_t)(n * n_tok) * H + h];
-    float4 vv_next = IO<T>::load4(v + vec_of(0) + lane * 4);
-    for (int tt = 0; tt < n_tok; ++tt) {
-        const int b = tt & 1;
-        if (t < kD) {
-            s_a[b][t] = expf(pa);
-            s_k[b][t] = pk;
-            s_q[b][t] = pq;
-            if (tt + 1 < n_tok) {
-                const size_t vec = vec_of(tt + 1);
-                pa = log_alpha[vec + t];
-                pk = to_f<T>(k[vec + t]);
-                pq = to_f<T>(q[vec + t]);
+    for (int g0 = 0; g0 < n_tok; g0 += GT) {
+        const int gn = (n_tok - g0) < GT ? (n_tok - g0) : GT;
+        __syncthreads();   // the previous group's vectors are no longer read
+        {   // thread (half, c): channel c of tokens half, half + 2, ...  -- all loads first, then the stores
+            const int c = t & (kD - 1), half = t >> 7;
+            float la[GT / 2], kk[GT / 2], qq[GT / 2], vv[GT / 2];
+#pragma unroll
+            for (int j = 0; j < GT / 2; ++j) {
+                const int tok = half + 2 * j;
+                if (tok < gn) {
+                    const size_t vec = vec_of(g0 + tok) + c;
+                    la[j] = log_alpha[vec];
+                    kk[j] = to_f<T>(k[vec]);
+                    qq[j] = to_f<T>(q[vec]);
+                    vv[j] = to_f<T>(v[vec]);
+                }
             }
-        }
-        const size_t vec = vec_of(tt);
-        const float bt = bt_next;
-        const float4 vv = vv_next;
-        if (tt + 1 < n_tok) {
-            bt_next = beta[(size_t)(n * n_tok + tt + 1) * H + h];
-            vv_next = IO<T>::load4(v + vec_of(tt + 1) + lane * 4);
+#pragma unroll
+            for (int j = 0; j < GT / 2; ++j) {
+                const int tok = half + 2 * j;
+                if (tok < gn) {
+                    s_a[tok][c] = expf(la[j]);
+                    s_k[tok][c] = kk[j];
+                    s_q[tok][c] = qq[j];
+                    s_v[tok][c] = vv[j];
+                }
+            }
+            if (t < gn) s_b[t] = beta[(size_t)(n * n_tok + g0 + t) * H + h];
         }
         __syncthreads();
+        for (int tok = 0; tok < gn; ++tok) {
+            const int b = tok & 1;
+            const float bt = s_b[tok];
+            const float4 vv = *reinterpret_cast<const float4*>(&s_v[tok][lane * 4]);
+            float qk = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) qk += s_q[tok][lane * 4 + i] * s_k[tok][lane * 4 + i];
+#pragma unroll
+            for (int ofs = 16; ofs > 0; ofs >>= 1) qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
 
-        float qk = 0.f;
+            float4 p = make_float4(0.f, 0.f, 0.f, 0.f), s = p;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) qk += s_q[b][lane * 4 + i] * s_k[b][lane * 4 + i];
+            for (int m = 0; m < 16; ++m) {
+                const int row = warp + 8 * m;
+                mul4(x[m], s_a[tok][row]);
+                fma4(p, s_k[tok][row], x[m]);
+                fma4(s, s_q[tok][row], x[m]);
+            }
+            s_red[b][0][warp][lane] = p;
+            s_red[b][1][warp][lane] = s;
+            __syncthreads();
+            p = s_red[b][0][0][lane];
+            s = s_red[b][1][0][lane];
 #pragma unroll
-        for (int ofs = 16; ofs > 0; ofs >>= 1) qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
-
-        float4 p = make_float4(0.f, 0.f, 0.f, 0.f), s = p;
+            for (int w = 1; w < 8; ++w) {   // fixed order: bitwise reproducible
+                float4 a4 = s_red[b][0][w][lane], b4 = s_red[b][1][w][lane];
+                p.x += a4.x; p.y += a4.y; p.z += a4.z; p.w += a4.w;
+                s.x += b4.x; s.y += b4.y; s.z += b4.z; s.w += b4.w;
+            }
+            const float4 r = make_float4(vv.x - p.x, vv.y - p.y, vv.z - p.z, vv.w - p.w);
+            if (warp == 0) {
+                const float c = bt * qk;
+                IO<T>::store4(o + vec_of(g0 + tok) + lane * 4,
+                              make_float4(scale * (s.x + c * r.x), scale * (s.y + c * r.y),
+                                          scale * (s.z + c * r.z), scale * (s.w + c * r.w)));
+            }
 #pragma unroll
-        for (int m = 0; m < 16; ++m) {
-            const int row = warp + 8 * m;
-            const float a = s_a[b][row], kk = s_k[b][row], qq = s_q[b][row];
-            x[m].x *= a; x[m].y *= a; x[m].z *= a; x[m].w *= a;
-            p.x += kk * x[m].x; p.y += kk * x[m].y; p.z += kk * x[m].z; p.w += kk * x[m].w;
-            s.x += qq * x[m].x; s.y += qq * x[m].y; s.z += qq * x[m].z; s.w += qq * x[m].w;
-        }
-        s_red[b][0][warp][lane] = p;
-        s_red[b][1][warp][lane] = s;
-        __syncthreads();
-        p = s_red[b][0][0][lane];
-        s = s_red[b][1][0][lane];
-#pragma unroll
-        for (int w = 1; w < 8; ++w) {   // fixed order: bitwise reproducible
-            float4 a4 = s_red[b][0][w][lane], b4 = s_red[b][1][w][lane];
-            p.x += a4.x; p.y += a4.y; p.z += a4.z; p.w += a4.w;
-            s.x += b4.x; s.y += b4.y; s.z += b4.z; s.w += b4.w;
-        }
-        const float4 r = make_float4(vv.x - p.x, vv.y - p.y, vv.z - p.z, vv.w - p.w);
-        if (warp == 0) {
-            const float c = bt * qk;
-            IO<T>::store4(o + vec + lane * 4,
-                          make_float4(scale * (s.x + c * r.x), scale * (s.y + c * r.y),
-                                      scale * (s.z + c * r.z), scale * (s.w + c * r.w)));
-        }
-#pragma unroll
-        for (int m = 0; m < 16; ++m) {
-            const float c = bt * s_k[b][warp + 8 * m];
-            x[m].x += c * r.x; x[m].y += c * r.y; x[m].z += c * r.z; x[m].w += c * r.w;
+            for (int m = 0; m < 16; ++m) fma4(x[m], bt * s_k[tok][warp + 8 * m], r);
         }
     }
 #pragma unroll
