@@ -166,8 +166,8 @@ def oracle_arm(args, rank):
 
 
 def extra_workloads(K, inputs, torch, dev, peaks):
-    """Device-resident timing of the packed varlen batch (BASELINE configs[2]) and of the 1 Mi-token
-    state-only prefill (configs[3]); inputs are far larger than L2, so no rotation is needed."""
+    """Device-resident timing of the packed varlen batch (the packed-batch workload) and of the 1 Mi-token
+    state-only prefill; inputs are far larger than L2, so no rotation is needed."""
     out = {}
     stream = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -484,10 +484,10 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": "prefill B=1 T=4096 H=32 dk=dv=128 chunk=64, bf16 q/k/v, fp32 "
-                                   "gates/beta/state, S0~N(0,0.02) (BASELINE configs[1]); one batch "
+                                   "gates/beta/state, S0~N(0,0.02); one batch "
                                    "per GPU",
                        "l2": "inputs rotate over 3 copies of 206 MB each (> 126 MB L2)",
-                       "decode_workload": "256 seqs x 32 heads, 64 in-place steps (BASELINE configs[4])"},
+                       "decode_workload": "256 seqs x 32 heads, 64 in-place steps"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
             "decode": decode, "cpu_baseline": cpu,
         }
