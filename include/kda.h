@@ -17,10 +17,10 @@
  *   - All tensors are dense, innermost dimension contiguous, token-major:
  *       q, k, log_alpha : [total_tokens, H, dk]     v, o : [total_tokens, H, dv]
  *       beta            : [total_tokens, H]         S0, S_T, S : [n, H, dk, dv]  (dv contiguous)
- *   - alpha_t = exp(log_alpha_t), log_alpha <= 0 (a decay).  Within either 32-token half of a
- *     64-token chunk the cumulative log-decay of a channel must stay above -80 (a factor e^-80);
- *     below that the intra-chunk interactions of that channel are attenuated (they never overflow
- *     or turn NaN: exponents are clamped).
+ *   - alpha_t = exp(log_alpha_t), log_alpha <= 0 (a decay).  The cumulative log-decay of a channel
+ *     over one 64-token chunk must stay above -160 (a factor e^-160); below that the intra-chunk
+ *     interactions of that channel are attenuated (they never overflow or turn NaN: exponents are
+ *     clamped).
  *   - dt selects the storage type of q, k, v and o (fp32 or bf16).  Gates, beta and states are
  *     always fp32.  dt = KDA_BF16 runs the contractions on bf16 tensor cores with fp32
  *     accumulation; dt = KDA_F32 runs everything in fp32 FMA arithmetic.

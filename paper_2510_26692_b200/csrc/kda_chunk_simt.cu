@@ -13,7 +13,7 @@
 //          S <- Diag(gamma^C) S + ((gamma^C/Gamma).K)^T V_new (a8).  State columns are independent,
 //          which is what lets dv be sliced across CTAs.
 //
-// The decay ratios exp(G_i - G_j) are factored around the chunk's middle row m = 31 as
+// The decay ratios exp(G_i - G_j) are factored around G_m = G_C / 2 (per channel) as
 // exp(G_i - G_m) * exp(G_m - G_j), with each exponent clamped to [-80, 80], so no product
 // overflows fp32; entries above the diagonal are never used (selected to zero, not multiplied).
 #include "kda_common.cuh"
@@ -23,7 +23,6 @@ namespace {
 
 constexpr int LD = kD + 4;           // padded fp32 row (keeps float4 alignment, spreads banks)
 constexpr int LDA = kC + 1;
-constexpr int kRef = kC / 2 - 1;     // reference row of the decay factorisation
 constexpr float kClamp = 80.f;
 
 // scratch tile (floats)
@@ -92,8 +91,8 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, float* __r
             if (qp) qv = IO<T>::load4(qp + off);
         }
         const float4 G = *reinterpret_cast<const float4*>(sG + i * LD + c);
-        const float4 Gr = *reinterpret_cast<const float4*>(sG + kRef * LD + c);
         const float4 Gl = *reinterpret_cast<const float4*>(sG + (kC - 1) * LD + c);
+        const float4 Gr = make_float4(0.5f * Gl.x, 0.5f * Gl.y, 0.5f * Gl.z, 0.5f * Gl.w);   // reference: G_C / 2
         const float kk[4] = {kv.x, kv.y, kv.z, kv.w}, qq[4] = {qv.x, qv.y, qv.z, qv.w};
         const float gg[4] = {G.x, G.y, G.z, G.w}, gr[4] = {Gr.x, Gr.y, Gr.z, Gr.w};
         const float gl[4] = {Gl.x, Gl.y, Gl.z, Gl.w};

@@ -312,15 +312,11 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
             const float gc = reinterpret_cast<const float*>(sb + Cfg::kGC)[tid];          // gamma^C
             const float ct = reinterpret_cast<const float*>(sb + Cfg::kGC + 1024)[tid];   // exp(G_C - G_m)
             const float cgn = ref_scale_of(it + 1);   // fetched off the chain, before the wait below
-            // the next operand copy is exp(G_m') . S_new = (cgn gc) . S + (cgn ct) . D3: everything that
-            // does not need D3 is formed before the wait
-            float zpre[NS];
-            const float zb = cgn * ct;
-            {
-                const float za = cgn * gc;
+            // S_new = gc . S + ct . D3; the part that does not need D3 is formed before the wait.  (The
+            // scales are applied one after the other: ct . D3 is of ordinary size although ct can be
+            // e^-80 and D3 e^+80, whereas a pre-multiplied cgn * ct would underflow.)
 #pragma unroll
-                for (int j = 0; j < NS; ++j) zpre[j] = za * S[j];
-            }
+            for (int j = 0; j < NS; ++j) S[j] *= gc;
             wait(mma2_bar, par, 3);
             KDA_PHASE(hdr, 20);  // MMA2
             ptx::tc_fence_after();
@@ -328,14 +324,11 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 float ds[NS];
                 tmem_ld_sum<NS>(tmem_lane + d3, ds);
 #pragma unroll
-                for (int j = 0; j < NS; ++j) zpre[j] = fmaf(zb, ds[j], zpre[j]);
-                store_row<NS>(sbf, tid, zpre);
+                for (int j = 0; j < NS; ++j) S[j] = fmaf(ct, ds[j], S[j]);
+                store_scaled(cgn);   // next chunk's operand copy: bf16(exp(G_m') . S_new)
                 ptx::fence_async_smem();
                 ptx::tc_fence_before();
                 warp_arrive(sbf_ready);
-                // the fp32 master copy itself is not on the chain
-#pragma unroll
-                for (int j = 0; j < NS; ++j) S[j] = fmaf(ct, ds[j], gc * S[j]);
             }
             KDA_PHASE(hdr, 21);  // state update
             if (warp >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64)

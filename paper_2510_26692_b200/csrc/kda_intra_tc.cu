@@ -5,9 +5,9 @@
 //   a1   G = cumulative sum of log alpha over the chunk's tokens (fp32, registers + one exchange
 //        through shared memory)
 //        gated operands, all bf16:  Kg = K exp(G - G_m),  Qg = scale Q exp(G - G_m),
-//        Ki = K exp(G_m - G)   (m = row 31, the middle of the chunk, so that neither factor of
-//        exp(G_i - G_j) = exp(G_i - G_m) exp(G_m - G_j) leaves the bf16/fp32 range; exponents are
-//        clamped to +-80).  The same three images serve the inter-chunk stage, which restores the
+//        Ki = K exp(G_m - G)   (G_m = G_C / 2 per channel, the middle of the chunk's log-decay range,
+//        so that neither factor of exp(G_i - G_j) = exp(G_i - G_m) exp(G_m - G_j) leaves the
+//        bf16/fp32 range; exponents are clamped to +-80).  The same three images serve the inter-chunk stage, which restores the
 //        true scales exp(G_m), exp(G_C - G_m) in fp32 on its side
 //   a2/a5  one tcgen05 MMA group  [Kg ; Qg] (128 x 128)  x  Ki^T (128 x 64)  ->  TMEM:
 //        rows 0-63  = raw key Gram matrix, rows 64-127 = raw query-key matrix
@@ -263,10 +263,13 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (r2 < warp) base[e] += x[e];
-            if (r2 < kNW / 2) gref[e] += x[e];    // rows 0..31
             glast[e] += x[e];
         }
     }
+    // reference of the decay factorisation: half the chunk's total log-decay, per channel, so that
+    // |G_i - G_ref| <= |G_C| / 2 for every row whatever the distribution of the decay over the chunk
+#pragma unroll
+    for (int e = 0; e < 4; ++e) gref[e] = 0.5f * glast[e];
 
     // ---- gated operands ---------------------------------------------------------------------------------
     // the true scales exp(G_m), exp(G_C - G_m) and gamma^C go to the tile as fp32 vectors; the

@@ -200,6 +200,15 @@ def test_equal_length_batch(oracle_mod):
     check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
 
 
+def test_very_harsh_gates(oracle_mod):
+    """logsigmoid(N(-1.5,1)): about e^-110 per chunk and channel, inside the supported e^-160
+    (a reference taken at the middle token row instead of the middle of the log-decay range would
+    already clamp here whenever the decay is uneven over the chunk)."""
+    for dtype, tol in ((torch.float32, TOL[K.KDA_F32]), (torch.bfloat16, TOL[K.KDA_BF16])):
+        d = inputs.chunk_inputs([200], H=2, dtype=dtype, seed=37, gate_mean=-1.5, s0_std=0.02)
+        check_chunk(oracle_mod, d, tol)
+
+
 def test_beta_extremes(oracle_mod):
     d = inputs.chunk_inputs([192], H=2, dtype=torch.float32, seed=28, s0_std=0.02)
     for val in (0.0, 1.0):
