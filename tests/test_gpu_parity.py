@@ -134,6 +134,20 @@ def test_small_workspace_multi_pass(oracle_mod):
     check_chunk(oracle_mod, d, TOL[K.KDA_F32], workspace_bytes=lo)
 
 
+def test_small_workspace_multi_pass_bf16(oracle_mod):
+    """Same on the tensor-core path, packed batch: passes cut sequences at arbitrary chunk indices."""
+    lens = [700, 130, 64, 900, 0, 333]
+    d = inputs.chunk_inputs(lens, H=3, dtype=torch.bfloat16, seed=42, s0_std=0.02)
+    full = run_chunk(d)
+    N, T = len(lens), sum(lens)
+    lo = K.kda_chunk_fwd_min_workspace_bytes(T, N, 3, dt=K.KDA_BF16)
+    hi = K.kda_chunk_fwd_workspace_bytes(T, N, 3, dt=K.KDA_BF16)
+    for nbytes in (lo, lo + (hi - lo) // 5, lo + (hi - lo) // 2):
+        part = run_chunk(d, workspace_bytes=nbytes)
+        assert torch.equal(part[0], full[0]) and torch.equal(part[1], full[1])
+    check_chunk(oracle_mod, d, TOL[K.KDA_BF16], workspace_bytes=lo + (hi - lo) // 5)
+
+
 def test_scale_argument(oracle_mod):
     d = inputs.chunk_inputs([130], H=2, dtype=torch.float32, seed=24, scale_q=False)
     check_chunk(oracle_mod, d, TOL[K.KDA_F32], scale=128 ** -0.5)
@@ -374,3 +388,41 @@ def test_random_packed_batches(oracle_mod, seed):
                             s0_std=0.02 if seed % 2 else 0.0, gate_mean=float(torch.randint(0, 6, (1,), generator=g)))
     d["force_varlen"] = True
     check_chunk(oracle_mod, d, TOL[K.KDA_BF16 if bf16 else K.KDA_F32])
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_gate_and_scale_regimes(oracle_mod, dtype):
+    """No decay at all (alpha = 1, the delta rule), very slow decay, decay rates that differ by two
+    orders of magnitude between heads and channels, large values and a large initial state."""
+    tol = TOL[K.KDA_BF16 if dtype == torch.bfloat16 else K.KDA_F32]
+    T, H = 330, 4
+    base = inputs.chunk_inputs([T], H=H, dtype=dtype, seed=38, s0_std=0.02)
+    # alpha = 1
+    d = dict(base); d["log_alpha"] = torch.zeros_like(base["log_alpha"])
+    check_chunk(oracle_mod, d, tol)
+    # very slow decay
+    d = inputs.chunk_inputs([T], H=H, dtype=dtype, seed=39, s0_std=0.02, gate_mean=10.0)
+    check_chunk(oracle_mod, d, tol)
+    # per-head and per-channel spread of the decay rate: factors 0.03 ... 30 on the log-decay
+    d = dict(base)
+    g = torch.Generator().manual_seed(40)
+    factor = torch.exp(torch.empty((1, H, 128)).uniform_(-3.5, 3.4, generator=g))
+    d["log_alpha"] = (base["log_alpha"] * factor).clamp(min=-2.4)   # stays inside e^-160 per chunk
+    check_chunk(oracle_mod, d, tol)
+    # large values and a large initial state
+    d = dict(base)
+    d["v"] = (base["v"].float() * 64.0).to(dtype)
+    d["S0"] = base["S0"] * 500.0
+    check_chunk(oracle_mod, d, tol)
+
+
+def test_exact_recall_on_gpu(oracle_mod):
+    """beta = 1 and unit keys: querying with the key returns the value just written, o_t = scale v_t,
+    whatever the gates and the earlier state (reconstruction objective of Section 2.2).  Checked on
+    the fp32 path directly against v, without the oracle."""
+    T, H = 200, 2
+    d = inputs.chunk_inputs([T], H=H, dtype=torch.float32, seed=41, s0_std=0.5, scale_q=False)
+    d["q"] = d["k"].clone()
+    d["beta"] = torch.ones_like(d["beta"])
+    o, _ = run_chunk(d, scale=2.0)
+    assert rel_l2(to_np32(o), 2.0 * to_np32(d["v"])) < 1e-4
