@@ -148,6 +148,25 @@ def test_small_workspace_multi_pass_bf16(oracle_mod):
     check_chunk(oracle_mod, d, TOL[K.KDA_BF16], workspace_bytes=lo + (hi - lo) // 5)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_state_in_place(oracle_mod, dtype):
+    """S0 and S_T may be the same buffer (a state cache updated in place by a prefill)."""
+    lens = [150, 64, 700]
+    d = inputs.chunk_inputs(lens, H=2, dtype=dtype, seed=43, s0_std=0.02)
+    o_ref, S_ref = run_chunk(d)
+    g = {n: (t.cuda() if isinstance(t, torch.Tensor) else t) for n, t in d.items()}
+    T, N = sum(lens), len(lens)
+    dt = K.KDA_BF16 if dtype == torch.bfloat16 else K.KDA_F32
+    nb = K.kda_chunk_fwd_workspace_bytes(T, N, 2, dt=dt)
+    ws = torch.empty(nb, dtype=torch.uint8, device="cuda:0")
+    o = torch.empty_like(g["v"])
+    S = g["S0"].clone()
+    K.kda_chunk_fwd(g["q"], g["k"], g["v"], g["log_alpha"], g["beta"], S, o, S, g["cu_seqlens"],
+                    d["cu_seqlens"], N, T, 2, 128, 128, 64, 1.0, dt, ws, nb)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o_ref) and torch.equal(S, S_ref)
+
+
 def test_scale_argument(oracle_mod):
     d = inputs.chunk_inputs([130], H=2, dtype=torch.float32, seed=24, scale_q=False)
     check_chunk(oracle_mod, d, TOL[K.KDA_F32], scale=128 ** -0.5)
