@@ -166,8 +166,11 @@ kda_status_t kda_decode_multi(const void *q, const void *k, const void *v, const
  * from / written to HOST memory (pinned memory makes the copies asynchronous).  The device copies
  * live in the caller's device workspace, so these allocate nothing either.  cu_seqlens is given on
  * the host only.  For decode the states stay on the device (they are the resident cache);
- * state_slot is a host array or NULL.  Copies and kernels are enqueued on `cuda_stream`; outputs
- * are valid after the stream is synchronised.
+ * state_slot is a host array or NULL.  Outputs are valid after `cuda_stream` is synchronised.  For
+ * one long sequence (n_seqs = 1, at least 1024 tokens) kda_chunk_fwd_host pipelines copy-in,
+ * compute and copy-out over up to four segments of the sequence, using two helper streams that the
+ * library creates once per process; everything is still ordered after prior work on `cuda_stream`
+ * and complete when `cuda_stream` is.
  */
 size_t kda_chunk_fwd_host_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
                                           int chunk, kda_dtype_t dt);

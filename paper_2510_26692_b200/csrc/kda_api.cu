@@ -336,6 +336,79 @@ kda_status_t kda_chunk_fwd_host(const void* q_host, const void* k_host, const vo
     char* ws = static_cast<char*>(workspace);
     const size_t e = esize(dt), td = (size_t)total_tokens * H * kD;
     const size_t sb = (size_t)n_seqs * H * kD * kD * 4;
+
+    // One long sequence: copy-in, compute and copy-out are pipelined over a few segments of the
+    // sequence (the state handed from one segment to the next is exactly the resume property of
+    // the recurrence), on two helper streams owned by the library, so that the host link is busy
+    // in both directions while the kernels run.
+    constexpr int64_t kMinSegTokens = 512;
+    if (n_seqs == 1 && !cu_seqlens_host && total_tokens >= 2 * kMinSegTokens) {
+        static cudaStream_t c_in = nullptr, c_out = nullptr;
+        if (!c_in) {
+            KDA_CUDA_TRY(cudaStreamCreateWithFlags(&c_in, cudaStreamNonBlocking));
+            KDA_CUDA_TRY(cudaStreamCreateWithFlags(&c_out, cudaStreamNonBlocking));
+        }
+        int nseg = (int)(total_tokens / kMinSegTokens);
+        if (nseg > 4) nseg = 4;
+        const int64_t seg = ((total_tokens + nseg - 1) / nseg + kC - 1) / kC * kC;
+        std::vector<cudaEvent_t> evs;
+        auto new_event = [&](cudaEvent_t* ev) {
+            cudaError_t err = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+            if (err == cudaSuccess) evs.push_back(*ev);
+            return err;
+        };
+        kda_status_t rc = KDA_OK;
+        cudaError_t cerr = cudaSuccess;
+#define KDA_PIPE_TRY(expr)                                                          \
+    if (rc == KDA_OK && cerr == cudaSuccess) {                                      \
+        cerr = (expr);                                                              \
+        if (cerr != cudaSuccess)                                                    \
+            rc = fail(KDA_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(cerr)); \
+    }
+        cudaEvent_t fork = nullptr, join = nullptr;
+        KDA_PIPE_TRY(new_event(&fork));
+        KDA_PIPE_TRY(cudaEventRecord(fork, st));
+        KDA_PIPE_TRY(cudaStreamWaitEvent(c_in, fork, 0));
+        if (S0_host) KDA_PIPE_TRY(cudaMemcpyAsync(ws + L0.s0, S0_host, sb, cudaMemcpyHostToDevice, c_in));
+        float* state = reinterpret_cast<float*>(ws + L0.st);
+        for (int64_t t0 = 0, k = 0; t0 < total_tokens && rc == KDA_OK; t0 += seg, ++k) {
+            const int64_t t1 = (t0 + seg < total_tokens) ? t0 + seg : total_tokens;
+            const size_t r0 = (size_t)t0 * H * kD, rn = (size_t)(t1 - t0) * H * kD;
+            if (q_host)
+                KDA_PIPE_TRY(cudaMemcpyAsync(ws + L0.q + r0 * e, (const char*)q_host + r0 * e, rn * e, cudaMemcpyHostToDevice, c_in));
+            KDA_PIPE_TRY(cudaMemcpyAsync(ws + L0.k + r0 * e, (const char*)k_host + r0 * e, rn * e, cudaMemcpyHostToDevice, c_in));
+            KDA_PIPE_TRY(cudaMemcpyAsync(ws + L0.v + r0 * e, (const char*)v_host + r0 * e, rn * e, cudaMemcpyHostToDevice, c_in));
+            KDA_PIPE_TRY(cudaMemcpyAsync(ws + L0.g + r0 * 4, (const char*)log_alpha_host + r0 * 4, rn * 4, cudaMemcpyHostToDevice, c_in));
+            KDA_PIPE_TRY(cudaMemcpyAsync(ws + L0.b + (size_t)t0 * H * 4, (const char*)beta_host + (size_t)t0 * H * 4,
+                                         (size_t)(t1 - t0) * H * 4, cudaMemcpyHostToDevice, c_in));
+            cudaEvent_t in_done = nullptr, out_ready = nullptr;
+            KDA_PIPE_TRY(new_event(&in_done));
+            KDA_PIPE_TRY(cudaEventRecord(in_done, c_in));
+            KDA_PIPE_TRY(cudaStreamWaitEvent(st, in_done, 0));
+            if (rc == KDA_OK)
+                rc = kda_chunk_fwd(q_host ? ws + L0.q + r0 * e : nullptr, ws + L0.k + r0 * e, ws + L0.v + r0 * e,
+                                   reinterpret_cast<float*>(ws + L0.g) + r0, reinterpret_cast<float*>(ws + L0.b) + (size_t)t0 * H,
+                                   k == 0 ? (S0_host ? reinterpret_cast<float*>(ws + L0.s0) : nullptr) : state,
+                                   o_host ? ws + L0.o + r0 * e : nullptr, state, nullptr, nullptr, 1, t1 - t0, H, dk, dv,
+                                   chunk, scale, dt, ws + L0.inner, workspace_bytes - L0.inner, st);
+            if (o_host) {
+                KDA_PIPE_TRY(new_event(&out_ready));
+                KDA_PIPE_TRY(cudaEventRecord(out_ready, st));
+                KDA_PIPE_TRY(cudaStreamWaitEvent(c_out, out_ready, 0));
+                KDA_PIPE_TRY(cudaMemcpyAsync((char*)o_host + r0 * e, ws + L0.o + r0 * e, rn * e, cudaMemcpyDeviceToHost, c_out));
+            }
+        }
+        if (o_host) {   // the caller's stream completes only after the last copy-out
+            KDA_PIPE_TRY(new_event(&join));
+            KDA_PIPE_TRY(cudaEventRecord(join, c_out));
+            KDA_PIPE_TRY(cudaStreamWaitEvent(st, join, 0));
+        }
+        if (S_T_host) KDA_PIPE_TRY(cudaMemcpyAsync(S_T_host, state, sb, cudaMemcpyDeviceToHost, st));
+#undef KDA_PIPE_TRY
+        for (cudaEvent_t ev : evs) cudaEventDestroy(ev);   // released once the work that uses them is done
+        return rc;
+    }
+
     if (q_host && td) KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.q, q_host, td * e, cudaMemcpyHostToDevice, st));
     if (td) {
         KDA_CUDA_TRY(cudaMemcpyAsync(ws + L0.k, k_host, td * e, cudaMemcpyHostToDevice, st));

@@ -329,6 +329,32 @@ def test_host_buffer_entry_points(oracle_mod):
     assert torch.equal(o2, o1.cpu()) and torch.equal(S1, S2)
 
 
+def test_host_buffer_pipelined_long_sequence(oracle_mod):
+    """One long sequence through the host-buffer entry point (copies pipelined over segments of the
+    sequence on helper streams): same bits as the device-pointer call, twice in a row."""
+    T, H = 2100, 2
+    d = inputs.chunk_inputs([T], H=H, dtype=torch.bfloat16, seed=44, s0_std=0.02)
+    o_dev, S_dev = run_chunk(d)
+    pin = {n: (t.pin_memory() if isinstance(t, torch.Tensor) else t) for n, t in d.items()}
+    nbytes = K.kda_chunk_fwd_host_workspace_bytes(T, 1, H)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda:0")
+    for _ in range(2):
+        o_h = torch.zeros_like(pin["v"]).pin_memory()
+        S_h = torch.zeros((1, H, 128, 128), dtype=torch.float32).pin_memory()
+        K.kda_chunk_fwd_host(pin["q"], pin["k"], pin["v"], pin["log_alpha"], pin["beta"], pin["S0"],
+                             o_h, S_h, None, 1, T, H, 128, 128, 64, 1.0, K.KDA_BF16, ws)
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(o_h, o_dev.cpu()) and torch.equal(S_h, S_dev.cpu())
+    # state only, no S0
+    S_h = torch.zeros((1, H, 128, 128), dtype=torch.float32).pin_memory()
+    K.kda_chunk_fwd_host(None, pin["k"], pin["v"], pin["log_alpha"], pin["beta"], None, None, S_h,
+                         None, 1, T, H, 128, 128, 64, 1.0, K.KDA_BF16, ws)
+    torch.cuda.current_stream().synchronize()
+    d2 = dict(d); d2["S0"] = None
+    _, S_ref = run_chunk(d2, want_o=False)
+    assert torch.equal(S_h, S_ref.cpu())
+
+
 def test_status_word_clean(oracle_mod):
     d = inputs.chunk_inputs([128], H=2, dtype=torch.bfloat16, seed=34)
     g = {n: (t.cuda() if isinstance(t, torch.Tensor) else t) for n, t in d.items()}
