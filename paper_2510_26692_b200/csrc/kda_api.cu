@@ -4,6 +4,7 @@
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -24,6 +25,30 @@ kda_status_t fail(kda_status_t code, const char* fmt, ...)
     return code;
 }
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// ---- per-device state -------------------------------------------------------------------------------
+namespace {
+std::mutex g_dev_mu;
+DeviceState g_dev[kMaxDevices];
+}  // namespace
+DeviceState* device_slot(int ordinal)
+{
+    return (ordinal >= 0 && ordinal < kMaxDevices) ? &g_dev[ordinal] : nullptr;
+}
+DeviceLock::DeviceLock() : st(nullptr), rc(KDA_OK)
+{
+    g_dev_mu.lock();
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) {
+        rc = fail(KDA_ERR_CUDA, "cudaGetDevice failed: %s", cudaGetErrorString(e));
+        return;
+    }
+    st = device_slot(dev);
+    if (!st) rc = fail(KDA_ERR_UNSUPPORTED, "device ordinal %d is outside the supported range 0..%d", dev,
+                       kMaxDevices - 1);
+}
+DeviceLock::~DeviceLock() { g_dev_mu.unlock(); }
 
 // ---- per-kernel event timing ------------------------------------------------------------------------
 namespace {
@@ -93,6 +118,32 @@ int64_t max_chunks(int64_t total_tokens, int n_seqs)
     return (total_tokens + kC - 1) / kC + n_seqs;
 }
 
+// ---- fused bf16 path: workspace = header | flag words | round table | ring of tiles ---------------------
+constexpr int kSlotCap = 64;      // upper bound of concurrently running (sequence, head) chains
+constexpr int kRingMax = 8;       // tiles per chain the engines may run ahead
+constexpr size_t kFlagBytes = (size_t)kSlotCap * kRingMax * 8 + (size_t)kSlotCap * 4 * 8;
+struct FusedLayout {
+    size_t off_ready, off_consumed, off_table, off_ring;
+};
+FusedLayout fused_layout(int64_t J)
+{
+    FusedLayout L;
+    L.off_ready = sizeof(WsHeader);
+    L.off_consumed = L.off_ready + (size_t)kSlotCap * kRingMax * 8;
+    L.off_table = L.off_ready + kFlagBytes;
+    L.off_ring = L.off_table + align_up((size_t)(J + 1) * sizeof(uint32_t));
+    return L;
+}
+std::atomic<uint32_t> g_epoch{0};
+bool two_kernel_path()
+{
+    static const bool v = [] {
+        const char* e = getenv("KDA_TWO_KERNEL");
+        return e && e[0] == '1';
+    }();
+    return v;
+}
+
 }  // namespace
 }  // namespace kda
 
@@ -108,16 +159,26 @@ size_t kda_chunk_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H
                                          int chunk, kda_dtype_t dt)
 {
     if (!shape_ok(dk, dv, chunk, dt) || total_tokens < 0 || n_seqs < 0 || H <= 0) return 0;
-    return ws_layout(n_seqs, H).fixed + align_up((size_t)H * tile_bytes(dt));
+    const size_t two_pass = ws_layout(n_seqs, H).fixed + align_up((size_t)H * tile_bytes(dt));
+    if (dt != KDA_BF16) return two_pass;
+    const size_t fused = fused_layout((int64_t)n_seqs * H).off_ring + 2 * tc_tile_bytes();
+    return fused > two_pass ? fused : two_pass;
 }
 
 size_t kda_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
                                      int chunk, kda_dtype_t dt)
 {
     if (!shape_ok(dk, dv, chunk, dt) || total_tokens < 0 || n_seqs < 0 || H <= 0) return 0;
+    const size_t lo = kda_chunk_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt);
+    if (dt == KDA_BF16 && !two_kernel_path()) {
+        // the fused kernel keeps at most kRingMax tiles per running chain in flight
+        const int64_t J = (int64_t)n_seqs * H;
+        const size_t want = fused_layout(J).off_ring +
+                            (size_t)(J < kSlotCap ? J : kSlotCap) * kRingMax * tc_tile_bytes();
+        return want < lo ? lo : want;
+    }
     const size_t fixed = ws_layout(n_seqs, H).fixed;
     size_t want = fixed + align_up((size_t)max_chunks(total_tokens, n_seqs) * H * tile_bytes(dt));
-    const size_t lo = kda_chunk_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt);
     if (want > kWorkspaceCap) want = kWorkspaceCap;
     return want < lo ? lo : want;
 }
@@ -179,6 +240,83 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
     if (total_chunks > 0x7fffffff)
         return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: too many chunks");
 
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (dt == KDA_BF16 && !two_kernel_path()) {
+        // ---- one fused cooperative kernel ----
+        const int64_t J = (int64_t)n_seqs * H;
+        const FusedLayout FL = fused_layout(J);
+        const size_t tbf = tc_tile_bytes();
+        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) ||
+            workspace_bytes < FL.off_ring + 2 * tbf)
+            return fail(KDA_ERR_WORKSPACE, "kda_chunk_fwd: workspace must be 256-byte aligned and at "
+                        "least %zu bytes (got %zu)", FL.off_ring + 2 * tbf, workspace_bytes);
+        if (J > 0x3fffffff) return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: n_seqs*H too large");
+        char* wsb = static_cast<char*>(workspace);
+        WsHeader* hdrf = reinterpret_cast<WsHeader*>(wsb);
+        if (!o && !S_T) {   // nothing observable to produce: only leave a clean status word
+            KDA_CUDA_TRY(cudaMemsetAsync(hdrf, 0, sizeof(WsHeader), st));
+            return KDA_OK;
+        }
+        int n_sm = 0;
+        {
+            DeviceLock lk;
+            if (!lk.st) return lk.rc;
+            if (lk.st->n_sm == 0) {
+                int dev = 0;
+                KDA_CUDA_TRY(cudaGetDevice(&dev));
+                KDA_CUDA_TRY(cudaDeviceGetAttribute(&lk.st->n_sm, cudaDevAttrMultiProcessorCount, dev));
+            }
+            n_sm = lk.st->n_sm;
+        }
+        const int64_t avail = (int64_t)((workspace_bytes - FL.off_ring) / tbf);
+        int Qmax = fused_max_slots(n_sm);
+        if (Qmax > kSlotCap) Qmax = kSlotCap;
+        if (Qmax < 1) return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: the device has too few SMs");
+        // whole sequences per round when the heads of one fit, so that the chains of a round have
+        // equal lengths
+        int64_t Q = (H <= Qmax) ? (int64_t)H * (Qmax / H) : Qmax;
+        if (Q > J) Q = J;
+        if (Q * 2 > avail) Q = avail / 2;
+        int64_t R = avail / Q;
+        if (R > kRingMax) R = kRingMax;
+        const int64_t n_rounds = (J + Q - 1) / Q;
+        uint64_t n_prod = 0;
+        for (int64_t r = 0; r < n_rounds; ++r) {
+            const int64_t j0 = r * Q, j1 = (j0 + Q < J ? j0 + Q : J) - 1;
+            int64_t maxlen = 0;
+            for (int64_t n = j0 / H; n <= j1 / H; ++n) {
+                const int64_t len = chunk_cu[n + 1] - chunk_cu[n];
+                maxlen = len > maxlen ? len : maxlen;
+            }
+            n_prod += (uint64_t)maxlen * (uint64_t)(j1 - j0 + 1);
+        }
+        if (n_prod > 0x7fffffffull)
+            return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: too many (chunk, head) tiles in one call");
+        FusedArgs f;
+        f.a.q = q; f.a.k = k; f.a.v = v; f.a.log_alpha = log_alpha; f.a.beta = beta;
+        f.a.S_in = S0; f.a.S_out = S_T; f.a.o = o;
+        f.a.cu_seqlens = cu_seqlens_dev; f.a.chunk_cu = nullptr;
+        f.a.n_seqs = n_seqs; f.a.H = H; f.a.total_tokens = total_tokens; f.a.seq_len = seq_len;
+        f.a.chunks_per_seq = chunks_per_seq; f.a.g0 = 0; f.a.g1 = total_chunks; f.a.scale = scale;
+        f.ring = wsb + FL.off_ring;
+        f.ready = reinterpret_cast<unsigned long long*>(wsb + FL.off_ready);
+        f.consumed = reinterpret_cast<unsigned long long*>(wsb + FL.off_consumed);
+        f.round_base = cu_seqlens_dev ? reinterpret_cast<const uint32_t*>(wsb + FL.off_table) : nullptr;
+        f.hdr = hdrf;
+        f.Q = (int)Q; f.R = (int)R; f.J = (int)J; f.n_rounds = (int)n_rounds;
+        f.n_prod = (uint32_t)n_prod;
+        uint32_t ep = g_epoch.fetch_add(1, std::memory_order_relaxed) + 1;
+        if (ep == 0) ep = g_epoch.fetch_add(1, std::memory_order_relaxed) + 1;
+        f.epoch = ep;
+        f.n_chain_cta = (int)(4 * Q);
+        kda_status_t rcf = KDA_OK;
+        if (cu_seqlens_dev)
+            rcf = launch_fused_prep(hdrf, cu_seqlens_dev, reinterpret_cast<uint32_t*>(wsb + FL.off_table),
+                                    n_seqs, H, (int)Q, (int)n_rounds, st);
+        if (rcf != KDA_OK) return rcf;
+        return launch_fused_tc(f, q != nullptr && o != nullptr, cu_seqlens_dev == nullptr, st);
+    }
+
     const WsLayout L = ws_layout(n_seqs, H);
     const size_t tb = tile_bytes(dt);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) ||
@@ -189,7 +327,6 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
     int64_t cap = (int64_t)((workspace_bytes - L.fixed) / ((size_t)H * tb));
     if (cap > 0x7fffffff) cap = 0x7fffffff;
 
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
     int32_t* chunk_cu_dev = reinterpret_cast<int32_t*>(ws + L.off_table);
     // The prologue kernel clears the status word and builds the chunk table of a packed batch.  An

@@ -24,7 +24,7 @@ void count_launch(int n = 1);
 
 // Optional per-kernel timing (kda_profile_*): when enabled, every launch site is bracketed by a pair
 // of CUDA events on the launching stream.  A no-op when disabled.
-enum ProfKind { PROF_PREP = 0, PROF_INTRA = 1, PROF_INTER = 2, PROF_DECODE = 3, PROF_KINDS = 8 };
+enum ProfKind { PROF_PREP = 0, PROF_INTRA = 1, PROF_INTER = 2, PROF_DECODE = 3, PROF_FUSED = 4, PROF_KINDS = 8 };
 struct ProfScope {
     ProfScope(int kind, cudaStream_t st);
     ~ProfScope();
@@ -38,7 +38,9 @@ struct ProfScope {
 struct WsHeader {
     int status;       // 0 = ok, otherwise a kda_status_t
     int where;        // implementation-defined location code of the first failure
-    int pad[62];
+    unsigned int abort_epoch;   // call id of a fused-kernel call that gave up (its waiters return at once)
+    int flags;        // bit 0: a decay factor left the supported range in some chunk (see kda.h)
+    int pad[60];
 };
 static_assert(sizeof(WsHeader) == 256, "header is one 256-byte block");
 
@@ -61,6 +63,28 @@ struct ChunkArgs {
     int64_t chunks_per_seq;   // equal-length case
     int64_t g0, g1;           // global chunk range of this pass
     float scale;
+};
+
+// Work description of the fused bf16 chunk-forward kernel (one cooperative launch per call).
+//
+// Jobs are (sequence, head) pairs in natural order j = n * H + h.  Q of them run at a time ("round"
+// r covers jobs [r Q, (r + 1) Q)); slot q of a round is served by the chain roles of CTAs
+// 4 q .. 4 q + 3 (one 32-column slice of the state each).  The intra-chunk engines of all CTAs
+// produce the tiles of a round chunk by chunk (production index = base_r + c * Q_r + q) into a ring
+// of R tiles per slot; `ready` holds (epoch << 32 | production index + 1) per ring position and
+// `consumed` (epoch << 32 | number of production indices the slice has finished with) per chain
+// role, so nothing has to be cleared between calls.
+struct FusedArgs {
+    ChunkArgs a;                     // g0, g1 unused
+    char* ring;                      // [Q][R] tiles
+    unsigned long long* ready;       // [Q * R]
+    unsigned long long* consumed;    // [Q * 4]
+    const uint32_t* round_base;      // packed batches: [n_rounds + 1] production index base per round; else nullptr
+    WsHeader* hdr;
+    int Q, R, J, n_rounds;
+    uint32_t n_prod;                 // production indices in total (equal lengths; packed: round_base[n_rounds])
+    uint32_t epoch;                  // call id, never 0
+    int n_chain_cta;                 // 4 * Q
 };
 
 // ---- dtype helpers ------------------------------------------------------------------------------
@@ -167,6 +191,35 @@ kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, 
 size_t tc_tile_bytes();
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
                              WsHeader* hdr, bool clear_status, cudaStream_t st);
+
+// fused bf16 path: workspace bytes besides the ring (flags and round table), and the launcher
+size_t fused_fixed_bytes(int n_seqs, int H);
+int fused_max_slots(int n_sm);
+kda_status_t launch_fused_tc(FusedArgs f, bool has_q, bool clear_status, cudaStream_t st);
+kda_status_t launch_fused_prep(WsHeader* hdr, const int32_t* cu_seqlens, uint32_t* round_base, int n_seqs,
+                               int H, int Q, int n_rounds, cudaStream_t st);
+
+// ---- per-device library state ---------------------------------------------------------------------
+// Everything the library caches about a device (SM count, which kernels already carry their
+// dynamic-shared-memory attribute, helper streams) lives in one slot per device ordinal, created
+// on first use under a mutex.
+constexpr int kMaxDevices = 64;
+constexpr int kAttrSlots = 16;
+struct DeviceState {
+    int n_sm = 0;
+    bool attr_done[kAttrSlots] = {};
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+};
+// Locks the table and returns the slot of the calling thread's current device (nullptr + error set
+// on failure); the lock is released by ~DeviceLock.
+struct DeviceLock {
+    DeviceLock();
+    ~DeviceLock();
+    DeviceState* st;      // nullptr if the device could not be identified
+    kda_status_t rc;
+};
+// The slot table itself, without any CUDA call (unit-testable on a machine without a GPU).
+DeviceState* device_slot(int ordinal);
 
 kda_status_t launch_wait_selftest(WsHeader* hdr, uint64_t limit_ns, cudaStream_t st);
 
