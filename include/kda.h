@@ -132,6 +132,20 @@ kda_status_t kda_chunk_fwd_static(const void *q, const void *k, const void *v,
                                   void *cuda_stream);
 
 /*
+ * Chooses how kda_chunk_fwd schedules a bf16 call (process-wide; no counterpart in the paper).
+ *   0  automatic (default): when the workspace has room for every (chunk, head) tile of the call,
+ *      the intra-chunk stage (Section 3.1: gates, UT transform) runs as one kernel and the
+ *      inter-chunk stage (state and output equations) as a second one; with a smaller workspace
+ *      one fused cooperative kernel runs both stages at once and hands the tiles over through a
+ *      ring of a few tiles per (sequence, head) that stays in the L2 cache.
+ *   1  always the two kernels (a small workspace then makes the call walk the chunks in passes)
+ *   2  always the fused kernel
+ * All three give the same results up to the rounding of the chunk states' bf16 operand copies
+ * (identical arithmetic per tile).  Returns KDA_ERR_INVALID_ARG for any other mode.
+ */
+kda_status_t kda_set_chunk_path(int mode);
+
+/*
  * Recurrent decode step (Eq. 1 for one token per sequence).
  *
  *   q, k, log_alpha  [n_seqs,H,dk]   v, o  [n_seqs,H,dv]   beta  [n_seqs,H]

@@ -82,6 +82,8 @@ def load():
     lib.kda_last_error.restype = ctypes.c_char_p
     lib.kda_launch_count.restype = ctypes.c_uint64
     lib.kda_version.restype = ctypes.c_char_p
+    lib.kda_set_chunk_path.restype = i32
+    lib.kda_set_chunk_path.argtypes = [i32]
     _lib = lib
     return lib
 
@@ -96,6 +98,11 @@ def kda_launch_count() -> int:
 
 def kda_version() -> str:
     return load().kda_version().decode()
+
+
+def kda_set_chunk_path(mode: int) -> None:
+    """0 = automatic, 1 = always the two kernels, 2 = always the fused kernel (see kda.h)."""
+    _check(load().kda_set_chunk_path(int(mode)))
 
 
 def _check(rc: int):

@@ -120,7 +120,7 @@ int64_t max_chunks(int64_t total_tokens, int n_seqs)
 
 // ---- fused bf16 path: workspace = header | flag words | round table | ring of tiles ---------------------
 constexpr int kSlotCap = 64;      // upper bound of concurrently running (sequence, head) chains
-constexpr int kRingMax = 8;       // tiles per chain the engines may run ahead
+constexpr int kRingMax = 16;      // tiles per chain the engines may run ahead
 constexpr size_t kFlagBytes = (size_t)kSlotCap * kRingMax * 8 + (size_t)kSlotCap * 4 * 8;
 struct FusedLayout {
     size_t off_ready, off_consumed, off_table, off_ring;
@@ -135,14 +135,7 @@ FusedLayout fused_layout(int64_t J)
     return L;
 }
 std::atomic<uint32_t> g_epoch{0};
-bool two_kernel_path()
-{
-    static const bool v = [] {
-        const char* e = getenv("KDA_TWO_KERNEL");
-        return e && e[0] == '1';
-    }();
-    return v;
-}
+std::atomic<int> g_chunk_path{0};   // 0 = automatic, 1 = always two kernels, 2 = always the fused kernel
 
 }  // namespace
 }  // namespace kda
@@ -154,6 +147,13 @@ extern "C" {
 const char* kda_last_error(void) { return g_err; }
 uint64_t kda_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 const char* kda_version(void) { return "kda-b200 sm_100a"; }
+
+kda_status_t kda_set_chunk_path(int mode)
+{
+    if (mode < 0 || mode > 2) return fail(KDA_ERR_INVALID_ARG, "kda_set_chunk_path: mode must be 0, 1 or 2");
+    g_chunk_path.store(mode, std::memory_order_relaxed);
+    return KDA_OK;
+}
 
 size_t kda_chunk_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
                                          int chunk, kda_dtype_t dt)
@@ -170,13 +170,6 @@ size_t kda_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, in
 {
     if (!shape_ok(dk, dv, chunk, dt) || total_tokens < 0 || n_seqs < 0 || H <= 0) return 0;
     const size_t lo = kda_chunk_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, dt);
-    if (dt == KDA_BF16 && !two_kernel_path()) {
-        // the fused kernel keeps at most kRingMax tiles per running chain in flight
-        const int64_t J = (int64_t)n_seqs * H;
-        const size_t want = fused_layout(J).off_ring +
-                            (size_t)(J < kSlotCap ? J : kSlotCap) * kRingMax * tc_tile_bytes();
-        return want < lo ? lo : want;
-    }
     const size_t fixed = ws_layout(n_seqs, H).fixed;
     size_t want = fixed + align_up((size_t)max_chunks(total_tokens, n_seqs) * H * tile_bytes(dt));
     if (want > kWorkspaceCap) want = kWorkspaceCap;
@@ -241,7 +234,19 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
         return fail(KDA_ERR_INVALID_ARG, "kda_chunk_fwd: too many chunks");
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    if (dt == KDA_BF16 && !two_kernel_path()) {
+    // bf16: two paths.  With room for every tile of the call, the intra-chunk stage runs as one
+    // kernel over all SMs followed by the inter-chunk kernel (fastest on this device).  With less
+    // room, one fused cooperative kernel hands the tiles over through a small ring that stays in L2
+    // instead of walking the chunks in several passes.
+    bool fused = false;
+    if (dt == KDA_BF16) {
+        const int mode = g_chunk_path.load(std::memory_order_relaxed);
+        const WsLayout L2p = ws_layout(n_seqs, H);
+        const bool one_pass = workspace_bytes >= L2p.fixed &&
+                              (int64_t)((workspace_bytes - L2p.fixed) / ((size_t)H * tc_tile_bytes())) >= total_chunks;
+        fused = mode == 2 || (mode == 0 && !one_pass);
+    }
+    if (fused) {
         // ---- one fused cooperative kernel ----
         const int64_t J = (int64_t)n_seqs * H;
         const FusedLayout FL = fused_layout(J);
@@ -308,7 +313,7 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
         uint32_t ep = g_epoch.fetch_add(1, std::memory_order_relaxed) + 1;
         if (ep == 0) ep = g_epoch.fetch_add(1, std::memory_order_relaxed) + 1;
         f.epoch = ep;
-        f.n_chain_cta = (int)(4 * Q);
+        f.n_chain_cta = (int)(fused_slices() * Q);
         kda_status_t rcf = KDA_OK;
         if (cu_seqlens_dev)
             rcf = launch_fused_prep(hdrf, cu_seqlens_dev, reinterpret_cast<uint32_t*>(wsb + FL.off_table),

@@ -68,8 +68,8 @@ struct ChunkArgs {
 // Work description of the fused bf16 chunk-forward kernel (one cooperative launch per call).
 //
 // Jobs are (sequence, head) pairs in natural order j = n * H + h.  Q of them run at a time ("round"
-// r covers jobs [r Q, (r + 1) Q)); slot q of a round is served by the chain roles of CTAs
-// 4 q .. 4 q + 3 (one 32-column slice of the state each).  The intra-chunk engines of all CTAs
+// r covers jobs [r Q, (r + 1) Q)); slot q of a round is served by the chain CTAs 2 q and 2 q + 1
+// (one 64-column slice of the state each); the other CTAs run two intra-chunk engines each.  The intra-chunk engines of all CTAs
 // produce the tiles of a round chunk by chunk (production index = base_r + c * Q_r + q) into a ring
 // of R tiles per slot; `ready` holds (epoch << 32 | production index + 1) per ring position and
 // `consumed` (epoch << 32 | number of production indices the slice has finished with) per chain
@@ -78,13 +78,13 @@ struct FusedArgs {
     ChunkArgs a;                     // g0, g1 unused
     char* ring;                      // [Q][R] tiles
     unsigned long long* ready;       // [Q * R]
-    unsigned long long* consumed;    // [Q * 4]
+    unsigned long long* consumed;    // [Q * fused_slices()]
     const uint32_t* round_base;      // packed batches: [n_rounds + 1] production index base per round; else nullptr
     WsHeader* hdr;
     int Q, R, J, n_rounds;
     uint32_t n_prod;                 // production indices in total (equal lengths; packed: round_base[n_rounds])
     uint32_t epoch;                  // call id, never 0
-    int n_chain_cta;                 // 4 * Q
+    int n_chain_cta;                 // chain CTAs: fused_slices() per slot
 };
 
 // ---- dtype helpers ------------------------------------------------------------------------------
@@ -195,6 +195,7 @@ kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n
 // fused bf16 path: workspace bytes besides the ring (flags and round table), and the launcher
 size_t fused_fixed_bytes(int n_seqs, int H);
 int fused_max_slots(int n_sm);
+int fused_slices();
 kda_status_t launch_fused_tc(FusedArgs f, bool has_q, bool clear_status, cudaStream_t st);
 kda_status_t launch_fused_prep(WsHeader* hdr, const int32_t* cu_seqlens, uint32_t* round_base, int n_seqs,
                                int H, int Q, int n_rounds, cudaStream_t st);

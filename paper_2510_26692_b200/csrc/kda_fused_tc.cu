@@ -77,27 +77,31 @@ constexpr uint32_t E_TD = E_A + 64 * LDT * 4;     // fp32 4 x [16][LDD]: diagona
 constexpr uint32_t E_TD_BYTES = 4096;
 constexpr uint32_t E_BETA = E_TD + E_TD_BYTES;    // 64 fp32
 constexpr uint32_t E_DESC = E_BETA + 256;         // two tile descriptors
-constexpr uint32_t E_BAR = E_DESC + 128;          // mma barrier, tma barrier, abort word, (first engine) TMEM slot
-constexpr uint32_t E_BYTES = (E_BAR + 64 + 1023) / 1024 * 1024;
+constexpr uint32_t E_BAR = E_DESC + 128;          // 8-byte words: mma barrier, K barrier, abort word, Q barrier,
+                                                  // (first engine) TMEM slot, V barrier
+constexpr uint32_t E_KS = (E_BAR + 64 + 1023) / 1024 * 1024;   // raw k of the NEXT tile [2 K-halves][64][64] bf16
+constexpr uint32_t E_BYTES = E_KS + 16384;
 static_assert(E_TD_BYTES >= 8 * 128 * 4 && E_TD_BYTES >= 4 * 16 * LDD * 4, "scan exchange and diagonal blocks fit");
 
-// ---- shared-memory map of the chain role (bytes from its 1024-aligned base) ------------------------
+// ---- shared-memory map of a chain CTA (bytes from the 1024-aligned base) -----------------------------
+constexpr int NS = 64;                             // state columns per chain CTA
+constexpr int kSlices = kD / NS;                   // chain CTAs per (sequence, head)
 constexpr int kStagesAB = 2, kStagesG = 3;
 constexpr uint32_t C_QW = 0;                       // [2 K-halves][128][64]: rows 0-63 W', 64-127 Q'
 constexpr uint32_t C_KT = 32768;                   // K': [2 dk-halves][64 tokens][64], MN-major A operand
 constexpr uint32_t C_AQ = 49152;                   // Aqk [64][64]; used as rows 64-127 of a 128-row operand
-constexpr uint32_t C_U = 57344;                    // [64 tokens][32] block of U
-constexpr uint32_t C_STAGE = 61440;
-constexpr uint32_t C_SV = kStagesAB * C_STAGE;     // [128 rows][128 B], MN-major B operands, 128-byte swizzle:
-                                                   // columns 0-31 = bf16(exp(G_m) . S) (128 dk rows),
-                                                   // columns 32-63 of rows 0-63 = V_new (64 token rows)
-constexpr uint32_t C_GV = C_SV + 16384;            // [3] x (gamma^C | exp(G_m) | exp(G_C - G_m))
+constexpr uint32_t C_U = 57344;                    // two [64 tokens][32] blocks of U
+constexpr uint32_t C_UBYTES = (NS / 32) * tc::U_BLOCK;
+constexpr uint32_t C_STAGE = C_U + C_UBYTES;
+constexpr uint32_t C_SBF = kStagesAB * C_STAGE;    // B operand of MMA1, MN-major: [128 dk rows][128 B] = bf16(exp(G_m) . S)
+constexpr uint32_t C_VN = C_SBF + 128 * 128;       // B operand of MMA2, MN-major: [64 token rows][128 B] = V_new
+constexpr uint32_t C_GV = C_VN + 64 * 128;         // [3] x (gamma^C | exp(G_m) | exp(G_C - G_m))
 constexpr uint32_t C_BAR = C_GV + kStagesG * tc::GV_BYTES;
 constexpr uint32_t C_BYTES = C_BAR + 256;
-constexpr uint32_t kSmemBytes = E_BYTES + (C_BYTES > E_BYTES ? C_BYTES : E_BYTES);
+constexpr uint32_t kSmemBytes = 2 * E_BYTES > C_BYTES ? 2 * E_BYTES : C_BYTES;
 static_assert(C_STAGE % 1024 == 0 && E_BYTES % 1024 == 0, "operand images stay 1024-byte aligned");
 static_assert(kSmemBytes <= 232448, "fits the shared memory of one SM");
-constexpr uint32_t kTmemCols = 512;                // engine: 256, second engine or chain: 256
+constexpr uint32_t kTmemCols = 512;                // two engines of 256 columns, or one chain of 384
 
 // loads that the compiler may not sink below their issue point (register prefetch of the next tile)
 __device__ __forceinline__ void ld_nc_f4(const float* p, float& a, float& b, float& c, float& d) {
@@ -220,54 +224,90 @@ struct TileDesc {
 };
 static_assert(sizeof(TileDesc) == 64, "two descriptors fit the 128 bytes reserved");
 
-// Finds the engine's next tile at or after production index i (stride: number of engines) and
-// fills the descriptor.  Returns the index to continue from.  Runs in ONE thread.
-__device__ uint32_t next_tile(const FusedArgs& f, uint32_t i, uint32_t stride, TileDesc* d)
+// Hands out production indices in increasing order to whichever engine asks next (a slow engine
+// then delays one tile, not every tile of a fixed share).  The counter lives in the workspace header
+// and carries the call id in its upper half, so a value left by an earlier call is recognised and
+// replaced by the first asker instead of having to be cleared.
+__device__ __forceinline__ uint32_t fetch_index(const FusedArgs& f)
+{
+    unsigned long long* ctr = reinterpret_cast<unsigned long long*>(&f.hdr->pad[40]);
+    for (;;) {
+        const unsigned long long v = *reinterpret_cast<volatile unsigned long long*>(ctr);
+        if ((uint32_t)(v >> 32) == f.epoch) return (uint32_t)atomicAdd(ctr, 1ull);
+        if (atomicCAS(ctr, v, tag(f.epoch, 1u)) == v) return 0u;
+    }
+}
+// Describes the tile with production index i; false if there is no tile at that index (a shorter
+// sequence of the round, or past the end).
+__device__ bool describe_tile(const FusedArgs& f, uint32_t i, TileDesc* d)
 {
     d->len = 0;
-    for (; i < f.n_prod; i += stride) {
-        int r;
-        if (f.round_base) {
-            int lo = 0, hi = f.n_rounds - 1;   // last round with base <= i
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (f.round_base[mid] <= i) lo = mid; else hi = mid - 1;
-            }
-            r = lo;
-        } else {
-            r = (int)(i / ((uint32_t)f.a.chunks_per_seq * (uint32_t)f.Q));
+    if (i >= f.n_prod) return false;
+    int r;
+    if (f.round_base) {
+        int lo = 0, hi = f.n_rounds - 1;   // last round with base <= i
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (f.round_base[mid] <= i) lo = mid; else hi = mid - 1;
         }
-        const RoundInfo R = round_info(f, r);
-        const uint32_t il = i - R.base;
-        const int c = (int)(il / (uint32_t)R.Qr), q = (int)(il - (uint32_t)c * (uint32_t)R.Qr);
-        const JobInfo J = job_info(f, r * f.Q + q);
-        if (c >= J.nch) continue;   // a shorter sequence of the round: nothing at this index
-        const int pos = q * f.R + c % f.R;
-        d->tok0 = J.tok_begin + (int64_t)c * kC;
-        const int64_t rem = J.tok_end - d->tok0;
-        d->tile = f.ring + (size_t)pos * tc::TILE_BYTES;
-        d->ready = f.ready + pos;
-        d->ready_val = tag(f.epoch, i + 1u);
-        d->consumed = f.consumed + q * 4;
-        // the ring position was last used by chunk c - R of this job, or by the slot's job of an earlier round
-        d->need = c >= f.R ? i - (uint32_t)f.R * (uint32_t)R.Qr + 1u : R.base;
-        d->h = J.h;
-        d->len = rem < kC ? (int)rem : kC;
-        return i + stride;
+        r = lo;
+    } else {
+        r = (int)(i / ((uint32_t)f.a.chunks_per_seq * (uint32_t)f.Q));
     }
-    return i;
+    const RoundInfo R = round_info(f, r);
+    const uint32_t il = i - R.base;
+    const int c = (int)(il / (uint32_t)R.Qr), q = (int)(il - (uint32_t)c * (uint32_t)R.Qr);
+    const JobInfo J = job_info(f, r * f.Q + q);
+    if (c >= J.nch) return false;
+    const int pos = q * f.R + c % f.R;
+    d->tok0 = J.tok_begin + (int64_t)c * kC;
+    const int64_t rem = J.tok_end - d->tok0;
+    d->tile = f.ring + (size_t)pos * tc::TILE_BYTES;
+    d->ready = f.ready + pos;
+    d->ready_val = tag(f.epoch, i + 1u);
+    d->consumed = f.consumed + q * kSlices;
+    // the ring position was last used by chunk c - R of this job, or by the slot's job of an earlier round
+    d->need = c >= f.R ? i - (uint32_t)f.R * (uint32_t)R.Qr + 1u : R.base;
+    d->h = J.h;
+    d->len = rem < kC ? (int)rem : kC;
+    return true;
+}
+// The scheduler thread's look-ahead state: the request for the index after next is in flight while
+// a tile is worked on, and so is a first look at the progress of the next tile's consumers; neither
+// value is touched before it is needed, so the round trips cost nothing.
+struct SchedState {
+    unsigned long long pending;             // return value of the counter request in flight
+    unsigned long long seen[kSlices];       // progress words of the next tile's consumers, read a tile early
+};
+// The engine's next tile: takes the index requested a tile ago, requests the one after it, skips
+// indices without a tile.  ONE thread.
+__device__ void next_tile(const FusedArgs& f, SchedState& ss, TileDesc* d)
+{
+    unsigned long long* ctr = reinterpret_cast<unsigned long long*>(&f.hdr->pad[40]);
+    for (;;) {
+        // (the counter carries this call's id since the engine's first request)
+        const uint32_t i = (uint32_t)(ss.pending >> 32) == f.epoch ? (uint32_t)ss.pending : 0xffffffffu;
+        if (i >= f.n_prod) { d->len = 0; return; }
+        ss.pending = atomicAdd(ctr, 1ull);
+        if (describe_tile(f, i, d)) break;
+    }
+#pragma unroll
+    for (int sl = 0; sl < kSlices; ++sl) ss.seen[sl] = d->need > 0 ? ptx::ld_acquire_gpu(d->consumed + sl) : 0ull;
 }
 // Waits (bounded) until the chain roles have finished with the previous occupant of the tile's ring
 // position.  Runs in ONE thread, at a point where its engine holds no unfinished tile and has
 // published every finished one: a producer that waited for its consumers while sitting on a tile
 // they need would deadlock.
-__device__ void wait_slot_free(const FusedArgs& f, const TileDesc& d, volatile uint32_t* abort_word)
+__device__ void wait_slot_free(const FusedArgs& f, const TileDesc& d, const SchedState& ss,
+                               volatile uint32_t* abort_word)
 {
     if (d.need == 0) return;
     uint64_t t0 = 0;
-    for (int sl = 0; sl < 4; ++sl) {
+    for (int sl = 0; sl < kSlices; ++sl) {
+        unsigned long long v = ss.seen[sl];   // the look taken a tile ago usually settles it
         for (;;) {
-            const unsigned long long v = ptx::ld_acquire_gpu(d.consumed + sl);
+            if ((uint32_t)(v >> 32) == f.epoch && (uint32_t)v >= d.need) break;
+            v = ptx::ld_acquire_gpu(d.consumed + sl);
             if ((uint32_t)(v >> 32) == f.epoch && (uint32_t)v >= d.need) break;
             if (t0 == 0) t0 = ptx::globaltimer_ns();
             if (*abort_word || call_aborted(f)) { *abort_word = 1; return; }
@@ -287,7 +327,7 @@ __device__ void wait_slot_free(const FusedArgs& f, const TileDesc& d, volatile u
 // ====================================================================================================
 template <bool kHasQ>
 __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, int bar_id, int te,
-                           uint32_t first_index, uint32_t stride, const CUtensorMap* tm_k,
+                           const CUtensorMap* tm_k,
                            const CUtensorMap* tm_q, const CUtensorMap* tm_v)
 {
     constexpr bool has_q = kHasQ;
@@ -301,7 +341,9 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
     float* sBeta = reinterpret_cast<float*>(smem + E_BETA);
     TileDesc* desc = reinterpret_cast<TileDesc*>(smem + E_DESC);
     uint64_t* mma_bar = reinterpret_cast<uint64_t*>(smem + E_BAR);
-    uint64_t* tma_bar = mma_bar + 1;
+    uint64_t* bar_k = mma_bar + 1;   // raw k has landed in the staging buffer
+    uint64_t* bar_q = mma_bar + 3;   // raw q has landed in rows 64-127 of the operand image
+    uint64_t* bar_v = mma_bar + 5;   // v has landed
     volatile uint32_t* abort_word = reinterpret_cast<volatile uint32_t*>(mma_bar + 2);
 
     const int warp = te >> 5, lane = te & 31;
@@ -322,23 +364,30 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
             }
         }
     };
-    // k, q, v by 2-D tiled TMA loads straight into the swizzled operand images; beta by small
-    // asynchronous copies
-    auto prefetch_bufs = [&](const TileDesc& D) {
-        if (te == kBulkThread) {
-            ptx::mbar_expect_tx(tma_bar, (has_q ? 3 : 2) * 16384);
-            const int x = D.h * kD, y = (int)D.tok0;
+    // k, q, v of the NEXT tile by 2-D tiled TMA loads (128-byte swizzle), each requested as soon as
+    // its destination is free: k into a staging buffer (the gating loop reads it there and writes
+    // the gated image), q straight into rows 64-127 of the operand image (gated in place), v into
+    // the B operand buffer of the second MMA group; beta by small asynchronous copies.  Run by the
+    // bulk thread (beta: by the first 64 threads).
+    auto request_k = [&](const TileDesc& D) {
+        ptx::mbar_expect_tx(bar_k, 16384);
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                ptx::tma_load_2d(smem + E_KQ + hf * E_KQ_HALF, tm_k, x + hf * 64, y, tma_bar);
-                if (has_q)
-                    ptx::tma_load_2d(smem + E_KQ + hf * E_KQ_HALF + 8192, tm_q, x + hf * 64, y, tma_bar);
-                ptx::tma_load_2d(smem + E_V + hf * E_V_BLOCK, tm_v, x + hf * 64, y, tma_bar);
-            }
-        }
-#ifdef KDA_FUSED_TIMING
-        if (te == kBulkThread) *reinterpret_cast<volatile uint64_t*>(smem + E_BAR + 48) = ptx::globaltimer_ns();
-#endif
+        for (int hf = 0; hf < 2; ++hf)
+            ptx::tma_load_2d(smem + E_KS + hf * 8192, tm_k, D.h * kD + hf * 64, (int)D.tok0, bar_k);
+    };
+    auto request_q = [&](const TileDesc& D) {
+        ptx::mbar_expect_tx(bar_q, 16384);
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf)
+            ptx::tma_load_2d(smem + E_KQ + hf * E_KQ_HALF + 8192, tm_q, D.h * kD + hf * 64, (int)D.tok0, bar_q);
+    };
+    auto request_v = [&](const TileDesc& D) {
+        ptx::mbar_expect_tx(bar_v, 16384);
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf)
+            ptx::tma_load_2d(smem + E_V + hf * E_V_BLOCK, tm_v, D.h * kD + hf * 64, (int)D.tok0, bar_v);
+    };
+    auto request_beta = [&](const TileDesc& D) {
         if (te < kC) {
             const bool ok = te < D.len;
             ptx::cp_async4(sBeta + te, a.beta + (D.tok0 + (ok ? te : 0)) * a.H + D.h, ok ? 4u : 0u);
@@ -346,21 +395,31 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         ptx::cp_async_commit();
     };
 
-    bool timed_out = false, out_of_range = false, load_pending = false;
+    bool timed_out = false, out_of_range = false;
+    bool pend_k = false, pend_q = false, pend_v = false;   // (thread 0) requests not yet waited for
     uint32_t tma_parity = 0;
-    uint32_t next_index = first_index;
+    SchedState ss = {};   // (scheduler thread)
     int cur = 0;
     unsigned long long* pending_ready = nullptr;   // bulk thread: flag of the tile whose stores are in flight
     unsigned long long pending_val = 0;
 
-    if (te == kSchedThread) next_index = next_tile(f, next_index, stride, &desc[0]);
+    if (te == kSchedThread) {
+        ss.pending = tag(f.epoch, fetch_index(f));
+        next_tile(f, ss, &desc[0]);
+    }
     ebar();
     if (desc[0].len > 0 && !*abort_word) {
         prefetch_regs(desc[0]);
-        prefetch_bufs(desc[0]);
-        load_pending = true;
+        if (te == kBulkThread) {
+            request_k(desc[0]);
+            if (has_q) request_q(desc[0]);
+            request_v(desc[0]);
+        }
+        request_beta(desc[0]);
+        pend_k = pend_v = true;
+        pend_q = has_q;
     }
-    KT_DECL(13);
+    KT_DECL(10);
     while (true) {
         const TileDesc D = desc[cur];
         if (D.len == 0 || *abort_word) break;
@@ -377,25 +436,26 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         *reinterpret_cast<float4*>(sTot + warp * kD + d0) =
             make_float4(G[kRPT - 1][0], G[kRPT - 1][1], G[kRPT - 1][2], G[kRPT - 1][3]);
         if (te == kBulkThread && pending_ready) {
-            // the previous tile is complete in global memory: hand it to the chain roles (this also
-            // means its W' / U staging has been read out: the buffers are written again below)
+            // The previous tile is complete in global memory: hand it to the chain roles.  (This also
+            // means its W' / U staging has been read out: the buffers are written again below.)  It
+            // has to happen before this engine may wait for a ring position: a producer that waits
+            // for its consumers while holding back a tile they need would deadlock.
             ptx::bulk_wait_all0();
             ptx::fence_proxy_async_all();
-            __threadfence();
             ptx::st_release_gpu(pending_ready, pending_val);
             pending_ready = nullptr;
         }
-        if (te == kSchedThread) wait_slot_free(f, D, abort_word);   // (the previous tile is being published meanwhile)
+#ifdef KDA_FUSED_TIMING
+        const uint64_t ts0_ = te == kSchedThread ? ptx::globaltimer_ns() : 0;
+#endif
+        if (te == kSchedThread) wait_slot_free(f, D, ss, abort_word);
+#ifdef KDA_FUSED_TIMING
+        if (te == kSchedThread) atomicAdd(&f.hdr->pad[11], (int)((ptx::globaltimer_ns() - ts0_) >> 4));
+#endif
         ptx::cp_async_wait_all();             // beta
         ebar();
         KT_MARK(te == 0, 1);   // scan + publish + slot wait
         if (*abort_word) break;
-#ifdef KDA_FUSED_TIMING
-        if (te == 0) {
-            const uint64_t now_ = ptx::globaltimer_ns();
-            kt_acc_[11] += (uint32_t)(now_ - kt_last_);   // abort check
-        }
-#endif
         float base[4] = {0.f, 0.f, 0.f, 0.f}, gref[4], glast[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int r2 = 0; r2 < kNW; ++r2) {
@@ -413,12 +473,6 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         for (int e = 0; e < 4; ++e) gref[e] = 0.5f * glast[e];
         // the true scales exp(G_C), exp(G_m) and exp(G_C - G_m) go to the tile as fp32 vectors; the
         // chain applies them to the state in fp32
-#ifdef KDA_FUSED_TIMING
-        if (te == 0) {
-            const uint64_t now_ = ptx::globaltimer_ns();
-            kt_acc_[12] += (uint32_t)(now_ - kt_last_);   // prefix part
-        }
-#endif
         if (warp == 0) {
             *reinterpret_cast<float4*>(tile + tc::OFF_GV + d0 * 4) =
                 make_float4(ex2(glast[0]), ex2(glast[1]), ex2(glast[2]), ex2(glast[3]));
@@ -434,28 +488,12 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
 #ifdef KDA_FUSED_TIMING
         if (te == 0) {
             const uint64_t now_ = ptx::globaltimer_ns();
-            (void)now_;
         }
 #endif
-#ifdef KDA_FUSED_TIMING
-        if (te == 0) {
-            const uint64_t now_ = ptx::globaltimer_ns();
-        }
-#endif
-        if (!ptx::mbar_wait(tma_bar, tma_parity, kWaitLimitNs)) timed_out = true;   // k, q, v have landed
-        tma_parity ^= 1;
-        load_pending = false;
-#ifdef KDA_FUSED_TIMING
-        if (te == 0) kt_acc_[10] = kt_acc_[10] + (uint32_t)(ptx::globaltimer_ns() - *reinterpret_cast<volatile uint64_t*>(smem + E_BAR + 48));
-#endif
+        if (!ptx::mbar_wait(bar_k, tma_parity, kWaitLimitNs)) timed_out = true;   // raw k, q have landed
+        if (has_q && !ptx::mbar_wait(bar_q, tma_parity, kWaitLimitNs)) timed_out = true;
+        pend_k = pend_q = false;
         KT_MARK(te == 0, 2);   // prefix + TMA wait
-        if (D.len < kC) {   // short last chunk: rows past the end hold other tokens' v; zero them
-            for (int idx = te; idx < (kC - D.len) * 16; idx += kEngThreads) {
-                const int j = D.len + (idx >> 4), c16 = idx & 15;
-                *reinterpret_cast<uint4*>(smem + E_V + (c16 >> 3) * E_V_BLOCK + j * 128 +
-                                          (((c16 & 7) ^ (j & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-            }
-        }
         // ---- gated operands ---------------------------------------------------------------------------
         {
             const int hf = c4 >> 4;                       // K-half (channels 0-63 / 64-127)
@@ -464,7 +502,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                 const int i = i0 + r;
                 const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
                 uint8_t* pk = smem + E_KQ + hf * E_KQ_HALF + off;
-                uint2 k2 = *reinterpret_cast<const uint2*>(pk);
+                uint2 k2 = *reinterpret_cast<const uint2*>(smem + E_KS + hf * 8192 + off);
                 uint2 q2 = make_uint2(0u, 0u);
                 if (has_q) q2 = *reinterpret_cast<const uint2*>(pk + 8192);
                 if (i >= D.len) k2 = q2 = make_uint2(0u, 0u);
@@ -515,7 +553,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                                ptx::umma_desc_sw128(b0 + (k >> 2) * E_KI_HALF + (k & 3) * 32), idesc, k > 0);
             ptx::umma_commit(mma_bar);
         }
-        if (te == kSchedThread) next_index = next_tile(f, next_index, stride, &desc[cur ^ 1]);
+        if (te == kSchedThread) next_tile(f, ss, &desc[cur ^ 1]);
         if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) timed_out = true;
         // Q' and K' have been read out of shared memory by now: Aqk goes over the Q' rows next
         if (te == kBulkThread) ptx::bulk_wait_read0();
@@ -524,7 +562,11 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         KT_MARK(te == 0, 4);   // MMA A
         const TileDesc Dn = desc[cur ^ 1];
         const bool has_next = Dn.len > 0 && !*abort_word;
-        if (has_next) prefetch_regs(Dn);   // the next tile's log alpha: its registers are free since the gating loop
+        if (has_next) {
+            prefetch_regs(Dn);   // the next tile's log alpha: its registers are free since the gating loop
+            if (te == kBulkThread) request_k(Dn);   // the staging buffer was read by the gating loop
+            pend_k = true;
+        }
         {
             const int q4 = warp & 3, c0 = (warp >> 2) * 32;
             const int Rr = q4 * 32 + lane;
@@ -623,8 +665,23 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
             block16_mma(acc, blkA(3, 2), LDT, blkA(0, 2), LDT, lane);
             block16_store(blkA(0, 3), acc, -1.f, LDT, lane);
         }
-        // K' (overwritten by the Mm image) and the Aqk staging have been read out
-        if (te == kBulkThread) ptx::bulk_wait_read0();
+        // K' (overwritten by the Mm image) and the Aqk staging have been read out: the next tile's q
+        // may land over the Aqk staging
+        if (te == kBulkThread) {
+            ptx::bulk_wait_read0();
+            if (has_next && has_q) request_q(Dn);
+        }
+        if (has_next) pend_q = has_q;
+        if (!ptx::mbar_wait(bar_v, tma_parity, kWaitLimitNs)) timed_out = true;   // v has landed
+        pend_v = false;
+        tma_parity ^= 1;
+        if (D.len < kC) {   // short last chunk: rows past the end hold other tokens' v; zero them
+            for (int idx = te; idx < (kC - D.len) * 16; idx += kEngThreads) {
+                const int j = D.len + (idx >> 4), c16 = idx & 15;
+                *reinterpret_cast<uint4*>(smem + E_V + (c16 >> 3) * E_V_BLOCK + j * 128 +
+                                          (((c16 & 7) ^ (j & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
         ebar();
         KT_MARK(te == 0, 6);   // inverse
 
@@ -674,9 +731,10 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         }
         if (!ptx::mbar_wait(mma_bar, 1, kWaitLimitNs)) timed_out = true;
         KT_MARK(te == 0, 7);   // Mm + MMA B
-        if (has_next) {   // Kg, Qg rows and V are free: the next tile's inputs may land
-            prefetch_bufs(Dn);
-            load_pending = true;
+        if (has_next) {   // V and beta are free: the next tile's may land
+            if (te == kBulkThread) request_v(Dn);
+            request_beta(Dn);
+            pend_v = true;
         }
         ptx::tc_fence_after();
         {   // The A operand held every row twice, so TMEM lanes 0-63 and 64-127 both carry rows 0-63:
@@ -729,7 +787,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
 #endif
         cur ^= 1;
     }   // tile loop
-    KT_FLUSH(te == 0, f.hdr, 0, 13);
+    KT_FLUSH(te == 0, f.hdr, 0, 10);
 
     if (timed_out) report_timeout(f, 10);
     if (out_of_range) atomicOr(&f.hdr->flags, 1);
@@ -737,26 +795,33 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         ptx::bulk_wait_all0();   // shared memory must outlive the reads of every bulk store
         if (pending_ready && !timed_out && !*abort_word) {
             ptx::fence_proxy_async_all();
-            __threadfence();
             ptx::st_release_gpu(pending_ready, pending_val);
         }
     }
     ptx::cp_async_wait_all();
     // an aborted engine may still have a TMA load in flight (requested for a tile it never started)
-    if (load_pending && te == 0) ptx::mbar_wait(tma_bar, tma_parity, kWaitLimitNs);
+    if (te == 0) {
+        // tma_parity is the parity of the current / next tile's K and Q loads; V's flips in the Mm phase
+        if (pend_k) ptx::mbar_wait(bar_k, tma_parity, kWaitLimitNs);
+        if (pend_q) ptx::mbar_wait(bar_q, tma_parity, kWaitLimitNs);
+        if (pend_v) ptx::mbar_wait(bar_v, tma_parity, kWaitLimitNs);
+    }
     ptx::tc_fence_before();
     ebar();
 }
 
 // ====================================================================================================
-// inter-chunk chain: warps 8-15 of a chain CTA (tc = 0..255), 256 TMEM columns at tmem_c
+// inter-chunk chain: a whole CTA (t = 0..511), 384 TMEM columns at tmem_c
+//   warps 0-7  compute: TMEM lane quadrant = warp & 3 (token row for V_new / O, dk row for the state),
+//              32-column half of the slice = warp >> 2
+//   warps 8-9  lane 0 of each issues MMAs;  warp 10 lane 0 requests the operand copies
 // ====================================================================================================
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
     __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&p);
 }
-// 32 fp32 values as one bf16 row (four 16-byte chunks starting at chunk `c0`) of an MN-major operand
-// image with 128-byte rows and 128-byte swizzle
+// 32 fp32 values as bf16 into row `row` (four 16-byte chunks starting at chunk `c0`) of an MN-major
+// operand image with 128-byte rows and 128-byte swizzle
 __device__ __forceinline__ void store_row32(uint8_t* img, int row, int c0, const float (&x)[32]) {
 #pragma unroll
     for (int c = 0; c < 4; ++c)
@@ -764,13 +829,13 @@ __device__ __forceinline__ void store_row32(uint8_t* img, int row, int c0, const
             make_uint4(pack2(x[8 * c], x[8 * c + 1]), pack2(x[8 * c + 2], x[8 * c + 3]),
                        pack2(x[8 * c + 4], x[8 * c + 5]), pack2(x[8 * c + 6], x[8 * c + 7]));
 }
-// sum of the two partial accumulators (32 columns each, side by side in TMEM) of one matrix
+// sum of the two partial accumulators (NS columns apart in TMEM) of one matrix, 32 columns
 __device__ __forceinline__ void tmem_ld_sum32(uint32_t taddr, float (&acc)[32]) {
 #pragma unroll
     for (int hb = 0; hb < 2; ++hb) {
         uint32_t r[16], r2[16];
         ptx::tmem_ld_32x32b_x16(taddr + hb * 16, r);
-        ptx::tmem_ld_32x32b_x16(taddr + 32 + hb * 16, r2);
+        ptx::tmem_ld_32x32b_x16(taddr + NS + hb * 16, r2);
         ptx::tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 16; ++j) acc[hb * 16 + j] = __uint_as_float(r[j]) + __uint_as_float(r2[j]);
@@ -778,9 +843,8 @@ __device__ __forceinline__ void tmem_ld_sum32(uint32_t taddr, float (&acc)[32]) 
 }
 
 template <bool kHasQ>
-__device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, int tc_, int q, int slice)
+__device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, int t, int q, int slice)
 {
-    constexpr int NS = 32;
     const ChunkArgs& a = f.a;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C_BAR);
     uint64_t* fullA = bars;                  // [2] [W';Q'] landed
@@ -792,37 +856,41 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
     uint64_t* mma1_bar = emptyG + 3;         // MMA1 of a chunk complete
     uint64_t* mma2_bar = mma1_bar + 1;       // MMA2 of a chunk complete
     uint64_t* out_bar = mma2_bar + 1;        // [2] output accumulator of a chunk complete (alternating)
-    uint64_t* sbf_ready = out_bar + 2;       // 4 warp arrivals: bf16 state copy written
-    uint64_t* vn_ready = sbf_ready + 1;      // 2 warp arrivals: V_new written
+    uint64_t* sbf_ready = out_bar + 2;       // 8 warp arrivals: bf16 state copy written
+    uint64_t* vn_ready = sbf_ready + 1;      // 4 warp arrivals: V_new written
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(vn_ready + 1);
-    uint8_t* sv = smem + C_SV;
+    uint8_t* sbf = smem + C_SBF;
+    uint8_t* vn = smem + C_VN;
 
-    const int warp = tc_ >> 5, lane = tc_ & 31;
+    const int warp = t >> 5, lane = t & 31;
     const int col0 = slice * NS;
     __nv_bfloat16* op = kHasQ ? reinterpret_cast<__nv_bfloat16*>(a.o) : nullptr;
 
-    if (tc_ == 0) {
+    if (t == 0) {
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(&fullA[s], 1);
             ptx::mbar_init(&fullB[s], 1);
             ptx::mbar_init(&emptyA[s], 2);    // one commit from each MMA-issuing thread
-            ptx::mbar_init(&emptyB[s], 4);    // two commits + the two warps that read U
+            ptx::mbar_init(&emptyB[s], 6);    // two commits + the four warps that read U
             ptx::mbar_init(&out_bar[s], 1);
         }
 #pragma unroll
         for (int s = 0; s < 3; ++s) {
             ptx::mbar_init(&fullG[s], 1);
-            ptx::mbar_init(&emptyG[s], 4);    // the four compute warps
+            ptx::mbar_init(&emptyG[s], 8);    // the eight compute warps
         }
         ptx::mbar_init(mma1_bar, 2);
         ptx::mbar_init(mma2_bar, 2);
-        ptx::mbar_init(sbf_ready, 4);
-        ptx::mbar_init(vn_ready, 2);
-        *abort_flag = 0;
+        ptx::mbar_init(sbf_ready, 8);
+        ptx::mbar_init(vn_ready, 4);
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;   // s_ready
+        abort_flag[2] = 0;   // s_done
+        abort_flag[3] = 0;   // s_exit
         ptx::fence_mbar_init();
     }
-    ptx::named_bar_sync(3, 256);
+    __syncthreads();
 
     auto wait = [&](uint64_t* bar, uint32_t parity, int where) {
         if (*abort_flag) return;
@@ -830,7 +898,7 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
         const uint64_t t0 = ptx::globaltimer_ns();
         uint32_t spins = 0;
         while (!ptx::mbar_try(bar, parity)) {
-            if ((++spins & 63u) == 0) {
+            if ((++spins & 15u) == 0) {
                 if (*abort_flag) return;
                 if (call_aborted(f)) { *abort_flag = 1; return; }
                 if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
@@ -841,18 +909,89 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
             }
         }
     };
-    const uint32_t d1c = tmem_c, d3c = tmem_c + 4 * NS;   // D1 {parity 0,1} x {part 0,1}, then the D3 parts
+    // TMEM columns: D1 {parity 0,1} x {part 0,1} (NS each), then the two D3 parts
+    const uint32_t d1c = tmem_c, d3c = tmem_c + 4 * NS;
 
-    if (warp == 6) {
+    // two words the loader and the flag thread talk through (shared memory, CTA-scope ordering)
+    volatile uint32_t* s_ready = abort_flag + 1;   // chunks (running number) whose tiles are complete in the ring
+    volatile uint32_t* s_done = abort_flag + 2;    // progress value to publish for the engines
+    volatile uint32_t* s_exit = abort_flag + 3;    // the loader has finished
+    if (warp == 11) {
+        // ================= flag thread: all traffic with the flag words in global memory =================
+        // An acquire load or a release store at GPU scope costs of the order of a microsecond; done by
+        // the loader they would sit on the chain's path once per chunk.  This thread confirms tiles
+        // ahead of the loader (up to the ring depth) and publishes the loader's progress behind it.
+        if (lane == 0) {
+            unsigned long long* cw = f.consumed + q * kSlices + slice;
+            uint32_t pr = 0, published = 0;
+            int r = 0, c = 0;
+            bool jobs_left = r * f.Q + q < f.J;
+            RoundInfo R = {0, 1};
+            JobInfo J = {};
+            auto load_job = [&]() {
+                while (jobs_left) {
+                    R = round_info(f, r);
+                    J = job_info(f, r * f.Q + q);
+                    if (J.nch > 0) break;
+                    ++r;
+                    jobs_left = r * f.Q + q < f.J;
+                }
+                c = 0;
+            };
+            load_job();
+            uint64_t t0 = 0;
+            while (!*abort_flag) {
+                bool progressed = false;
+                if (jobs_left) {
+                    const int pos = q * f.R + c % f.R;
+                    const uint32_t idx = R.base + (uint32_t)c * (uint32_t)R.Qr + (uint32_t)q;
+                    if (ptx::ld_acquire_gpu(f.ready + pos) == tag(f.epoch, idx + 1u)) {
+                        ++pr;
+                        __threadfence_block();
+                        *s_ready = pr;
+                        progressed = true;
+                        if (++c == J.nch) {
+                            ++r;
+                            jobs_left = r * f.Q + q < f.J;
+                            load_job();
+                        }
+                    }
+                }
+                const uint32_t d = *s_done;
+                if (d != published) {
+                    __threadfence_block();
+                    ptx::st_release_gpu(cw, tag(f.epoch, d));
+                    published = d;
+                    progressed = true;
+                }
+                if (progressed) {
+                    t0 = 0;
+                } else {
+                    if (*s_exit && *s_done == published) break;
+                    if (t0 == 0) t0 = ptx::globaltimer_ns();
+                    if (call_aborted(f)) { *abort_flag = 1; break; }
+                    if (jobs_left && ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
+                        *abort_flag = 1;
+                        report_timeout(f, 30);
+                        break;
+                    }
+                    ptx::nanosleep(32);
+                }
+            }
+        }
+    } else if (warp == 10) {
         // ================= loader: one thread requests every piece as early as its buffer frees up =======
         if (lane == 0) {
             uint32_t p = 0;                       // running chunk number of this chain role
             uint32_t nG = 0, nA = 0, nB = 0;      // pieces requested so far
-            unsigned long long* cw = f.consumed + q * 4 + slice;
-            uint32_t prev_done = 0;               // production index + 1 of chunk p - 1
-            bool have_prev = false;
+            // production index + 1 of the last two chunks; a chunk counts as consumed (its ring
+            // position may be overwritten) once its copies have landed, which is certain when the
+            // stage it went to is free again, i.e. two chunks later.  A ring of fewer than four
+            // positions cannot afford that lag: there the landing is waited for.
+            uint32_t done1 = 0, done2 = 0;
+            const bool lazy = f.R >= 4;
             KT_DECL(6);
-            auto landed = [&](uint32_t pp) {      // every piece of chunk pp has landed: its ring position may be reused
+            auto landed = [&](uint32_t pp) {
                 wait(&fullG[pp % 3], (pp / 3) & 1u, 31);
                 wait(&fullA[pp & 1], (pp >> 1) & 1u, 32);
                 wait(&fullB[pp & 1], (pp >> 1) & 1u, 33);
@@ -860,25 +999,25 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
             for (int r = 0; r * f.Q + q < f.J && !*abort_flag; ++r) {
                 const RoundInfo R = round_info(f, r);
                 const JobInfo J = job_info(f, r * f.Q + q);
+                const uint32_t p0 = p;
                 for (int c = 0; c < J.nch && !*abort_flag; ++c, ++p) {
                     const int pos = q * f.R + c % f.R;
                     const char* tile = f.ring + (size_t)pos * tc::TILE_BYTES;
                     const uint32_t idx = R.base + (uint32_t)c * (uint32_t)R.Qr + (uint32_t)q;
                     KT_MARK(true, 0);
-                    {   // the engines have completed the tile
-                        const unsigned long long want = tag(f.epoch, idx + 1u);
+                    {   // the engines have completed the tile (confirmed by the flag thread)
                         uint64_t t0 = 0;
-                        while (ptx::ld_acquire_gpu(f.ready + pos) != want) {
+                        while (*s_ready <= p) {
                             if (t0 == 0) t0 = ptx::globaltimer_ns();
-                            if (*abort_flag || call_aborted(f)) { *abort_flag = 1; break; }
-                            if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
+                            if (*abort_flag) break;
+                            if (ptx::globaltimer_ns() - t0 > 2 * kWaitLimitNs) {   // (the flag thread gives up first)
                                 *abort_flag = 1;
-                                report_timeout(f, 30);
+                                report_timeout(f, 37);
                                 break;
                             }
-                            ptx::nanosleep(64);
                         }
                         if (*abort_flag) break;
+                        __threadfence_block();
                         ptx::fence_proxy_async_all();
                     }
                     KT_MARK(true, 1);   // tile ready
@@ -902,30 +1041,31 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                     ++nA;
                     wait(&emptyB[s2], ((p >> 1) & 1u) ^ 1u, 36);
                     if (*abort_flag) break;
-                    ptx::mbar_expect_tx(&fullB[s2], (kHasQ ? 24576u : 16384u) + tc::U_BLOCK);
+                    ptx::mbar_expect_tx(&fullB[s2], (kHasQ ? 24576u : 16384u) + C_UBYTES);
                     ptx::bulk_g2s(sb + C_KT, tile + tc::OFF_KI, kHasQ ? 24576u : 16384u, &fullB[s2]);
-                    ptx::bulk_g2s(sb + C_U, tile + tc::OFF_U + (size_t)slice * tc::U_BLOCK, tc::U_BLOCK, &fullB[s2]);
+                    ptx::bulk_g2s(sb + C_U, tile + tc::OFF_U + (size_t)slice * C_UBYTES, C_UBYTES, &fullB[s2]);
                     ++nB;
                     KT_MARK(true, 2);   // buffers free + requests
-                    if (have_prev) {
+                    if (lazy) {
+                        // stage s2 was free: the chunk that used it two steps ago (if of this job) has landed
+                        if (p >= p0 + 2) *s_done = done2;
+                    } else if (p > p0) {
                         landed(p - 1);
-                        if (!*abort_flag) ptx::st_release_gpu(cw, tag(f.epoch, prev_done));
+                        if (!*abort_flag) *s_done = done1;
                     }
-                    prev_done = idx + 1u;
-                    have_prev = true;
-                    KT_MARK(true, 3);   // previous chunk landed
+                    done2 = done1;
+                    done1 = idx + 1u;
+                    KT_MARK(true, 3);   // progress handed to the flag thread
                 }
                 if (*abort_flag) break;
-                // the job is over for this slice: everything of this round counts as consumed
-                if (have_prev) {
-                    landed(p - 1);
-                    have_prev = false;
-                }
-                if (!*abort_flag) {
-                    const uint32_t nb = (r + 1 < f.n_rounds) ? round_info(f, r + 1).base : f.n_prod;
-                    ptx::st_release_gpu(cw, tag(f.epoch, nb));
-                }
+                // the job is over for this slice: once its last copies have landed, everything of this
+                // round counts as consumed
+                if (p > p0) landed(p - 1);
+                if (p > p0 + 1) landed(p - 2);
+                if (!*abort_flag) *s_done = (r + 1 < f.n_rounds) ? round_info(f, r + 1).base : f.n_prod;
             }
+            __threadfence_block();
+            *s_exit = 1;
             KT_FLUSH(true, f.hdr, 24, 4);
             if (*abort_flag) {
                 // drain: the copies already requested must land before the shared memory goes away
@@ -938,17 +1078,17 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                     ptx::mbar_wait(&fullB[pp & 1], (pp >> 1) & 1u, kWaitLimitNs / 8);
             }
         }
-    } else if (warp >= 4 && warp < 6) {
+    } else if (warp == 8 || warp == 9) {
         // ================= control warps: lane 0 of each issues MMAs =================
         // Issuing one tcgen05.mma costs the issuing thread several tens of cycles whatever the tile
-        // size, and both products on the sequential chain are tiny, so each is split along its
+        // size, and both products on the sequential chain are small, so each is split along its
         // summation index between the two control threads, into one accumulator each; the
-        // accumulators are added when they are read back.  Warp 4's thread also issues the output
+        // accumulators are added when they are read back.  The first thread also issues the output
         // product.
-        const int half = warp - 4;
+        const int half = warp - 8;
         if (lane == 0) {
             const uint32_t idesc = ptx::umma_idesc_bf16(128, NS) | ptx::kIdescBMajorMN;
-            const uint32_t sbf_a = ptx::smem_u32(sv), vn_a = sbf_a + 64;   // V_new: columns 32-63 of the same rows
+            const uint32_t sbf_a = ptx::smem_u32(sbf), vn_a = ptx::smem_u32(vn);
             uint32_t g = 0, last_out = 0;
             bool any_out = false;
             KT_DECL(8);
@@ -1015,21 +1155,22 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
             if (half == 0 && any_out) wait(&out_bar[last_out & 1], (last_out >> 1) & 1u, 7);
             else if (g > 0) wait(&emptyB[(g - 1) & 1], ((g - 1) >> 1) & 1u, 8);
         }
-    } else if (warp < 4) {
-        // ================= compute warps (TMEM lane quadrant = warp) =================
-        const int tid = tc_;   // 0..127: token row for V_new / O, dk row for the state
-        const uint32_t tmem_lane = ((uint32_t)(warp * 32) << 16);
+    } else if (warp < 8) {
+        // ================= compute warps =================
+        const int quad = warp & 3, ch = warp >> 2;       // TMEM lane quadrant, 32-column half of the slice
+        const int tid = quad * 32 + lane;                // 0..127: token row for V_new / O, dk row for the state
+        const uint32_t tmem_lane = ((uint32_t)(quad * 32) << 16) + (uint32_t)ch * 32;
         auto warp_arrive = [&](uint64_t* bar) {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar);
         };
-        float S[NS];
+        float S[32];
         uint32_t g = 0;
         for (int r = 0; r * f.Q + q < f.J; ++r) {
             const JobInfo J = job_info(f, r * f.Q + q);
-            const size_t sbase = ((size_t)J.n * a.H + J.h) * (size_t)(kD * kD) + (size_t)tid * kD + col0;
+            const size_t sbase = ((size_t)J.n * a.H + J.h) * (size_t)(kD * kD) + (size_t)tid * kD + col0 + ch * 32;
 #pragma unroll
-            for (int j = 0; j < NS; j += 4) {
+            for (int j = 0; j < 32; j += 4) {
                 float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (a.S_in) x = *reinterpret_cast<const float4*>(a.S_in + sbase + j);
                 S[j] = x.x; S[j + 1] = x.y; S[j + 2] = x.z; S[j + 3] = x.w;
@@ -1039,10 +1180,10 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                 return reinterpret_cast<const float*>(smem + C_GV + (gg % 3) * tc::GV_BYTES + 512)[tid];
             };
             auto store_scaled = [&](float cgn) {
-                float z[NS];
+                float z[32];
 #pragma unroll
-                for (int j = 0; j < NS; ++j) z[j] = cgn * S[j];
-                store_row32(sv, tid, 0, z);
+                for (int j = 0; j < 32; ++j) z[j] = cgn * S[j];
+                store_row32(sbf, tid, ch * 4, z);
             };
             if (J.nch > 0) {
                 store_scaled(ref_scale_of(g));
@@ -1053,21 +1194,21 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                 const uint32_t s2 = g & 1, par = g & 1u;
                 const uint8_t* sb = smem + s2 * C_STAGE;
                 const uint32_t d1 = d1c + tmem_lane + (uint32_t)(g & 1) * 2 * NS;
-                if (warp < 2) {   // a6: V_new = U - W S  (token row = tid)
+                if (quad < 2) {   // a6: V_new = U - W S  (token row = tid)
                     wait(&fullB[s2], (g >> 1) & 1u, 1);
                     uint4 uq[4];   // this token's 32 values of U
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc)
-                        uq[cc] = *reinterpret_cast<const uint4*>(sb + C_U + tc::u_off(tid, cc));
+                        uq[cc] = *reinterpret_cast<const uint4*>(sb + C_U + ch * tc::U_BLOCK + tc::u_off(tid, cc));
                     warp_arrive(&emptyB[s2]);
                     const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
                     wait(mma1_bar, par, 2);
                     ptx::tc_fence_after();
-                    float x[NS];
+                    float x[32];
                     tmem_ld_sum32(d1, x);
 #pragma unroll
-                    for (int j = 0; j < NS; ++j) x[j] = __bfloat162float(U[j]) - x[j];
-                    store_row32(sv, tid, 4, x);
+                    for (int j = 0; j < 32; ++j) x[j] = __bfloat162float(U[j]) - x[j];
+                    store_row32(vn, tid, ch * 4, x);
                     ptx::fence_async_smem();
                     ptx::tc_fence_before();
                     warp_arrive(vn_ready);
@@ -1083,14 +1224,14 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                 // scales are applied one after the other: ct . D3 is of ordinary size although ct can be
                 // e^-80 and D3 e^+80, whereas a pre-multiplied cgn * ct would underflow.)
 #pragma unroll
-                for (int j = 0; j < NS; ++j) S[j] *= gc;
+                for (int j = 0; j < 32; ++j) S[j] *= gc;
                 wait(mma2_bar, par, 3);
                 ptx::tc_fence_after();
                 {   // a8: S <- gamma^C . S + exp(G_C - G_m) . (K'^T V_new) ; refresh the bf16 operand copy
-                    float ds[NS];
+                    float ds[32];
                     tmem_ld_sum32(d3c + tmem_lane, ds);
 #pragma unroll
-                    for (int j = 0; j < NS; ++j) S[j] = fmaf(ct, ds[j], S[j]);
+                    for (int j = 0; j < 32; ++j) S[j] = fmaf(ct, ds[j], S[j]);
                     if (more) {
                         store_scaled(cgn);   // next chunk's operand copy: bf16(exp(G_m') . S_new)
                         ptx::fence_async_smem();
@@ -1098,18 +1239,18 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                     ptx::tc_fence_before();
                     if (more) warp_arrive(sbf_ready);
                 }
-                if (warp >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64)
+                if (quad >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64)
                     const int i = tid - 64;
                     const int64_t tok0 = J.tok_begin + (int64_t)c * kC;
                     const int len = (J.tok_end - tok0) < kC ? (int)(J.tok_end - tok0) : kC;
-                    __nv_bfloat16* orow = op + ((tok0 + i) * a.H + J.h) * kD + col0;
+                    __nv_bfloat16* orow = op + ((tok0 + i) * a.H + J.h) * kD + col0 + ch * 32;
                     wait(&out_bar[g & 1], (g >> 1) & 1u, 6);
                     ptx::tc_fence_after();
-                    float ov[NS];
+                    float ov[32];
                     tmem_ld_sum32(d1, ov);
                     if (i < len && !*abort_flag) {
 #pragma unroll
-                        for (int j = 0; j < NS; j += 8)
+                        for (int j = 0; j < 32; j += 8)
                             *reinterpret_cast<uint4*>(orow + j) =
                                 make_uint4(pack2(ov[j], ov[j + 1]), pack2(ov[j + 2], ov[j + 3]),
                                            pack2(ov[j + 4], ov[j + 5]), pack2(ov[j + 6], ov[j + 7]));
@@ -1118,14 +1259,16 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                 }
             }
             if (*abort_flag) break;
-            float* so = a.S_out + sbase;
+            if (a.S_out) {
+                float* so = a.S_out + sbase;
 #pragma unroll
-            for (int j = 0; j < NS; j += 4)
-                *reinterpret_cast<float4*>(so + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4*>(so + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
+            }
         }
     }
     ptx::tc_fence_before();
-    ptx::named_bar_sync(3, 256);
+    __syncthreads();
 }
 
 template <bool kHasQ>
@@ -1135,20 +1278,23 @@ kda_fused_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtens
              int clear_status)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + E_BAR + 32);
     const int t = threadIdx.x, warp = t >> 5;
+    const bool chain_cta = (int)blockIdx.x < f.n_chain_cta;
+    // (the TMEM slot sits in a spare word of the barrier block of either layout)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + (chain_cta ? C_BAR + 248 : E_BAR + 32));
 
     if (clear_status && blockIdx.x == 0 && t == 0) {
         f.hdr->status = 0;      // (an equal-length call has no prologue kernel to do this)
         f.hdr->where = 0;
         f.hdr->flags = 0;
     }
-    const bool chain_cta = (int)blockIdx.x < f.n_chain_cta;
     // barriers of the engines
-    if (t == 0 || (t == kEngThreads && !chain_cta)) {
+    if (!chain_cta && (t == 0 || t == kEngThreads)) {
         uint64_t* mb = reinterpret_cast<uint64_t*>(smem + (t ? E_BYTES : 0) + E_BAR);
-        ptx::mbar_init(mb, 1);
-        ptx::mbar_init(mb + 1, 1);
+        ptx::mbar_init(mb, 1);       // MMA group complete
+        ptx::mbar_init(mb + 1, 1);   // k landed
+        ptx::mbar_init(mb + 3, 1);   // q landed
+        ptx::mbar_init(mb + 5, 1);   // v landed
         *reinterpret_cast<volatile uint32_t*>(mb + 2) = 0;
         ptx::fence_mbar_init();
         if (t == 0) {
@@ -1168,20 +1314,14 @@ kda_fused_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtens
     const bool aligned = (ptx::smem_u32(smem) & 1023u) == 0;   // the operand images need 1024-byte alignment
     if (!aligned) {
         if (t == 0) report_timeout(f, 90);
+    } else if (chain_cta) {
+        chain_run<kHasQ>(f, smem, tmem_base, t, (int)blockIdx.x / kSlices, (int)blockIdx.x % kSlices);
     } else {
-        // engines: one per CTA, and a second one in the CTAs without a chain role
-        const uint32_t n_eng = gridDim.x + (gridDim.x - (uint32_t)f.n_chain_cta);
-        if (t < kEngThreads) {
-            engine_run<kHasQ>(f, smem, tmem_base, 1, t, blockIdx.x, n_eng, &tm_k, &tm_q, &tm_v);
-        } else if (!chain_cta) {
-            engine_run<kHasQ>(f, smem + E_BYTES, tmem_base + 256, 2, t - kEngThreads,
-                              gridDim.x + (blockIdx.x - (uint32_t)f.n_chain_cta), n_eng, &tm_k, &tm_q, &tm_v);
-        } else {
-#ifndef KDA_DEBUG_NO_CHAIN
-            chain_run<kHasQ>(f, smem + E_BYTES, tmem_base + 256, t - kEngThreads, (int)blockIdx.x >> 2,
-                             (int)blockIdx.x & 3);
-#endif
-        }
+        // two engines per CTA
+        if (t < kEngThreads)
+            engine_run<kHasQ>(f, smem, tmem_base, 1, t, &tm_k, &tm_q, &tm_v);
+        else
+            engine_run<kHasQ>(f, smem + E_BYTES, tmem_base + 256, 2, t - kEngThreads, &tm_k, &tm_q, &tm_v);
     }
     ptx::tc_fence_before();
     __syncthreads();
@@ -1282,7 +1422,9 @@ kda_status_t launch_fused_prep(WsHeader* hdr, const int32_t* cu_seqlens, uint32_
     return KDA_OK;
 }
 
-int fused_max_slots(int n_sm) { return n_sm / 4; }
+// chain CTAs: kSlices per running (sequence, head); at least half of the SMs stay with the engines
+int fused_max_slots(int n_sm) { return n_sm / (2 * kSlices); }
+int fused_slices() { return kSlices; }
 
 kda_status_t launch_fused_tc(FusedArgs f, bool has_q, bool clear_status, cudaStream_t st)
 {
@@ -1313,8 +1455,9 @@ kda_status_t launch_fused_tc(FusedArgs f, bool has_q, bool clear_status, cudaStr
     if (rc == KDA_OK) rc = make_tmap(&tm_v, f.a.v, f.a.total_tokens, f.a.H);
     if (rc == KDA_OK) rc = make_tmap(&tm_q, has_q ? f.a.q : f.a.k, f.a.total_tokens, f.a.H);
     if (rc != KDA_OK) return rc;
-    if (f.n_chain_cta > n_sm)
-        return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: %d chain roles on %d SMs", f.n_chain_cta, n_sm);
+    if (f.n_chain_cta >= n_sm)
+        return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: %d chain CTAs leave no SM of %d for the engines",
+                    f.n_chain_cta, n_sm);
     int cs = clear_status ? 1 : 0;
     void* args[] = {(void*)&f, (void*)&tm_k, (void*)&tm_q, (void*)&tm_v, (void*)&cs};
     const void* fn = has_q ? (const void*)kda_fused_tc<true> : (const void*)kda_fused_tc<false>;

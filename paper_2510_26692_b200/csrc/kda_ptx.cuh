@@ -32,18 +32,14 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
     return t;
 }
-// The waiting thread is suspended in hardware until the phase completes or a time of the order of
-// `kSuspendHintNs` has passed (so a waiting warp does not compete for issue slots with the warps
-// that do the work), then the call returns whether the phase has completed.
-constexpr uint32_t kSuspendHintNs = 2000;
 __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
+        : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
     return ok != 0;
 }
@@ -128,6 +124,8 @@ __device__ __forceinline__ void st_release_gpu(unsigned long long* p, unsigned l
 __device__ __forceinline__ void nanosleep(uint32_t ns) { asm volatile("nanosleep.u32 %0;" ::"r"(ns)); }
 // all bulk stores of this thread have completed (their writes are performed), not only read out
 __device__ __forceinline__ void bulk_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// the same for all but the most recently committed group
+__device__ __forceinline__ void bulk_wait_all1() { asm volatile("cp.async.bulk.wait_group 1;" ::: "memory"); }
 // orders generic-proxy and async-proxy (TMA engine) accesses of this thread, all state spaces
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
