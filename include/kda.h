@@ -18,9 +18,14 @@
  *       q, k, log_alpha : [total_tokens, H, dk]     v, o : [total_tokens, H, dv]
  *       beta            : [total_tokens, H]         S0, S_T, S : [n, H, dk, dv]  (dv contiguous)
  *   - alpha_t = exp(log_alpha_t), log_alpha <= 0 (a decay).  The cumulative log-decay of a channel
- *     over one 64-token chunk must stay above -160 (a factor e^-160); below that the intra-chunk
- *     interactions of that channel are attenuated (they never overflow or turn NaN: exponents are
- *     clamped).
+ *     over one 64-token chunk must stay above -160 (a factor e^-160).  The decay ratio
+ *     exp(G_i - G_j) of two tokens of a chunk is formed as exp(G_i - G_m) * exp(G_m - G_j) around the
+ *     middle G_m of the chunk's log-decay range, each exponent clamped to +-80.  Inside the limit
+ *     that is exact.  Beyond it a pair of tokens that both lie more than 80 from G_m on the same
+ *     side gets the product of two clamped factors, i.e. a ratio that is TOO LARGE (up to 1 where
+ *     the true ratio is smaller): the results stay finite but that channel's intra-chunk terms are
+ *     wrong.  The library detects the condition per chunk and channel and reports it through
+ *     kda_check_status as KDA_ERR_GATE_RANGE.
  *   - dt selects the storage type of q, k, v and o (fp32 or bf16).  Gates, beta and states are
  *     always fp32.  dt = KDA_BF16 runs the contractions on bf16 tensor cores with fp32
  *     accumulation; dt = KDA_F32 runs everything in fp32 FMA arithmetic.
@@ -51,17 +56,20 @@ typedef enum {
     KDA_ERR_UNSUPPORTED = 2, /* shape or dtype outside the supported set */
     KDA_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than the minimum */
     KDA_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
-    KDA_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (reported by kda_check_status) */
+    KDA_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (reported by kda_check_status) */
+    KDA_ERR_GATE_RANGE = 6   /* a channel decayed by more than e^-160 inside one chunk: results are
+                                finite but not exact (reported by kda_check_status) */
 } kda_status_t;
 
 typedef enum { KDA_F32 = 0, KDA_BF16 = 1 } kda_dtype_t;
 
 /*
- * Workspace size that lets kda_chunk_fwd process the whole call in one pass (all chunks of the
- * intra-chunk stage in flight at once), capped at 8 GiB.  Any workspace of at least
- * kda_chunk_fwd_min_workspace_bytes() works: a smaller one makes the call proceed in several
- * passes over ranges of chunks with the state carried between them.  Both return 0 for an
- * unsupported shape.
+ * Workspace size that lets kda_chunk_fwd keep every (chunk, head) tile of the call at once (the
+ * fastest schedule on this device: one kernel per stage), capped at 8 GiB.  Any workspace of at
+ * least kda_chunk_fwd_min_workspace_bytes() works: with less than the full size a bf16 call runs
+ * as one fused kernel whose stages exchange tiles through a ring (of up to 16 tiles per running
+ * head) inside the workspace, and an fp32 call proceeds in several passes over ranges of chunks
+ * with the state carried between them.  Both return 0 for an unsupported shape.
  */
 size_t kda_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
                                      int chunk, kda_dtype_t dt);
@@ -110,20 +118,25 @@ kda_status_t kda_chunk_fwd(const void *q, const void *k, const void *v, const fl
  *
  * Same arguments, results and error codes as kda_chunk_fwd, with these differences:
  *   - A call whose minimum scratch (kda_chunk_fwd_min_workspace_bytes) exceeds the 16 MiB is
- *     rejected with KDA_ERR_WORKSPACE and a message naming both sizes; nothing is launched.  The
- *     minimum grows with n_seqs * H (64 KiB of state scratch per sequence and head) and with H
- *     (one tile per head), so this entry point is for small batches -- e.g. up to 6 sequences of
- *     32 heads; long sequences are fine, they are processed in several passes.
+ *     rejected with KDA_ERR_WORKSPACE and a message naming both sizes; nothing is launched.  For
+ *     bf16 the minimum is a few hundred KiB plus 4 bytes per (sequence, head), so practically every
+ *     batch fits: the call runs as the fused kernel with a ring of about 220 tiles (e.g. 6 tiles
+ *     ahead for each of 32 concurrently running heads).  For fp32 the minimum holds 64 KiB of state
+ *     scratch per (sequence, head), which limits that path to about 200 of them.
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress, with the calling thread's current device).  Make that first call
  *     before starting any stream capture.
  *   - The entry point calls no cudaMalloc, cudaFree or allocating library routine.
  *   - All calls on one device share the one array, and it keeps the previous call's contents.
- *     Nothing in it has to be cleared by the caller (the call clears the status word itself), but
- *     two calls that overlap on the GPU -- different streams, or one stream per thread -- race on
- *     it: serialise them.  kda_check_status does not apply (no workspace pointer to pass).
+ *     Nothing in it has to be cleared by the caller (every call clears or re-tags what it reads),
+ *     but two calls that overlap on the GPU -- different streams, or one stream per thread -- race
+ *     on it: serialise them.
+ *   - The status word lives in the array: kda_chunk_fwd_static_check_status(stream) reads and
+ *     clears it exactly as kda_check_status does for a caller's workspace (it synchronises the
+ *     stream; it allocates nothing either).
  */
 size_t kda_chunk_fwd_static_max_bytes(void);
+kda_status_t kda_chunk_fwd_static_check_status(void *cuda_stream);
 kda_status_t kda_chunk_fwd_static(const void *q, const void *k, const void *v,
                                   const float *log_alpha, const float *beta, const float *S0,
                                   void *o, float *S_T, const int32_t *cu_seqlens_dev,
@@ -203,8 +216,9 @@ kda_status_t kda_decode_step_host(const void *q_host, const void *k_host, const 
 
 /*
  * Reads back (synchronising the stream) the status word that device code sets when one of its
- * bounded waits runs out, and clears it.  The word lives at the start of the workspace passed to
- * kda_chunk_fwd.  Returns KDA_OK or KDA_ERR_TIMEOUT.
+ * bounded waits runs out, and the flag that marks a decay outside the supported range (see the
+ * conventions at the top), and clears both.  They live at the start of the workspace passed to
+ * kda_chunk_fwd.  Returns KDA_OK, KDA_ERR_TIMEOUT or KDA_ERR_GATE_RANGE (a timeout wins).
  */
 kda_status_t kda_check_status(void *workspace, void *cuda_stream);
 
@@ -225,6 +239,14 @@ kda_status_t kda_selftest_wait_timeout(void *workspace, int limit_ms, void *cuda
  */
 void kda_profile_enable(int on);
 kda_status_t kda_profile_read(int kind, double *total_ms, int *launches);
+
+/*
+ * Self-test of the table in which the library keeps what it caches per device (SM count, kernel
+ * attributes already set, helper streams), one slot per device ordinal behind a mutex; no CUDA call
+ * is made, so it runs on a machine without a GPU.  Returns 0 when the table behaves (no counterpart
+ * in the paper).
+ */
+int kda_selftest_device_table(void);
 
 /* Description of the calling thread's last error ("" if none); static storage, never NULL. */
 const char *kda_last_error(void);

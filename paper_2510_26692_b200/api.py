@@ -16,7 +16,7 @@ import torch
 KDA_F32 = 0
 KDA_BF16 = 1
 _STATUS = {0: "KDA_OK", 1: "KDA_ERR_INVALID_ARG", 2: "KDA_ERR_UNSUPPORTED", 3: "KDA_ERR_WORKSPACE",
-           4: "KDA_ERR_CUDA", 5: "KDA_ERR_TIMEOUT"}
+           4: "KDA_ERR_CUDA", 5: "KDA_ERR_TIMEOUT", 6: "KDA_ERR_GATE_RANGE"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libkda_b200.so")
@@ -54,6 +54,8 @@ def load():
                                   i32, f32, i32, vp, sz, vp]
     lib.kda_chunk_fwd_static_max_bytes.restype = sz
     lib.kda_chunk_fwd_static_max_bytes.argtypes = []
+    lib.kda_chunk_fwd_static_check_status.restype = i32
+    lib.kda_chunk_fwd_static_check_status.argtypes = [vp]
     lib.kda_chunk_fwd_static.restype = i32
     lib.kda_chunk_fwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32,
                                          i32, i32, f32, i32, vp]
@@ -284,3 +286,9 @@ def kda_profile_read(kind: int):
 
 def kda_check_status(workspace, stream=None):
     _check(load().kda_check_status(_ptr(workspace, True, None, "workspace"), _stream(stream)))
+
+
+def kda_chunk_fwd_static_check_status(stream=None):
+    """Reads and clears the status word of the library's built-in scratch (the counterpart of
+    ``kda_check_status`` for ``kda_chunk_fwd_static`` calls); synchronises the stream."""
+    _check(load().kda_chunk_fwd_static_check_status(_stream(stream)))

@@ -148,6 +148,25 @@ const char* kda_last_error(void) { return g_err; }
 uint64_t kda_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 const char* kda_version(void) { return "kda-b200 sm_100a"; }
 
+int kda_selftest_device_table(void)
+{
+    // the slot table alone (no CUDA call): distinct slots for distinct ordinals, stable addresses,
+    // nothing for ordinals outside the table, and mutual exclusion of the lock
+    DeviceState* s0 = device_slot(0);
+    DeviceState* s1 = device_slot(1);
+    if (!s0 || !s1 || s0 == s1 || device_slot(0) != s0) return 1;
+    if (device_slot(-1) || device_slot(kMaxDevices)) return 2;
+    DeviceState* last = device_slot(kMaxDevices - 1);
+    if (!last || last == s0) return 3;
+    const bool a0 = s0->attr_done[5];
+    s1->attr_done[5] = !a0;
+    if (s0->attr_done[5] != a0) return 4;   // a write to one device's slot leaves the others alone
+    s1->attr_done[5] = false;
+    if (!g_dev_mu.try_lock()) return 5;     // (not held by this thread)
+    g_dev_mu.unlock();
+    return 0;
+}
+
 kda_status_t kda_set_chunk_path(int mode)
 {
     if (mode < 0 || mode > 2) return fail(KDA_ERR_INVALID_ARG, "kda_set_chunk_path: mode must be 0, 1 or 2");
@@ -159,10 +178,10 @@ size_t kda_chunk_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H
                                          int chunk, kda_dtype_t dt)
 {
     if (!shape_ok(dk, dv, chunk, dt) || total_tokens < 0 || n_seqs < 0 || H <= 0) return 0;
-    const size_t two_pass = ws_layout(n_seqs, H).fixed + align_up((size_t)H * tile_bytes(dt));
-    if (dt != KDA_BF16) return two_pass;
-    const size_t fused = fused_layout((int64_t)n_seqs * H).off_ring + 2 * tc_tile_bytes();
-    return fused > two_pass ? fused : two_pass;
+    // fp32: state scratch + one tile per head (the call then walks the chunks one at a time).
+    // bf16: what the fused kernel needs -- header, flag words, round table and a ring of two tiles.
+    if (dt != KDA_BF16) return ws_layout(n_seqs, H).fixed + align_up((size_t)H * tile_bytes(dt));
+    return fused_layout((int64_t)n_seqs * H).off_ring + 2 * tc_tile_bytes();
 }
 
 size_t kda_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
@@ -173,6 +192,12 @@ size_t kda_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, in
     const size_t fixed = ws_layout(n_seqs, H).fixed;
     size_t want = fixed + align_up((size_t)max_chunks(total_tokens, n_seqs) * H * tile_bytes(dt));
     if (want > kWorkspaceCap) want = kWorkspaceCap;
+    if (dt == KDA_BF16) {
+        // never below a full ring for the fused kernel (the path of a capped workspace)
+        const int64_t J = (int64_t)n_seqs * H;
+        const size_t ring = fused_layout(J).off_ring + (size_t)(J < kSlotCap ? J : kSlotCap) * kRingMax * tc_tile_bytes();
+        if (want < ring) want = ring;
+    }
     return want < lo ? lo : want;
 }
 
@@ -367,7 +392,7 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
         if (dt == KDA_BF16)
             rc = launch_chunk_tc(a, ws + L.off_tiles, n_begin, n_count, hdr, tc_clears && first, st);
         else
-            rc = launch_chunk_simt(a, dt, ws + L.off_tiles, n_begin, n_count, st);
+            rc = launch_chunk_simt(a, dt, ws + L.off_tiles, n_begin, n_count, hdr, st);
         if (rc != KDA_OK) return rc;
         g0 = g1;
         first = false;
@@ -485,10 +510,16 @@ kda_status_t kda_chunk_fwd_host(const void* q_host, const void* k_host, const vo
     // in both directions while the kernels run.
     constexpr int64_t kMinSegTokens = 512;
     if (n_seqs == 1 && !cu_seqlens_host && total_tokens >= 2 * kMinSegTokens) {
-        static cudaStream_t c_in = nullptr, c_out = nullptr;
-        if (!c_in) {
-            KDA_CUDA_TRY(cudaStreamCreateWithFlags(&c_in, cudaStreamNonBlocking));
-            KDA_CUDA_TRY(cudaStreamCreateWithFlags(&c_out, cudaStreamNonBlocking));
+        cudaStream_t c_in = nullptr, c_out = nullptr;   // helper streams of the calling thread's current device
+        {
+            DeviceLock lk;
+            if (!lk.st) return lk.rc;
+            if (!lk.st->copy_in)
+                KDA_CUDA_TRY(cudaStreamCreateWithFlags(&lk.st->copy_in, cudaStreamNonBlocking));
+            if (!lk.st->copy_out)
+                KDA_CUDA_TRY(cudaStreamCreateWithFlags(&lk.st->copy_out, cudaStreamNonBlocking));
+            c_in = lk.st->copy_in;
+            c_out = lk.st->copy_out;
         }
         int nseg = (int)(total_tokens / kMinSegTokens);
         if (nseg > 4) nseg = 4;
@@ -667,10 +698,15 @@ kda_status_t kda_check_status(void* workspace, void* cuda_stream)
     WsHeader h;
     KDA_CUDA_TRY(cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, st));
     KDA_CUDA_TRY(cudaStreamSynchronize(st));
-    if (h.status != 0) {
-        KDA_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st));
-        return fail((kda_status_t)h.status, "device code reported status %d at location %d",
-                    h.status, h.where);
+    if (h.status != 0 || (h.flags & 1)) {
+        // only the words the device reports through are cleared (a fused call keeps a counter
+        // further down in the header)
+        KDA_CUDA_TRY(cudaMemsetAsync(workspace, 0, 16, st));
+        if (h.status != 0)
+            return fail((kda_status_t)h.status, "device code reported status %d at location %d",
+                        h.status, h.where);
+        return fail(KDA_ERR_GATE_RANGE, "a channel decayed by more than e^-160 within one 64-token "
+                    "chunk: its intra-chunk terms were formed from clamped factors and are not exact");
     }
     return KDA_OK;
 }

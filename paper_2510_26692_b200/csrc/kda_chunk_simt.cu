@@ -42,7 +42,7 @@ constexpr size_t kInterSmem =
 __device__ __forceinline__ float clampf(float x) { return fminf(fmaxf(x, -kClamp), kClamp); }
 
 template <typename T>
-__global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, float* __restrict__ tiles)
+__global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, float* __restrict__ tiles, WsHeader* hdr)
 {
     extern __shared__ __align__(16) float smem[];
     float* sG = smem;                    // log-decay cumsum, later V
@@ -97,6 +97,9 @@ __global__ void __launch_bounds__(256, 1) kda_intra_simt(ChunkArgs a, float* __r
         const float gg[4] = {G.x, G.y, G.z, G.w}, gr[4] = {Gr.x, Gr.y, Gr.z, Gr.w};
         const float gl[4] = {Gl.x, Gl.y, Gl.z, Gl.w};
         float okg[4], oki[4], oqg[4], oKG[4], oQG[4], oKT[4], ogc[4];
+        // a channel that decays by more than e^-160 inside the chunk leaves the range of the
+        // two-factor form (the clamp keeps everything finite): flag the call
+        if (fminf(fminf(gl[0], gl[1]), fminf(gl[2], gl[3])) < -2.f * kClamp) atomicOr(&hdr->flags, 1);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float e1 = expf(clampf(gg[e] - gr[e]));
@@ -309,6 +312,7 @@ __global__ void kda_prep_kernel(WsHeader* hdr, const int32_t* __restrict__ cu,
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         hdr->status = 0;
         hdr->where = 0;
+        hdr->flags = 0;
         if (cu) {
             int acc = 0;
             chunk_cu[0] = 0;
@@ -321,23 +325,29 @@ __global__ void kda_prep_kernel(WsHeader* hdr, const int32_t* __restrict__ cu,
 }
 
 template <typename T>
-kda_status_t launch_simt_t(const ChunkArgs& a, float* tiles, int n_begin, int n_count, cudaStream_t st)
+kda_status_t launch_simt_t(const ChunkArgs& a, float* tiles, int n_begin, int n_count, WsHeader* hdr,
+                           cudaStream_t st)
 {
-    static bool attr_done = false;   // per dtype instantiation
-    if (!attr_done) {
-        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_simt<T>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)kIntraSmem));
-        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_simt<T>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)kInterSmem));
-        attr_done = true;
+    {
+        DeviceLock lk;
+        if (!lk.st) return lk.rc;
+        if (!lk.st->attr_done[4]) {
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_simt<T>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kIntraSmem));
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_simt<T>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kInterSmem));
+            lk.st->attr_done[4] = true;
+        }
     }
+    if (n_count > 65535)
+        return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: more than 65535 sequences in one fp32 call");
     const int64_t n_chunks = a.g1 - a.g0;
     if (n_chunks > 0) {
         dim3 grid((unsigned)n_chunks, (unsigned)a.H);
         ProfScope ps(PROF_INTRA, st);
-        kda_intra_simt<T><<<grid, 256, kIntraSmem, st>>>(a, tiles);
+        kda_intra_simt<T><<<grid, 256, kIntraSmem, st>>>(a, tiles, hdr);
         count_launch();
         KDA_CUDA_TRY(cudaGetLastError());
     }
@@ -356,10 +366,10 @@ kda_status_t launch_simt_t(const ChunkArgs& a, float* tiles, int n_begin, int n_
 size_t simt_tile_bytes() { return (size_t)T_FLOATS * sizeof(float); }
 
 kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, int n_begin,
-                               int n_count, cudaStream_t st)
+                               int n_count, WsHeader* hdr, cudaStream_t st)
 {
-    if (dt == KDA_BF16) return launch_simt_t<__nv_bfloat16>(a, (float*)tiles, n_begin, n_count, st);
-    return launch_simt_t<float>(a, (float*)tiles, n_begin, n_count, st);
+    if (dt != KDA_F32) return fail(KDA_ERR_UNSUPPORTED, "the FMA path serves fp32 storage only");
+    return launch_simt_t<float>(a, (float*)tiles, n_begin, n_count, hdr, st);
 }
 
 kda_status_t launch_prep(WsHeader* hdr, const int32_t* cu_seqlens, int32_t* chunk_cu, int n_seqs,

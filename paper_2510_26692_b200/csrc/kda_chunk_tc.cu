@@ -34,7 +34,7 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, boo
 namespace {
 
 constexpr uint64_t kWaitLimitNs = 1000000000ull;   // 1 s per wait
-constexpr int kNCtrl = 2;                          // MMA-issuing threads (one per control warp): 2 or 4
+constexpr int kNCtrl = 2;                          // MMA-issuing threads (one per control warp)
 
 template <int NS> struct InterCfg {
     static_assert(NS == 32 || NS == 64, "state columns per CTA: one or two 32-column blocks");
@@ -68,13 +68,6 @@ __device__ __forceinline__ void tmem_ld_sum(uint32_t taddr, float (&acc)[NS]) {
         ptx::tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 32; ++j) acc[blk * 32 + j] = __uint_as_float(r[j]) + __uint_as_float(r2[j]);
-        if (kNCtrl == 4) {
-            ptx::tmem_ld_32x32b_x32(taddr + 2 * NS + blk * 32, r);
-            ptx::tmem_ld_32x32b_x32(taddr + 3 * NS + blk * 32, r2);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) acc[blk * 32 + j] += __uint_as_float(r[j]) + __uint_as_float(r2[j]);
-        }
     }
 }
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
@@ -138,7 +131,6 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     if (ce > a.g1) ce = a.g1;
     const int nchunks = ce > cb ? (int)(ce - cb) : 0;
 
-    KDA_PHASE_DECL;
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < NSTG; ++s) ptx::mbar_init(&full[s], 1);
@@ -282,7 +274,6 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         store_scaled(ref_scale_of(0));
         ptx::fence_async_smem();
         warp_arrive(sbf_ready);
-        KDA_PHASE(hdr, 16);  // set-up
 
         for (int it = 0; it < nchunks; ++it) {
             const int s = it % NSTG;
@@ -297,7 +288,6 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                     uq[c] = *reinterpret_cast<const uint4*>(sb + Cfg::kU + (c >> 2) * tc::U_BLOCK + tc::u_off(tid, c & 3));
                 const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
                 wait(mma1_bar, par, 2);
-                KDA_PHASE(hdr, 18);  // MMA1
                 ptx::tc_fence_after();
                 float x[NS];
                 tmem_ld_sum<NS>(tmem_lane + d1, x);
@@ -307,7 +297,6 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::fence_async_smem();
                 ptx::tc_fence_before();
                 warp_arrive(vn_ready);
-                KDA_PHASE(hdr, 19);  // V_new
             }
             const float gc = reinterpret_cast<const float*>(sb + Cfg::kGC)[tid];          // gamma^C
             const float ct = reinterpret_cast<const float*>(sb + Cfg::kGC + 1024)[tid];   // exp(G_C - G_m)
@@ -318,7 +307,6 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
 #pragma unroll
             for (int j = 0; j < NS; ++j) S[j] *= gc;
             wait(mma2_bar, par, 3);
-            KDA_PHASE(hdr, 20);  // MMA2
             ptx::tc_fence_after();
             {   // a8: S <- gamma^C . S + exp(G_C - G_m) . (K'^T V_new) ; refresh the bf16 operand copy
                 float ds[NS];
@@ -330,7 +318,6 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::tc_fence_before();
                 warp_arrive(sbf_ready);
             }
-            KDA_PHASE(hdr, 21);  // state update
             if (warp >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64)
                 const int i = tid - 64;
                 const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
@@ -357,7 +344,6 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 *reinterpret_cast<float4*>(so + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
         }
     }
-    KDA_PHASE_FLUSH(hdr);
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 0) ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
@@ -368,11 +354,15 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
                                WsHeader* hdr, bool after_intra, cudaStream_t st)
 {
     using Cfg = InterCfg<NS>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_tc<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)Cfg::kSmem));
-        attr_done = true;
+    {
+        DeviceLock lk;
+        if (!lk.st) return lk.rc;
+        const int slot = NS == 32 ? 2 : 3;
+        if (!lk.st->attr_done[slot]) {
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_tc<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)Cfg::kSmem));
+            lk.st->attr_done[slot] = true;
+        }
     }
     ProfScope ps(PROF_INTER, st);
     cudaLaunchConfig_t cfg = {};
@@ -428,12 +418,20 @@ kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n
     // 32 state columns per CTA give the most CTAs (the chains are latency-bound); once there are
     // more chains than the GPU can hold at one CTA per SM, 64 columns per CTA do twice the work per
     // MMA issue and halve the operand traffic from L2.
-    static int n_sm = 0;
-    if (n_sm == 0) {
-        int dev = 0;
-        KDA_CUDA_TRY(cudaGetDevice(&dev));
-        KDA_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    int n_sm = 0;
+    {
+        DeviceLock lk;
+        if (!lk.st) return lk.rc;
+        if (lk.st->n_sm == 0) {
+            int dev = 0;
+            KDA_CUDA_TRY(cudaGetDevice(&dev));
+            KDA_CUDA_TRY(cudaDeviceGetAttribute(&lk.st->n_sm, cudaDevAttrMultiProcessorCount, dev));
+        }
+        n_sm = lk.st->n_sm;
     }
+    if (n_count > 65535)
+        return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: more than 65535 sequences in one two-kernel pass "
+                    "(use kda_set_chunk_path(2) or fewer sequences per call)");
     if ((int64_t)n_count * a.H * 4 > 2 * (int64_t)n_sm)
         return launch_inter_tc_t<64>(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);
     return launch_inter_tc_t<32>(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);

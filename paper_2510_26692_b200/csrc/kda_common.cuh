@@ -114,33 +114,6 @@ template <> struct IO<__nv_bfloat16> {
     }
 };
 
-// Optional phase timing (compile with -DKDA_PHASE_TIMING): thread 0 of every CTA adds the cycles
-// spent since its previous mark to hdr->pad[slot].  Compiled out of the product build.
-#ifdef KDA_PHASE_TIMING
-#define KDA_PHASE_DECL                  \
-    long long kda_phase_last_ = clock64(); \
-    int kda_phase_acc_[24] = {0}
-#define KDA_PHASE(hdr, slot)                                                  \
-    do {                                                                      \
-        if (threadIdx.x == 0) {                                               \
-            const long long now_ = clock64();                                 \
-            kda_phase_acc_[slot] += (int)(now_ - kda_phase_last_);            \
-            kda_phase_last_ = now_;                                           \
-        }                                                                     \
-    } while (0)
-#define KDA_PHASE_FLUSH(hdr)                                                  \
-    do {                                                                      \
-        if (threadIdx.x == 0) {                                               \
-            _Pragma("unroll") for (int s_ = 0; s_ < 24; ++s_)                 \
-                if (kda_phase_acc_[s_]) atomicAdd(&(hdr)->pad[s_], kda_phase_acc_[s_] >> 4); \
-        }                                                                     \
-    } while (0)
-#else
-#define KDA_PHASE_DECL do {} while (0)
-#define KDA_PHASE(hdr, slot) do {} while (0)
-#define KDA_PHASE_FLUSH(hdr) do {} while (0)
-#endif
-
 // Locate global chunk g: sequence index, first token, number of valid tokens (1..64).
 struct ChunkLoc {
     int n;
@@ -185,7 +158,7 @@ kda_status_t launch_decode_multi(const void* q, const void* k, const void* v, co
 // fp32 FMA path (also accepts bf16 storage): per-tile scratch size and pass launcher
 size_t simt_tile_bytes();
 kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, int n_begin,
-                               int n_count, cudaStream_t st);
+                               int n_count, WsHeader* hdr, cudaStream_t st);
 
 // bf16 tensor-core path (tcgen05 + bulk copies): per-tile scratch size and pass launcher
 size_t tc_tile_bytes();

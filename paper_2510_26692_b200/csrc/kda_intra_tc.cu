@@ -56,13 +56,9 @@ constexpr uint32_t S_U = S_M + 16384;          // U: four [64][32] bf16 blocks
 constexpr uint32_t S_BETA = S_T + 64 * LDT * 4;
 constexpr uint32_t S_BAR = S_BETA + 256;        // mma barrier, tma barrier, TMEM slot
 constexpr uint32_t S_TOTAL = S_BAR + 64;
-#ifndef KDA_INTRA_THREADS
-#define KDA_INTRA_THREADS 256
-#endif
-constexpr int kNT = KDA_INTRA_THREADS;   // threads per CTA (256 or 512), two CTAs per SM
+constexpr int kNT = 256;                 // threads per CTA, two CTAs per SM
 constexpr int kNW = kNT / 32;            // warps
-constexpr int kRPT = kC / kNW;           // token rows per thread in the gating phase (8 or 4)
-static_assert(kNT == 256 || kNT == 512, "thread mappings below are written for 8 or 16 warps");
+constexpr int kRPT = kC / kNW;           // token rows per thread in the gating phase
 constexpr int kBulkThread = kNT / 2;     // lane 0 of a middle warp issues every bulk copy; thread 0 the MMAs
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kClamp2 = 80.f * 1.4426950408889634f;   // the +-80 clamp in the log2 domain
@@ -152,18 +148,20 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     uint64_t* mma_bar = reinterpret_cast<uint64_t*>(smem + S_BAR);
     uint64_t* tma_bar = mma_bar + 1;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_bar + 2);
+    volatile uint32_t* abort_word = tmem_slot + 1;   // set by the first thread whose bounded wait runs out
 
     const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
 
-    KDA_PHASE_DECL;
     ptx::grid_dep_launch();   // the inter-chunk kernel may set itself up while this one drains
     if (clear_status && blockIdx.x == 0 && t == 0) {
         hdr->status = 0;      // (an equal-length call has no prologue kernel to do this)
         hdr->where = 0;
+        hdr->flags = 0;
     }
     if (t == 0) {
         ptx::mbar_init(mma_bar, 1);
         ptx::mbar_init(tma_bar, 1);
+        *abort_word = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tm_k);
         ptx::prefetch_tmap(&tm_q);
@@ -224,7 +222,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    bool timed_out = false;
+    bool timed_out = false, load_pending = false, out_of_range = false;
     uint32_t tma_parity = 0;
 
     uint32_t cur = blockIdx.x;
@@ -234,6 +232,7 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         locate(cur, L, h);
         prefetch_regs(L, h);
         prefetch_bufs(L, h);
+        load_pending = true;
     }
     for (; cur < ntiles; cur += gridDim.x) {
     char* tile = tiles + (size_t)cur * tc::TILE_BYTES;
@@ -242,7 +241,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     int hn = h;
 
     // ---- a1: cumulative log-decay, in the log2 domain (exponentials below are bare ex2) -------
-    KDA_PHASE(hdr, 13);  // loop overhead
 #pragma unroll
     for (int e = 0; e < 4; ++e) G[0][e] *= kLog2e;
 #pragma unroll
@@ -250,11 +248,11 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
 #pragma unroll
         for (int e = 0; e < 4; ++e) G[r][e] = fmaf(G[r][e], kLog2e, G[r - 1][e]);
     *reinterpret_cast<float4*>(sTot + warp * kD + d0) = make_float4(G[kRPT - 1][0], G[kRPT - 1][1], G[kRPT - 1][2], G[kRPT - 1][3]);
-    KDA_PHASE(hdr, 14);  // G arrived + local scan
     ptx::cp_async_wait_all();             // beta
-    KDA_PHASE(hdr, 15);  // beta wait
     __syncthreads();
-    KDA_PHASE(hdr, 0);   // loads arrived + local scan
+    // a wait of the previous tile ran out: stop here (uniform: the flag was set before the barrier);
+    // the copies in flight are drained after the loop
+    if (*abort_word) break;
     float base[4] = {0.f, 0.f, 0.f, 0.f}, gref[4] = {0.f, 0.f, 0.f, 0.f}, glast[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int r2 = 0; r2 < kNW; ++r2) {
@@ -282,11 +280,13 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         *reinterpret_cast<float4*>(tile + tc::OFF_GV + 1024 + d0 * 4) =
             make_float4(ex2(glast[0] - gref[0]), ex2(glast[1] - gref[1]), ex2(glast[2] - gref[2]),
                         ex2(glast[3] - gref[3]));
+        // a channel that decays by more than e^-160 inside this chunk leaves the range of the
+        // two-factor form (the clamp below keeps everything finite): flag the call at the end
+        if (fminf(fminf(glast[0], glast[1]), fminf(glast[2], glast[3])) < -2.f * kClamp2) out_of_range = true;
     }
-    KDA_PHASE(hdr, 10);  // prefix + per-channel factors
-    if (!ptx::mbar_wait(tma_bar, tma_parity, kWaitLimitNs)) timed_out = true;   // k, q, v have landed
+    if (!ptx::mbar_wait(tma_bar, tma_parity, kWaitLimitNs)) { timed_out = true; *abort_word = 1; }   // k, q, v have landed
     tma_parity ^= 1;
-    KDA_PHASE(hdr, 11);  // TMA wait
+    load_pending = false;
     if (L.len < kC) {   // short last chunk: rows past the end hold the next sequence's v; zero them
         for (int idx = t; idx < (kC - L.len) * 16; idx += kNT) {
             const int j = L.len + (idx >> 4), c16 = idx & 15;
@@ -332,11 +332,9 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     };
     gate_rows(std::integral_constant<bool, kHasQ>{});
 
-    KDA_PHASE(hdr, 12);  // element loop + stores (thread 0)
     ptx::fence_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
-    KDA_PHASE(hdr, 1);   // gated operands
     ptx::tc_fence_after();
 
     // ---- a2 + a5: [Kg ; Qg] Ki^T ------------------------------------------------------------------------
@@ -363,20 +361,18 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         locate(nxt, Ln, hn);
         prefetch_regs(Ln, hn);
     }
-    if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) timed_out = true;
+    if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) { timed_out = true; *abort_word = 1; }
     // the previous tile's W/U staging (and this tile's Q', K' stores) have been read out by now; the
     // staging area is written next (L, Aqk)
     if (t == kBulkThread) ptx::bulk_wait_read0();
     __syncthreads();
-    KDA_PHASE(hdr, 2);   // first MMA group
     ptx::tc_fence_after();
     {
-        constexpr int NCA = 64 / (kNW / 4);   // accumulator columns per warp: 32 (8 warps) or 16 (16 warps)
+        constexpr int NCA = 32;   // accumulator columns per warp
         const int q4 = warp & 3, c0 = (warp >> 2) * NCA;
         const int R = q4 * 32 + lane;
         uint32_t r[NCA];
-        if (NCA == 32) ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q4 * 32) << 16) + c0, reinterpret_cast<uint32_t(&)[32]>(r));
-        else ptx::tmem_ld_32x32b_x16(tmem_base + ((uint32_t)(q4 * 32) << 16) + c0, reinterpret_cast<uint32_t(&)[16]>(r));
+        ptx::tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q4 * 32) << 16) + c0, r);
         ptx::tmem_ld_wait();
         if (R < 64) {
             const int i = R;
@@ -414,7 +410,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         ptx::bulk_s2g(tile + tc::OFF_AQ, smem + S_AQ, 8192);
         ptx::bulk_commit();
     }
-    KDA_PHASE(hdr, 3);   // TMEM -> L, Aqk
 
     // ---- a3: T = (I + L)^-1, blocked forward substitution -------------------------------------------
     if (t < 64) {   // diagonal 16x16 blocks: one column per thread, rows unrolled in registers
@@ -432,7 +427,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         for (int r = 0; r < 16; ++r) sT[(I * 16 + r) * LDT + I * 16 + c] = x[r];
     }
     __syncthreads();
-    KDA_PHASE(hdr, 4);   // diagonal blocks
     // X_IM = T_II L_IM for the six sub-diagonal blocks (one warp each, in place), then
     // T_IJ = - sum_{M=J..I-1} X_IM T_MJ in three dependency stages; the terms of a sum that do not
     // depend on blocks still being computed are taken early (kept, un-negated, in the block's place).
@@ -454,7 +448,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         block16_store(blk(sT, I, M), acc2, (I - M == 1) ? -1.f : 1.f, LDT, lane);
     }
     __syncthreads();
-    KDA_PHASE(hdr, 5);   // X + stage A
     if (warp < 3) {
         // warp 0: T20 (M = 1), warp 1: T31 (M = 2), warp 2: P30 += X31 T10
         const int I = warp == 0 ? 2 : 3, J = warp == 1 ? 1 : 0, M = warp == 1 ? 2 : 1;
@@ -472,10 +465,9 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     }
     __syncthreads();
 
-    KDA_PHASE(hdr, 6);   // block levels
     // ---- a4: Mm = T Diag(beta) as the A operand; [W | U] = Mm [Kg | V] ---------------------------------
     {
-        constexpr int NCM = 64 / (kNT / 64);   // columns per thread: 16 (256 threads) or 8 (512 threads)
+        constexpr int NCM = 16;   // columns per thread
         const int i = t / (kNT / 64), jq = t % (kNT / 64);
         const int j0 = jq * NCM;
         float x[NCM];
@@ -503,7 +495,6 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
     ptx::fence_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
-    KDA_PHASE(hdr, 7);   // Mm
     if (t == 0) {
         ptx::tc_fence_after();
         const uint32_t idesc = ptx::umma_idesc_bf16(128, 128) | ptx::kIdescBMajorMN;
@@ -519,13 +510,15 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
                            ptx::umma_desc_sw128_mn(v0 + k * 2048, S_V_BLOCK), idesc, k > 0);
         ptx::umma_commit(mma_bar);
     }
-    if (!ptx::mbar_wait(mma_bar, 1, kWaitLimitNs)) timed_out = true;
-    if (nxt < ntiles) prefetch_bufs(Ln, hn);
-    KDA_PHASE(hdr, 8);   // second MMA group
+    if (!ptx::mbar_wait(mma_bar, 1, kWaitLimitNs)) { timed_out = true; *abort_word = 1; }
+    if (nxt < ntiles) {
+        prefetch_bufs(Ln, hn);
+        load_pending = true;
+    }
     ptx::tc_fence_after();
     {   // The A operand held every row twice, so TMEM lanes 0-63 and 64-127 both carry rows 0-63:
         // each warp converts rows 32 (q4 & 1) + lane of one NCE-column block of [W | U].
-        constexpr int NCE = 256 / (kNW / 2);   // 64 columns per warp (8 warps) or 32 (16 warps)
+        constexpr int NCE = 64;   // columns per warp
         const int q4 = warp & 3, cbk = (warp >> 2) * 2 + (q4 >> 1);
         const int col0 = cbk * NCE;            // first column inside [W | U]
         const int i = (q4 & 1) * 32 + lane;
@@ -565,13 +558,13 @@ kda_intra_tc(ChunkArgs a, char* __restrict__ tiles, WsHeader* hdr,
         ptx::bulk_s2g(tile + tc::OFF_U, smem + S_U, 16384);
         ptx::bulk_commit();   // read-out completion is awaited before the staging area is reused
     }
-    KDA_PHASE(hdr, 9);   // W, U epilogue
     L = Ln;
     h = hn;
     }   // tile loop
 
     if (timed_out && atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = 10;
-    KDA_PHASE_FLUSH(hdr);
+    if (out_of_range) atomicOr(&hdr->flags, 1);
+    if (load_pending && t == 0) ptx::mbar_wait(tma_bar, tma_parity, kWaitLimitNs);   // a requested tile must land before the CTA ends
     if (t == kBulkThread) ptx::bulk_wait_read0();   // shared memory must outlive the reads of every bulk store
     ptx::cp_async_wait_all();
     ptx::tc_fence_before();
@@ -620,24 +613,28 @@ kda_status_t make_tmap(CUtensorMap* tm, const void* base, int64_t total_tokens, 
 kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, bool clear_status,
                              cudaStream_t st)
 {
-    static bool attr_done = false;
-    if (!attr_done) {
-        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)kIntraTcSmem));
-        KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)kIntraTcSmem));
-        attr_done = true;
+    int n_sm = 0;
+    {
+        DeviceLock lk;
+        if (!lk.st) return lk.rc;
+        if (!lk.st->attr_done[1]) {
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kIntraTcSmem));
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kIntraTcSmem));
+            lk.st->attr_done[1] = true;
+        }
+        if (lk.st->n_sm == 0) {
+            int dev = 0;
+            KDA_CUDA_TRY(cudaGetDevice(&dev));
+            KDA_CUDA_TRY(cudaDeviceGetAttribute(&lk.st->n_sm, cudaDevAttrMultiProcessorCount, dev));
+        }
+        n_sm = lk.st->n_sm;
     }
     const int64_t n_tiles = (a.g1 - a.g0) * a.H;
     if (n_tiles <= 0) return KDA_OK;
     if (n_tiles > 0x7fffffff || a.total_tokens > 0x7fffffff)
         return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: more than 2^31 tokens or tiles in one pass");
-    static int n_sm = 0;
-    if (n_sm == 0) {
-        int dev = 0;
-        KDA_CUDA_TRY(cudaGetDevice(&dev));
-        KDA_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-    }
     CUtensorMap tm_k, tm_q, tm_v;
     kda_status_t rc = make_tmap(&tm_k, a.k, a.total_tokens, a.H);
     if (rc == KDA_OK) rc = make_tmap(&tm_v, a.v, a.total_tokens, a.H);

@@ -49,6 +49,14 @@ extern "C" {
 
 size_t kda_chunk_fwd_static_max_bytes(void) { return kStaticScratchBytes; }
 
+kda_status_t kda_chunk_fwd_static_check_status(void* cuda_stream)
+{
+    void* scratch = nullptr;
+    kda_status_t rc = scratch_address(&scratch);
+    if (rc != KDA_OK) return rc;
+    return kda_check_status(scratch, cuda_stream);
+}
+
 kda_status_t kda_chunk_fwd_static(const void* q, const void* k, const void* v, const float* log_alpha,
                                   const float* beta, const float* S0, void* o, float* S_T,
                                   const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host,

@@ -92,3 +92,26 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(api, "_LIB_PATH", "/nonexistent/libkda_b200.so")
     with pytest.raises(ImportError):
         api.kda_version()
+
+
+def test_per_device_table(lib):
+    """What the library caches per device lives in one slot per device ordinal behind a mutex; the
+    self-test exercises the table without any CUDA call.  Also from several threads at once."""
+    import threading
+    lib.kda_selftest_device_table.restype = ctypes.c_int
+    assert lib.kda_selftest_device_table() == 0
+    out = []
+    ts = [threading.Thread(target=lambda: out.append(lib.kda_selftest_device_table())) for _ in range(8)]
+    for t in ts:
+        t.start()
+    for t in ts:
+        t.join()
+    # (the lock probe may find the mutex taken by a sibling thread: code 5 is not a table fault)
+    assert all(c in (0, 5) for c in out) and 0 in out
+
+
+def test_chunk_path_switch(lib):
+    import paper_2510_26692_b200 as K
+    for mode in (2, 1, 0):
+        K.kda_set_chunk_path(mode)
+    assert lib.kda_set_chunk_path(3) == 1 and lib.kda_set_chunk_path(-1) == 1
