@@ -40,6 +40,10 @@ FLOPS_PER_TOKEN_HEAD = 6 * D * D + 3 * CHUNK * D + CHUNK * CHUNK   # the paper's
 # profiles/ (prefill: intra 168.4 + 99.7 MB, inter 156.3 + 20.1 MB; decode: 547.4 + 484.7 MB)
 PREFILL_DRAM_TRAFFIC = {"intra_chunk": 268.1e6, "inter_chunk": 176.4e6}
 DECODE_DRAM_TRAFFIC = 1032.1e6
+FUSED_DRAM_TRAFFIC = None
+TRAFFIC_SOURCE = "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the summaries under profiles/ (not measured in this run)"
+MIN_TIMED_S = 0.5      # the timed region is extended (whole blocks of `steps` calls) to at least this
+MAX_BLOCKS = 2000
 
 
 def load_peaks():
@@ -197,8 +201,11 @@ def extra_workloads(K, inputs, torch, dev, peaks):
                                        S_T, cu_dev, cu_host, 16, T, H, D, D, CHUNK, 1.0, K.KDA_BF16,
                                        ws, nb, stream), 10)
     nbytes = T * H * BYTES_PER_TOKEN_HEAD + 16 * H * STATE_BYTES
-    out["varlen_16seq"] = {"total_tokens": T, "lengths": lens, "ms": ms, "tokens_per_s": T / (ms * 1e-3),
-                           "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    out["varlen_16seq"] = {"workload": "16 packed sequences, lengths uniform on [512, 16384], H=32, bf16, per-sequence S0",
+                           "total_tokens": T, "lengths": lens, "ms": ms, "tokens_per_s": T / (ms * 1e-3),
+                           "algorithmic_bytes": nbytes, "achieved_gbs": nbytes / (ms * 1e-3) / 1e9,
+                           "frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                           "traffic_note": "not captured: the workload is above the size an ncu capture is kept to"}
     del d, ws, o, S_T
     torch.cuda.empty_cache()
 
@@ -212,8 +219,11 @@ def extra_workloads(K, inputs, torch, dev, peaks):
                                        S_T, None, None, 1, T, H, D, D, CHUNK, 1.0, K.KDA_BF16, ws, nb,
                                        stream), 3)
     nbytes = T * H * 1028 + H * STATE_BYTES     # k, v, gates, beta; no q, no o
-    out["long_context_1Mi_state_only"] = {"total_tokens": T, "ms": ms, "tokens_per_s": T / (ms * 1e-3),
-                                          "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    out["long_context_1Mi_state_only"] = {"workload": "B=1, T=1048576, H=32, bf16, gates logsigmoid(N(6,1)), final state only (o = NULL)",
+                                          "total_tokens": T, "ms": ms, "tokens_per_s": T / (ms * 1e-3),
+                                          "algorithmic_bytes": nbytes, "achieved_gbs": nbytes / (ms * 1e-3) / 1e9,
+                                          "frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                                          "traffic_note": "not captured: the workload is above the size an ncu capture is kept to"}
     del d, ws, S_T
     torch.cuda.empty_cache()
     return out
@@ -251,6 +261,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-reps", type=int, default=5)
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the packed-batch and 1 Mi-token workloads (they run by default)")
     ap.add_argument("--all-workloads", action="store_true",
                     help="also time the packed varlen batch (16 sequences) and the 1 Mi-token "
                          "state-only prefill; needs ~70 GB of device memory")
@@ -318,16 +330,30 @@ def main():
     sampler.start()
     l0 = K.kda_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        prefill_step(i)
-    e1.record(stream)
-    barrier()
+    # The timed unit is a block of exactly `steps` calls between two events (barrier and
+    # synchronize on both sides, max over ranks).  Blocks are repeated until at least
+    # MIN_TIMED_S of device time has been measured, so that the clock sampler sees the load, and
+    # the median block is reported (min and max beside it).
+    block_ms = []
+    while True:
+        barrier()
+        e0.record(stream)
+        for i in range(args.steps):
+            prefill_step(i)
+        e1.record(stream)
+        barrier()
+        block_ms.append(max_over_ranks(e0.elapsed_time(e1)))
+        if sum(block_ms) >= MIN_TIMED_S * 1e3 or len(block_ms) >= MAX_BLOCKS:
+            break
     launches = K.kda_launch_count() - l0
     clocks = sampler.finish()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    srt = sorted(block_ms)
+    ms_total = srt[len(srt) // 2]
     ms_step = ms_total / args.steps
     tokens_per_s = whole_job_rate(T_PREFILL, world, ms_step)
+    timing = {"blocks": len(block_ms), "steps_per_block": args.steps, "reported": "median block",
+              "ms_per_step_min": srt[0] / args.steps, "ms_per_step_max": srt[-1] / args.steps,
+              "timed_region_ms": sum(block_ms)}
 
     # per-kernel durations (separate pass: the event pairs perturb back-to-back launches slightly)
     K.kda_profile_enable(True)
@@ -344,15 +370,15 @@ def main():
     # that the whole path's algorithmic bytes are divided by is the device time of one call in the
     # timed region; the per-kernel event pairs below serialise the kernels and are kept as shares.
     step_bytes = T_PREFILL * H * BYTES_PER_TOKEN_HEAD + H * STATE_BYTES
-    achieved = step_bytes / (e0.elapsed_time(e1) / args.steps * 1e-3) / 1e9
+    achieved = step_bytes / (ms_step * 1e-3) / 1e9
     roofline = {
         "bound": "hbm", "kernel": "kda_chunk_fwd (all kernels of one call: %s)" % "+".join(kern),
-        "duration_ms": e0.elapsed_time(e1) / args.steps,
+        "duration_ms": ms_step,
         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
         "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "peak_source": peaks["source"],
         "frac_of_8TBs_nominal": (achieved / 8000.0) if achieved else None,
         "algorithmic_bytes_per_step": step_bytes, "traffic": sum(PREFILL_DRAM_TRAFFIC.values()),
-        "traffic_per_kernel": PREFILL_DRAM_TRAFFIC, "kernels": kern,
+        "traffic_per_kernel": PREFILL_DRAM_TRAFFIC, "traffic_source": TRAFFIC_SOURCE, "kernels": kern,
         "tensor_bound_tokens_per_s": peaks["bf16_tflops"] * 1e12 / (H * FLOPS_PER_TOKEN_HEAD),
         "hbm_bound_tokens_per_s": peaks["hbm_gbs"] * 1e9 / (step_bytes / T_PREFILL),
         "note": "HBM is the slower bound at d=128, C=64; the tensor-pipe bound is above it",
@@ -362,7 +388,8 @@ def main():
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": tokens_per_s, "unit": "tokens/s",
                               "ms_per_step": ms_step, "steps": args.steps, "warmup": args.warmup,
-                              "gpu_launches": launches, "kernels": kern, "partial": "prefill-only"}))
+                              "gpu_launches": launches, "kernels": kern, "timing": timing,
+                              "partial": "prefill-only"}))
         if world > 1:
             dist.destroy_process_group()
         return 0
@@ -451,10 +478,36 @@ def main():
                      "algorithmic_bytes_per_step": dec_bytes, "traffic": DECODE_DRAM_TRAFFIC},
     }
 
-    # ---- the other prefill workloads (on request) ----------------------------------------------------
+    # ---- the same prefill through the fused cooperative kernel (the path of small workspaces) --------
+    fused = None
+    if world == 1:
+        K.kda_set_chunk_path(2)
+        try:
+            for i in range(3):
+                prefill_step(i)
+            barrier()
+            e0.record(stream)
+            for i in range(20):
+                prefill_step(i)
+            e1.record(stream)
+            barrier()
+            fms = e0.elapsed_time(e1) / 20
+            fused = {"kernel": "kda_fused_tc (one cooperative launch: intra-chunk engines and inter-chunk "
+                               "chains, tiles through a ring in L2)", "ms_per_step": fms,
+                     "tokens_per_s": T_PREFILL / (fms * 1e-3),
+                     "frac": step_bytes / (fms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "traffic": FUSED_DRAM_TRAFFIC, "traffic_source": TRAFFIC_SOURCE}
+        finally:
+            K.kda_set_chunk_path(0)
+
+    # ---- the other prefill workloads (packed batch, 1 Mi tokens) -------------------------------------
     other = None
-    if args.all_workloads and world == 1:
-        other = extra_workloads(K, inputs, torch, dev, peaks)
+    free_b, _ = torch.cuda.mem_get_info()
+    if world == 1 and not args.no_other_workloads:
+        if free_b >= 80 * (1 << 30):
+            other = extra_workloads(K, inputs, torch, dev, peaks)
+        else:
+            other = {"skipped": "needs about 70 GB of free device memory, %.0f GB free" % (free_b / 2 ** 30)}
 
     # ---- CPU oracle beside it (rank 0, single-GPU runs only) --------------------------------------
     cpu = None
@@ -488,9 +541,11 @@ def main():
                                    "per GPU",
                        "l2": "inputs rotate over 3 copies of 206 MB each (> 126 MB L2)",
                        "decode_workload": "256 seqs x 32 heads, 64 in-place steps"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-            "decode": decode, "cpu_baseline": cpu,
+            "clocks": clocks, "timing": timing, "e2e": e2e, "gpu_launches": launches,
+            "roofline": roofline, "decode": decode, "cpu_baseline": cpu,
         }
+        if fused is not None:
+            line["fused_path"] = fused
         if other is not None:
             line["other_workloads"] = other
         print(json.dumps(line))
