@@ -325,9 +325,29 @@ __device__ void wait_slot_free(const FusedArgs& f, const TileDesc& d, const Sche
 // ====================================================================================================
 // intra-chunk engine: 256 threads (te = 0..255), named barrier `bar_id`, 256 TMEM columns at tmem_e
 // ====================================================================================================
-template <bool kHasQ>
+// Stand-alone use (kFused = false, the intra-chunk kernel of the two-kernel schedule): tile number
+// idx of the pass = (chunk of the pass) * H + head goes to position idx of a plain tile array, the
+// engines take the tiles first, first + stride, ...; nothing is waited for or published.
+__device__ bool static_tile(const FusedArgs& f, uint32_t idx, TileDesc* d)
+{
+    d->len = 0;
+    if (idx >= f.n_prod) return false;
+    const uint32_t gl = idx / (uint32_t)f.a.H;
+    const ChunkLoc L = locate_chunk(f.a, f.a.g0 + gl);
+    d->tok0 = L.tok0;
+    d->tile = f.ring + (size_t)idx * tc::TILE_BYTES;
+    d->ready = nullptr;
+    d->ready_val = 0;
+    d->consumed = nullptr;
+    d->need = 0;
+    d->h = (int)(idx - gl * (uint32_t)f.a.H);
+    d->len = L.len;
+    return true;
+}
+
+template <bool kHasQ, bool kFused>
 __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, int bar_id, int te,
-                           const CUtensorMap* tm_k,
+                           uint32_t first, uint32_t stride, const CUtensorMap* tm_k,
                            const CUtensorMap* tm_q, const CUtensorMap* tm_v)
 {
     constexpr bool has_q = kHasQ;
@@ -399,13 +419,20 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
     bool pend_k = false, pend_q = false, pend_v = false;   // (thread 0) requests not yet waited for
     uint32_t tma_parity = 0;
     SchedState ss = {};   // (scheduler thread)
+    uint32_t next_static = first;
+    bool stores_pending = false;   // (bulk thread) the previous tile's staging may still be read out
     int cur = 0;
     unsigned long long* pending_ready = nullptr;   // bulk thread: flag of the tile whose stores are in flight
     unsigned long long pending_val = 0;
 
     if (te == kSchedThread) {
-        ss.pending = tag(f.epoch, fetch_index(f));
-        next_tile(f, ss, &desc[0]);
+        if (kFused) {
+            ss.pending = tag(f.epoch, fetch_index(f));
+            next_tile(f, ss, &desc[0]);
+        } else {
+            static_tile(f, next_static, &desc[0]);
+            next_static += stride;
+        }
     }
     ebar();
     if (desc[0].len > 0 && !*abort_word) {
@@ -435,7 +462,8 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
             for (int e = 0; e < 4; ++e) G[r][e] = fmaf(G[r][e], kLog2e, G[r - 1][e]);
         *reinterpret_cast<float4*>(sTot + warp * kD + d0) =
             make_float4(G[kRPT - 1][0], G[kRPT - 1][1], G[kRPT - 1][2], G[kRPT - 1][3]);
-        if (te == kBulkThread && pending_ready) {
+        if (!kFused && te == kBulkThread && stores_pending) ptx::bulk_wait_read0();   // staging read out
+        if (kFused && te == kBulkThread && pending_ready) {
             // The previous tile is complete in global memory: hand it to the chain roles.  (This also
             // means its W' / U staging has been read out: the buffers are written again below.)  It
             // has to happen before this engine may wait for a ring position: a producer that waits
@@ -448,7 +476,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
 #ifdef KDA_FUSED_TIMING
         const uint64_t ts0_ = te == kSchedThread ? ptx::globaltimer_ns() : 0;
 #endif
-        if (te == kSchedThread) wait_slot_free(f, D, ss, abort_word);
+        if (kFused && te == kSchedThread) wait_slot_free(f, D, ss, abort_word);
 #ifdef KDA_FUSED_TIMING
         if (te == kSchedThread) atomicAdd(&f.hdr->pad[11], (int)((ptx::globaltimer_ns() - ts0_) >> 4));
 #endif
@@ -553,7 +581,14 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                                ptx::umma_desc_sw128(b0 + (k >> 2) * E_KI_HALF + (k & 3) * 32), idesc, k > 0);
             ptx::umma_commit(mma_bar);
         }
-        if (te == kSchedThread) next_tile(f, ss, &desc[cur ^ 1]);
+        if (te == kSchedThread) {
+            if (kFused) {
+                next_tile(f, ss, &desc[cur ^ 1]);
+            } else {
+                static_tile(f, next_static, &desc[cur ^ 1]);
+                next_static += stride;
+            }
+        }
         if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) timed_out = true;
         // Q' and K' have been read out of shared memory by now: Aqk goes over the Q' rows next
         if (te == kBulkThread) ptx::bulk_wait_read0();
@@ -780,6 +815,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
             ptx::bulk_commit();
             pending_ready = D.ready;
             pending_val = D.ready_val;
+            stores_pending = true;
         }
         KT_MARK(te == 0, 8);   // epilogue
 #ifdef KDA_FUSED_TIMING
@@ -793,7 +829,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
     if (out_of_range) atomicOr(&f.hdr->flags, 1);
     if (te == kBulkThread) {
         ptx::bulk_wait_all0();   // shared memory must outlive the reads of every bulk store
-        if (pending_ready && !timed_out && !*abort_word) {
+        if (kFused && pending_ready && !timed_out && !*abort_word) {
             ptx::fence_proxy_async_all();
             ptx::st_release_gpu(pending_ready, pending_val);
         }
@@ -1319,13 +1355,60 @@ kda_fused_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtens
     } else {
         // two engines per CTA
         if (t < kEngThreads)
-            engine_run<kHasQ>(f, smem, tmem_base, 1, t, &tm_k, &tm_q, &tm_v);
+            engine_run<kHasQ, true>(f, smem, tmem_base, 1, t, 0, 0, &tm_k, &tm_q, &tm_v);
         else
-            engine_run<kHasQ>(f, smem + E_BYTES, tmem_base + 256, 2, t - kEngThreads, &tm_k, &tm_q, &tm_v);
+            engine_run<kHasQ, true>(f, smem + E_BYTES, tmem_base + 256, 2, t - kEngThreads, 0, 0, &tm_k, &tm_q, &tm_v);
     }
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 0) ptx::tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ---- the intra-chunk stage alone (first kernel of the two-kernel schedule) --------------------------------
+// Persistent CTAs of one engine each, two per SM; the tiles of the pass go to a plain array.
+template <bool kHasQ>
+__global__ void __launch_bounds__(kEngThreads, 2)
+kda_intra_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtensorMap tm_k,
+             const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_v,
+             int clear_status)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int t = threadIdx.x, warp = t >> 5;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + E_BAR + 32);
+    ptx::grid_dep_launch();   // the inter-chunk kernel may set itself up while this one drains
+    if (clear_status && blockIdx.x == 0 && t == 0) {
+        f.hdr->status = 0;      // (an equal-length call has no prologue kernel to do this)
+        f.hdr->where = 0;
+        f.hdr->flags = 0;
+    }
+    if (t == 0) {
+        uint64_t* mb = reinterpret_cast<uint64_t*>(smem + E_BAR);
+        ptx::mbar_init(mb, 1);       // MMA group complete
+        ptx::mbar_init(mb + 1, 1);   // k landed
+        ptx::mbar_init(mb + 3, 1);   // q landed
+        ptx::mbar_init(mb + 5, 1);   // v landed
+        *reinterpret_cast<volatile uint32_t*>(mb + 2) = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tm_k);
+        ptx::prefetch_tmap(&tm_q);
+        ptx::prefetch_tmap(&tm_v);
+    }
+    if (warp == 0) {
+        ptx::tmem_alloc(tmem_slot, 256);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if ((ptx::smem_u32(smem) & 1023u) != 0) {
+        if (t == 0) report_timeout(f, 90);   // the operand images need 1024-byte alignment
+    } else {
+        engine_run<kHasQ, false>(f, smem, tmem_base, 1, t, blockIdx.x, gridDim.x, &tm_k, &tm_q, &tm_v);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) ptx::tmem_dealloc(tmem_base, 256);
 }
 
 // ---- prologue of a packed batch: status word + production-index base of every round ----------------------
@@ -1423,6 +1506,54 @@ kda_status_t launch_fused_prep(WsHeader* hdr, const int32_t* cu_seqlens, uint32_
 }
 
 // chain CTAs: kSlices per running (sequence, head); at least half of the SMs stay with the engines
+kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, bool clear_status,
+                             cudaStream_t st)
+{
+    int n_sm = 0;
+    {
+        DeviceLock lk;
+        if (!lk.st) return lk.rc;
+        if (!lk.st->attr_done[1]) {
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)E_BYTES));
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)E_BYTES));
+            lk.st->attr_done[1] = true;
+        }
+        if (lk.st->n_sm == 0) {
+            int dev = 0;
+            KDA_CUDA_TRY(cudaGetDevice(&dev));
+            KDA_CUDA_TRY(cudaDeviceGetAttribute(&lk.st->n_sm, cudaDevAttrMultiProcessorCount, dev));
+        }
+        n_sm = lk.st->n_sm;
+    }
+    const int64_t n_tiles = (a.g1 - a.g0) * a.H;
+    if (n_tiles <= 0) return KDA_OK;
+    if (n_tiles > 0x7fffffff || a.total_tokens > 0x7fffffff)
+        return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: more than 2^31 tokens or tiles in one pass");
+    FusedArgs f = {};
+    f.a = a;
+    f.ring = static_cast<char*>(tiles);
+    f.hdr = hdr;
+    f.n_prod = (uint32_t)n_tiles;
+    const bool has_q = a.q != nullptr && a.o != nullptr;
+    CUtensorMap tm_k, tm_q, tm_v;
+    kda_status_t rc = make_tmap(&tm_k, a.k, a.total_tokens, a.H);
+    if (rc == KDA_OK) rc = make_tmap(&tm_v, a.v, a.total_tokens, a.H);
+    if (rc == KDA_OK) rc = make_tmap(&tm_q, has_q ? a.q : a.k, a.total_tokens, a.H);
+    if (rc != KDA_OK) return rc;
+    const int64_t resident = 2 * (int64_t)n_sm;   // two CTAs per SM
+    const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
+    ProfScope ps(PROF_INTRA, st);
+    if (has_q)
+        kda_intra_tc<true><<<grid, kEngThreads, E_BYTES, st>>>(f, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
+    else
+        kda_intra_tc<false><<<grid, kEngThreads, E_BYTES, st>>>(f, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
+    count_launch();
+    KDA_CUDA_TRY(cudaGetLastError());
+    return KDA_OK;
+}
+
 int fused_max_slots(int n_sm) { return n_sm / (2 * kSlices); }
 int fused_slices() { return kSlices; }
 
