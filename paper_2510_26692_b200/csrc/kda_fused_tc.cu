@@ -354,6 +354,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
     constexpr int kNW = 8, kRPT = 8;
     constexpr int kBulkThread = 128;   // lane 0 of warp 4 issues every bulk copy; thread 0 the MMAs
     constexpr int kSchedThread = 32;   // lane 0 of warp 1 finds the next tile
+    constexpr int kMma2Thread = 64;    // lane 0 of warp 2 issues half of the second MMA group
     const ChunkArgs& a = f.a;
     float* sA = reinterpret_cast<float*>(smem + E_A);
     float* sTd = reinterpret_cast<float*>(smem + E_TD);
@@ -523,14 +524,20 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         pend_k = pend_q = false;
         KT_MARK(te == 0, 2);   // prefix + TMA wait
         // ---- gated operands ---------------------------------------------------------------------------
-        {
+        // (two copies of the loop, chosen per warp: without the clamp when no channel of the warp's
+        // share of the tile can reach it, since |G_i - G_m| <= |G_C| / 2)
+        auto gate_rows = [&](auto clamp_tag) {
+            constexpr bool kClamp = decltype(clamp_tag)::value;
             const int hf = c4 >> 4;                       // K-half (channels 0-63 / 64-127)
+            float off[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) off[e] = base[e] - gref[e];
 #pragma unroll
             for (int r = 0; r < kRPT; ++r) {
                 const int i = i0 + r;
-                const uint32_t off = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
-                uint8_t* pk = smem + E_KQ + hf * E_KQ_HALF + off;
-                uint2 k2 = *reinterpret_cast<const uint2*>(smem + E_KS + hf * 8192 + off);
+                const uint32_t o2 = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
+                uint8_t* pk = smem + E_KQ + hf * E_KQ_HALF + o2;
+                uint2 k2 = *reinterpret_cast<const uint2*>(smem + E_KS + hf * 8192 + o2);
                 uint2 q2 = make_uint2(0u, 0u);
                 if (has_q) q2 = *reinterpret_cast<const uint2*>(pk + 8192);
                 if (i >= D.len) k2 = q2 = make_uint2(0u, 0u);
@@ -541,7 +548,8 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                 float okg[4], oqg[4], oki[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const float x = fminf(fmaxf(G[r][e] + base[e] - gref[e], -kClamp2), kClamp2);
+                    float x = G[r][e] + off[e];
+                    if (kClamp) x = fminf(fmaxf(x, -kClamp2), kClamp2);
                     const float e1 = ex2(x);                     // exp(G - G_m)
                     const float e2 = ex2(-x);                    // exp(G_m - G)
                     okg[e] = kf[e] * e1;
@@ -552,9 +560,14 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                 if (has_q)
                     *reinterpret_cast<uint2*>(pk + 8192) =
                         make_uint2(pack_bf16(oqg[0], oqg[1]), pack_bf16(oqg[2], oqg[3]));
-                *reinterpret_cast<uint2*>(smem + E_KI + hf * E_KI_HALF + off) =
+                *reinterpret_cast<uint2*>(smem + E_KI + hf * E_KI_HALF + o2) =
                     make_uint2(pack_bf16(oki[0], oki[1]), pack_bf16(oki[2], oki[3]));
             }
+        };
+        {
+            const bool may_clamp = fminf(fminf(gref[0], gref[1]), fminf(gref[2], gref[3])) < -kClamp2;
+            if (__any_sync(0xffffffffu, may_clamp)) gate_rows(std::true_type{});
+            else gate_rows(std::false_type{});
         }
         ptx::fence_async_smem();
         ptx::tc_fence_before();
@@ -581,6 +594,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                                ptx::umma_desc_sw128(b0 + (k >> 2) * E_KI_HALF + (k & 3) * 32), idesc, k > 0);
             ptx::umma_commit(mma_bar);
         }
+        if (te == kMma2Thread) ptx::umma_commit(mma_bar);   // (the barrier counts both issuing threads)
         if (te == kSchedThread) {
             if (kFused) {
                 next_tile(f, ss, &desc[cur ^ 1]);
@@ -753,11 +767,17 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
             ptx::tc_fence_after();
             const uint32_t idesc = ptx::umma_idesc_bf16(128, 128) | ptx::kIdescBMajorMN;
             const uint32_t m0 = ptx::smem_u32(smem + E_KI);
-            const uint32_t kg0 = ptx::smem_u32(smem + E_KQ), v0 = ptx::smem_u32(smem + E_V);
+            const uint32_t kg0 = ptx::smem_u32(smem + E_KQ);
 #pragma unroll
             for (int k = 0; k < 4; ++k)
                 ptx::umma_bf16(tmem_e, ptx::umma_desc_sw128(m0 + k * 32),
                                ptx::umma_desc_sw128_mn(kg0 + k * 2048, E_KQ_HALF), idesc, k > 0);
+            ptx::umma_commit(mma_bar);
+        }
+        if (te == kMma2Thread) {   // the U half of the group is issued by a second thread at the same time
+            ptx::tc_fence_after();
+            const uint32_t idesc = ptx::umma_idesc_bf16(128, 128) | ptx::kIdescBMajorMN;
+            const uint32_t m0 = ptx::smem_u32(smem + E_KI), v0 = ptx::smem_u32(smem + E_V);
 #pragma unroll
             for (int k = 0; k < 4; ++k)
                 ptx::umma_bf16(tmem_e + 128, ptx::umma_desc_sw128(m0 + k * 32),
@@ -1327,7 +1347,7 @@ kda_fused_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtens
     // barriers of the engines
     if (!chain_cta && (t == 0 || t == kEngThreads)) {
         uint64_t* mb = reinterpret_cast<uint64_t*>(smem + (t ? E_BYTES : 0) + E_BAR);
-        ptx::mbar_init(mb, 1);       // MMA group complete
+        ptx::mbar_init(mb, 2);       // MMA group complete (two issuing threads)
         ptx::mbar_init(mb + 1, 1);   // k landed
         ptx::mbar_init(mb + 3, 1);   // q landed
         ptx::mbar_init(mb + 5, 1);   // v landed
@@ -1383,7 +1403,7 @@ kda_intra_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtens
     }
     if (t == 0) {
         uint64_t* mb = reinterpret_cast<uint64_t*>(smem + E_BAR);
-        ptx::mbar_init(mb, 1);       // MMA group complete
+        ptx::mbar_init(mb, 2);       // MMA group complete (two issuing threads)
         ptx::mbar_init(mb + 1, 1);   // k landed
         ptx::mbar_init(mb + 3, 1);   // q landed
         ptx::mbar_init(mb + 5, 1);   // v landed
