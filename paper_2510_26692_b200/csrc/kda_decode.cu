@@ -120,99 +120,133 @@ kda_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
 // decoding, continuation of a chunked prefill by a few tokens) with the state held in registers
 // across the tokens: it crosses HBM once in each direction per call instead of once per token.
 // Layout: q, k, log_alpha [n_seqs, T, H, 128], v, o [n_seqs, T, H, 128], beta [n_seqs, T, H].
+// Thread layout of the multi-token kernel: warp w owns the 16 state columns 16w..16w+15 for ALL 128
+// dk rows; lane (rg, cg) = (lane >> 2, lane & 3) holds rows rg, rg + 8, ..., rg + 120 and the four
+// columns 16w + 4cg .. +3.  The two column reductions of a token (S^T k and S^T q, over the dk rows)
+// then stay inside the warp: 16 rows in the thread's registers, the 8 row groups by three
+// butterfly shuffles.  No shared-memory reduction and no CTA-wide barrier per token (the
+// single-token kernel keeps its fully coalesced row layout: it has no token loop to protect).
+//
+// The token loop is bound by instruction issue, so a CTA that only started to fetch its state when
+// it began would leave HBM idle while it computes.  CTAs are therefore persistent (two per SM) and
+// fetch the NEXT state into shared memory with asynchronous 16-byte copies while they work on the
+// current one; every thread copies exactly the elements it will own into its own slots, so the
+// hand-over needs no barrier: a thread waits for its own copies only.
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src_gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)),
+                 "l"(src_gmem)
+                 : "memory");
+}
 template <typename T>
 __global__ void __launch_bounds__(256, 2)
 kda_decode_multi_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                         const float* __restrict__ log_alpha, const float* __restrict__ beta, float* S,
-                        const int32_t* __restrict__ slot, T* __restrict__ o, int H, int n_tok, float scale)
+                        const int32_t* __restrict__ slot, T* __restrict__ o, int H, int n_tok, float scale,
+                        int n_items)
 {
     constexpr int GT = 8;   // tokens whose vectors are staged together: one memory latency per group
+    extern __shared__ float4 s_next[];   // [16][256]: the next state, element m of thread t at [m][t]
     __shared__ float s_a[GT][kD], s_k[GT][kD], s_q[GT][kD], s_v[GT][kD];
-    __shared__ float s_b[GT];
-    __shared__ float4 s_red[2][2][8][32];
-    const int item = blockIdx.x;
-    const int n = item / H, h = item - n * H;
+    __shared__ float s_b[GT], s_qk[GT];
     const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
-    const size_t sl = slot ? (size_t)slot[n] : (size_t)n;
-    float* Sp = S + (sl * H + h) * (size_t)(kD * kD) + lane * 4;
+    const int rg = lane >> 2, cg = lane & 3, col = warp * 16 + cg * 4;
 
-    float4 x[16];
+    auto state_of = [&](int item) {
+        const int n = item / H, h = item - n * H;
+        const size_t sl = slot ? (size_t)slot[n] : (size_t)n;
+        return S + (sl * H + h) * (size_t)(kD * kD) + col;
+    };
+    auto fetch = [&](int item) {   // a copy instruction of a warp covers 8 consecutive rows x 64 contiguous bytes
+        const float* Sp = state_of(item);
 #pragma unroll
-    for (int m = 0; m < 16; ++m) x[m] = ld_stream(Sp + (size_t)(warp + 8 * m) * kD);
+        for (int m = 0; m < 16; ++m) cp_async16(&s_next[m * 256 + t], Sp + (size_t)(rg + 8 * m) * kD);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
 
-    auto vec_of = [&](int tt) { return ((size_t)(n * n_tok + tt) * H + h) * kD; };
-    for (int g0 = 0; g0 < n_tok; g0 += GT) {
-        const int gn = (n_tok - g0) < GT ? (n_tok - g0) : GT;
-        __syncthreads();   // the previous group's vectors are no longer read
-        {   // thread (half, c): channel c of tokens half, half + 2, ...  -- all loads first, then the stores
-            const int c = t & (kD - 1), half = t >> 7;
-            float la[GT / 2], kk[GT / 2], qq[GT / 2], vv[GT / 2];
+    int item = blockIdx.x;
+    if (item < n_items) fetch(item);
+    for (; item < n_items; item += gridDim.x) {
+        const int n = item / H, h = item - n * H;
+        float* Sp = state_of(item);
+        float4 x[16];
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
-            for (int j = 0; j < GT / 2; ++j) {
-                const int tok = half + 2 * j;
-                if (tok < gn) {
-                    const size_t vec = vec_of(g0 + tok) + c;
-                    la[j] = log_alpha[vec];
-                    kk[j] = to_f<T>(k[vec]);
-                    qq[j] = to_f<T>(q[vec]);
-                    vv[j] = to_f<T>(v[vec]);
+        for (int m = 0; m < 16; ++m) x[m] = s_next[m * 256 + t];
+        if (item + (int)gridDim.x < n_items) fetch(item + gridDim.x);   // overlaps the token loop below
+
+        auto vec_of = [&](int tt) { return ((size_t)(n * n_tok + tt) * H + h) * kD; };
+        for (int g0 = 0; g0 < n_tok; g0 += GT) {
+            const int gn = (n_tok - g0) < GT ? (n_tok - g0) : GT;
+            __syncthreads();   // the previous group's vectors are no longer read
+            {   // thread (half, c): channel c of tokens half, half + 2, ...  -- all loads first, then the stores
+                const int c = t & (kD - 1), half = t >> 7;
+                float la[GT / 2], kk[GT / 2], qq[GT / 2], vv[GT / 2];
+#pragma unroll
+                for (int j = 0; j < GT / 2; ++j) {
+                    const int tok = half + 2 * j;
+                    if (tok < gn) {
+                        const size_t vec = vec_of(g0 + tok) + c;
+                        la[j] = log_alpha[vec];
+                        kk[j] = to_f<T>(k[vec]);
+                        qq[j] = to_f<T>(q[vec]);
+                        vv[j] = to_f<T>(v[vec]);
+                    }
                 }
-            }
 #pragma unroll
-            for (int j = 0; j < GT / 2; ++j) {
-                const int tok = half + 2 * j;
-                if (tok < gn) {
-                    s_a[tok][c] = expf(la[j]);
-                    s_k[tok][c] = kk[j];
-                    s_q[tok][c] = qq[j];
-                    s_v[tok][c] = vv[j];
+                for (int j = 0; j < GT / 2; ++j) {
+                    const int tok = half + 2 * j;
+                    if (tok < gn) {
+                        s_a[tok][c] = expf(la[j]);
+                        s_k[tok][c] = kk[j];
+                        s_q[tok][c] = qq[j];
+                        s_v[tok][c] = vv[j];
+                    }
                 }
+                if (t < gn) s_b[t] = beta[(size_t)(n * n_tok + g0 + t) * H + h];
             }
-            if (t < gn) s_b[t] = beta[(size_t)(n * n_tok + g0 + t) * H + h];
-        }
-        __syncthreads();
-        for (int tok = 0; tok < gn; ++tok) {
-            const int b = tok & 1;
-            const float bt = s_b[tok];
-            const float4 vv = *reinterpret_cast<const float4*>(&s_v[tok][lane * 4]);
-            float qk = 0.f;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) qk += s_q[tok][lane * 4 + i] * s_k[tok][lane * 4 + i];
-#pragma unroll
-            for (int ofs = 16; ofs > 0; ofs >>= 1) qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
-
-            float4 p = make_float4(0.f, 0.f, 0.f, 0.f), s = p;
-#pragma unroll
-            for (int m = 0; m < 16; ++m) {
-                const int row = warp + 8 * m;
-                mul4(x[m], s_a[tok][row]);
-                fma4(p, s_k[tok][row], x[m]);
-                fma4(s, s_q[tok][row], x[m]);
-            }
-            s_red[b][0][warp][lane] = p;
-            s_red[b][1][warp][lane] = s;
             __syncthreads();
-            p = s_red[b][0][0][lane];
-            s = s_red[b][1][0][lane];
+            if (warp < gn) {   // q.k of token `warp` (4 channels per lane, butterfly reduce)
+                float qk = 0.f;
 #pragma unroll
-            for (int w = 1; w < 8; ++w) {   // fixed order: bitwise reproducible
-                float4 a4 = s_red[b][0][w][lane], b4 = s_red[b][1][w][lane];
-                p.x += a4.x; p.y += a4.y; p.z += a4.z; p.w += a4.w;
-                s.x += b4.x; s.y += b4.y; s.z += b4.z; s.w += b4.w;
-            }
-            const float4 r = make_float4(vv.x - p.x, vv.y - p.y, vv.z - p.z, vv.w - p.w);
-            if (warp == 0) {
-                const float c = bt * qk;
-                IO<T>::store4(o + vec_of(g0 + tok) + lane * 4,
-                              make_float4(scale * (s.x + c * r.x), scale * (s.y + c * r.y),
-                                          scale * (s.z + c * r.z), scale * (s.w + c * r.w)));
-            }
+                for (int i = 0; i < 4; ++i) qk += s_q[warp][lane * 4 + i] * s_k[warp][lane * 4 + i];
 #pragma unroll
-            for (int m = 0; m < 16; ++m) fma4(x[m], bt * s_k[tok][warp + 8 * m], r);
+                for (int ofs = 16; ofs > 0; ofs >>= 1) qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
+                if (lane == 0) s_qk[warp] = qk;
+            }
+            __syncthreads();
+            for (int tok = 0; tok < gn; ++tok) {
+                const float bt = s_b[tok];
+                float4 p = make_float4(0.f, 0.f, 0.f, 0.f), s = p;
+#pragma unroll
+                for (int m = 0; m < 16; ++m) {
+                    const int row = rg + 8 * m;
+                    mul4(x[m], s_a[tok][row]);
+                    fma4(p, s_k[tok][row], x[m]);
+                    fma4(s, s_q[tok][row], x[m]);
+                }
+                // the eight row groups of a column group: lanes that differ in bits 2..4 (fixed order)
+#pragma unroll
+                for (int ofs = 4; ofs < 32; ofs <<= 1) {
+                    p.x += __shfl_xor_sync(0xffffffffu, p.x, ofs); p.y += __shfl_xor_sync(0xffffffffu, p.y, ofs);
+                    p.z += __shfl_xor_sync(0xffffffffu, p.z, ofs); p.w += __shfl_xor_sync(0xffffffffu, p.w, ofs);
+                    s.x += __shfl_xor_sync(0xffffffffu, s.x, ofs); s.y += __shfl_xor_sync(0xffffffffu, s.y, ofs);
+                    s.z += __shfl_xor_sync(0xffffffffu, s.z, ofs); s.w += __shfl_xor_sync(0xffffffffu, s.w, ofs);
+                }
+                const float4 vv = *reinterpret_cast<const float4*>(&s_v[tok][col]);
+                const float4 r = make_float4(vv.x - p.x, vv.y - p.y, vv.z - p.z, vv.w - p.w);
+                if (rg == 0) {
+                    const float c = bt * s_qk[tok];
+                    IO<T>::store4(o + vec_of(g0 + tok) + col,
+                                  make_float4(scale * (s.x + c * r.x), scale * (s.y + c * r.y),
+                                              scale * (s.z + c * r.z), scale * (s.w + c * r.w)));
+                }
+#pragma unroll
+                for (int m = 0; m < 16; ++m) fma4(x[m], bt * s_k[tok][rg + 8 * m], r);
+            }
         }
-    }
 #pragma unroll
-    for (int m = 0; m < 16; ++m) st_stream(Sp + (size_t)(warp + 8 * m) * kD, x[m]);
+        for (int m = 0; m < 16; ++m) st_stream(Sp + (size_t)(rg + 8 * m) * kD, x[m]);
+    }
 }
 
 }  // namespace
@@ -243,16 +277,36 @@ kda_status_t launch_decode_multi(const void* q, const void* k, const void* v, co
                                  int n_tok, int H, float scale, kda_dtype_t dt, cudaStream_t st)
 {
     if (n_seqs == 0 || n_tok == 0) return KDA_OK;
-    const unsigned grid = (unsigned)((size_t)n_seqs * H);
+    constexpr int kNextBytes = 16 * 256 * 16;   // the prefetched state
+    int n_sm = 0;
+    {
+        DeviceLock lk;
+        if (!lk.st) return lk.rc;
+        if (!lk.st->attr_done[6]) {
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_decode_multi_kernel<__nv_bfloat16>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kNextBytes));
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_decode_multi_kernel<float>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kNextBytes));
+            lk.st->attr_done[6] = true;
+        }
+        if (lk.st->n_sm == 0) {
+            int dev = 0;
+            KDA_CUDA_TRY(cudaGetDevice(&dev));
+            KDA_CUDA_TRY(cudaDeviceGetAttribute(&lk.st->n_sm, cudaDevAttrMultiProcessorCount, dev));
+        }
+        n_sm = lk.st->n_sm;
+    }
+    const int n_items = n_seqs * H;
+    const unsigned grid = (unsigned)(n_items < 2 * n_sm ? n_items : 2 * n_sm);   // persistent, two CTAs per SM
     ProfScope ps(PROF_DECODE, st);
     if (dt == KDA_BF16) {
         using T = __nv_bfloat16;
-        kda_decode_multi_kernel<T><<<grid, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v, log_alpha,
-                                                         beta, S, slot, (T*)o, H, n_tok, scale);
+        kda_decode_multi_kernel<T><<<grid, 256, kNextBytes, st>>>((const T*)q, (const T*)k, (const T*)v, log_alpha,
+                                                                  beta, S, slot, (T*)o, H, n_tok, scale, n_items);
     } else {
-        kda_decode_multi_kernel<float><<<grid, 256, 0, st>>>((const float*)q, (const float*)k,
-                                                             (const float*)v, log_alpha, beta, S, slot,
-                                                             (float*)o, H, n_tok, scale);
+        kda_decode_multi_kernel<float><<<grid, 256, kNextBytes, st>>>((const float*)q, (const float*)k,
+                                                                      (const float*)v, log_alpha, beta, S, slot,
+                                                                      (float*)o, H, n_tok, scale, n_items);
     }
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());

@@ -382,7 +382,8 @@ def test_bounded_wait_reports_timeout(oracle_mod):
 @pytest.mark.parametrize("dtype,n_tok", [(torch.bfloat16, 4), (torch.float32, 7), (torch.bfloat16, 16)])
 def test_decode_multi_token(oracle_mod, dtype, n_tok):
     """n_tok tokens per sequence in one call: equals the recurrence over those tokens from the
-    slot's state (oracle), and equals n_tok single-token decode calls bit for bit."""
+    slot's state (oracle), and equals n_tok single-token decode calls up to fp32 rounding (the two
+    kernels sum the dk rows in different orders); run to run it is bit-reproducible."""
     N, H = 6, 3
     d = inputs.decode_inputs(N, H, n_tok, dtype=dtype, seed=36)       # [n_tok, N, H, .]
     dev = "cuda:0"
@@ -405,7 +406,14 @@ def test_decode_multi_token(oracle_mod, dtype, n_tok):
                           N, H, 128, 128, 0.7, dt)
         o1[:, t] = ot
     torch.cuda.synchronize()
-    assert torch.equal(o, o1) and torch.equal(S, S1)
+    assert rel_l2(to_np32(S), to_np32(S1)) <= 1e-6
+    assert rel_l2(to_np32(o), to_np32(o1)) <= (1e-6 if dtype == torch.float32 else 4e-3)
+    S2 = S0.to(dev)
+    o2 = torch.empty_like(o)
+    K.kda_decode_multi(q.to(dev), k.to(dev), v.to(dev), la.to(dev), be.to(dev), S2, slots.to(dev), o2,
+                       N, n_tok, H, 128, 128, 0.7, dt)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o2) and torch.equal(S, S2)
     # oracle: each sequence is n_tok tokens starting from its slot's state
     flat = lambda t: to_np32(t.reshape((N * n_tok,) + tuple(t.shape[2:])))
     cu = np.arange(N + 1, dtype=np.int64) * n_tok
