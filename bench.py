@@ -37,10 +37,11 @@ STATE_BYTES = 2 * D * D * 4
 DEC_BYTES_PER_STATE = 2 * D * D * 4 + 4 * D * 2 + D * 4 + 4
 FLOPS_PER_TOKEN_HEAD = 6 * D * D + 3 * CHUNK * D + CHUNK * CHUNK   # the paper's FLOPs model
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (prefill: intra 168.4 + 99.7 MB, inter 156.3 + 20.1 MB; decode: 547.4 + 484.7 MB)
-PREFILL_DRAM_TRAFFIC = {"intra_chunk": 268.1e6, "inter_chunk": 176.4e6}
+# profiles/ (prefill: intra 168.4 + 98.7 MB, inter 156.3 + 20.0 MB, fused kernel 170.8 + 33.6 MB;
+# decode: 547.4 + 484.7 MB)
+PREFILL_DRAM_TRAFFIC = {"intra_chunk": 267.1e6, "inter_chunk": 176.3e6}
 DECODE_DRAM_TRAFFIC = 1032.1e6
-FUSED_DRAM_TRAFFIC = None
+FUSED_DRAM_TRAFFIC = 204.4e6
 TRAFFIC_SOURCE = "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the summaries under profiles/ (not measured in this run)"
 MIN_TIMED_S = 0.5      # the timed region is extended (whole blocks of `steps` calls) to at least this
 MAX_BLOCKS = 2000
@@ -266,6 +267,11 @@ def main():
     ap.add_argument("--all-workloads", action="store_true",
                     help="also time the packed varlen batch (16 sequences) and the 1 Mi-token "
                          "state-only prefill; needs ~70 GB of device memory")
+    ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S,
+                    help="repeat the block of --steps calls until this much device time is measured "
+                         "(0: one block, for runs under a profiler)")
+    ap.add_argument("--chunk-path", type=int, default=0, choices=[0, 1, 2],
+                    help="kda_set_chunk_path mode for the timed prefill: 0 automatic, 1 two kernels, 2 fused kernel")
     ap.add_argument("--prefill-only", action="store_true",
                     help="time only the device-resident prefill loop (short runs under a profiler)")
     ap.add_argument("--decode-only", action="store_true",
@@ -303,6 +309,7 @@ def main():
 
     if args.decode_only:
         return decode_only(args, K, inputs, torch, dev, peaks)
+    K.kda_set_chunk_path(args.chunk_path)
 
     # ---- prefill workload: 3 input copies (each 206 MB > L2) rotated between steps ---------------
     n_copies = 3
@@ -343,7 +350,7 @@ def main():
         e1.record(stream)
         barrier()
         block_ms.append(max_over_ranks(e0.elapsed_time(e1)))
-        if sum(block_ms) >= MIN_TIMED_S * 1e3 or len(block_ms) >= MAX_BLOCKS:
+        if sum(block_ms) >= args.min_timed_s * 1e3 or len(block_ms) >= MAX_BLOCKS:
             break
     launches = K.kda_launch_count() - l0
     clocks = sampler.finish()
