@@ -137,6 +137,24 @@ __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src_gmem)
                  "l"(src_gmem)
                  : "memory");
 }
+// Dynamic shared memory of the multi-token kernel
+template <typename T> struct MultiSmem {
+    static constexpr int GT = 8;                        // tokens staged together
+    static constexpr int kState = 16 * 256 * 16;        // the prefetched state: element m of thread t at [m][t]
+    static constexpr int kAkq = GT * kD * 16;           // per token and dk row: (alpha, k, q, beta k)
+    static constexpr int kV = GT * kD * 4;
+    static constexpr int kRawA = GT * kD * 4;           // raw log alpha of the next item's first tokens
+    static constexpr int kRawX = GT * kD * (int)sizeof(T);   // raw k / q / v of the same tokens
+    static constexpr int oAkq = kState, oV = oAkq + kAkq, oRawA = oV + kV, oRawK = oRawA + kRawA,
+                         oRawQ = oRawK + kRawX, oRawV = oRawQ + kRawX, oRawB = oRawV + kRawX,
+                         kTotal = oRawB + 64;
+};
+__device__ __forceinline__ void cp_async4b(void* dst_smem, const void* src_gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)),
+                 "l"(src_gmem)
+                 : "memory");
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256, 2)
 kda_decode_multi_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
@@ -144,22 +162,44 @@ kda_decode_multi_kernel(const T* __restrict__ q, const T* __restrict__ k, const 
                         const int32_t* __restrict__ slot, T* __restrict__ o, int H, int n_tok, float scale,
                         int n_items)
 {
-    constexpr int GT = 8;   // tokens whose vectors are staged together: one memory latency per group
-    extern __shared__ float4 s_next[];   // [16][256]: the next state, element m of thread t at [m][t]
-    __shared__ float s_a[GT][kD], s_k[GT][kD], s_q[GT][kD], s_v[GT][kD];
+    using L = MultiSmem<T>;
+    constexpr int GT = L::GT;
+    extern __shared__ __align__(16) unsigned char sm[];
+    float4* s_next = reinterpret_cast<float4*>(sm);
+    float4 (*s_akq)[kD] = reinterpret_cast<float4(*)[kD]>(sm + L::oAkq);
+    float (*s_v)[kD] = reinterpret_cast<float(*)[kD]>(sm + L::oV);
+    float (*r_a)[kD] = reinterpret_cast<float(*)[kD]>(sm + L::oRawA);
+    T (*r_k)[kD] = reinterpret_cast<T(*)[kD]>(sm + L::oRawK);
+    T (*r_q)[kD] = reinterpret_cast<T(*)[kD]>(sm + L::oRawQ);
+    T (*r_v)[kD] = reinterpret_cast<T(*)[kD]>(sm + L::oRawV);
+    float* r_b = reinterpret_cast<float*>(sm + L::oRawB);
     __shared__ float s_b[GT], s_qk[GT];
     const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
     const int rg = lane >> 2, cg = lane & 3, col = warp * 16 + cg * 4;
+    const int gfirst = n_tok < GT ? n_tok : GT;   // tokens of an item's first group
 
     auto state_of = [&](int item) {
         const int n = item / H, h = item - n * H;
         const size_t sl = slot ? (size_t)slot[n] : (size_t)n;
         return S + (sl * H + h) * (size_t)(kD * kD) + col;
     };
-    auto fetch = [&](int item) {   // a copy instruction of a warp covers 8 consecutive rows x 64 contiguous bytes
-        const float* Sp = state_of(item);
+    // Everything the next item needs first -- its state and the vectors of its first tokens -- is
+    // requested with asynchronous copies while the current item is worked on.
+    auto fetch = [&](int item) {
+        const float* Sp = state_of(item);   // a copy instruction of a warp covers 8 consecutive rows x 64 contiguous bytes
 #pragma unroll
         for (int m = 0; m < 16; ++m) cp_async16(&s_next[m * 256 + t], Sp + (size_t)(rg + 8 * m) * kD);
+        const int n = item / H, h = item - n * H;
+        constexpr int CA = kD * 4 / 16, CX = kD * (int)sizeof(T) / 16;   // 16-byte pieces per token
+        for (int idx = t; idx < gfirst * (CA + 3 * CX); idx += 256) {
+            const int tok = idx / (CA + 3 * CX), j = idx - tok * (CA + 3 * CX);
+            const size_t vec = ((size_t)(n * n_tok + tok) * H + h) * kD;
+            if (j < CA) cp_async16(&r_a[tok][j * 4], log_alpha + vec + j * 4);
+            else if (j < CA + CX) cp_async16(&r_k[tok][(j - CA) * (16 / (int)sizeof(T))], k + vec + (j - CA) * (16 / (int)sizeof(T)));
+            else if (j < CA + 2 * CX) cp_async16(&r_q[tok][(j - CA - CX) * (16 / (int)sizeof(T))], q + vec + (j - CA - CX) * (16 / (int)sizeof(T)));
+            else cp_async16(&r_v[tok][(j - CA - 2 * CX) * (16 / (int)sizeof(T))], v + vec + (j - CA - 2 * CX) * (16 / (int)sizeof(T)));
+        }
+        if (t < gfirst) cp_async4b(&r_b[t], beta + (size_t)(n * n_tok + t) * H + h);
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
@@ -171,58 +211,79 @@ kda_decode_multi_kernel(const T* __restrict__ q, const T* __restrict__ k, const 
         float4 x[16];
         asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
-        for (int m = 0; m < 16; ++m) x[m] = s_next[m * 256 + t];
-        if (item + (int)gridDim.x < n_items) fetch(item + gridDim.x);   // overlaps the token loop below
-
+        for (int m = 0; m < 16; ++m) x[m] = s_next[m * 256 + t];   // (each thread reads back its own copies)
+        __syncthreads();   // the raw vectors were copied by other threads; the previous item's vectors are no longer read
         auto vec_of = [&](int tt) { return ((size_t)(n * n_tok + tt) * H + h) * kD; };
         for (int g0 = 0; g0 < n_tok; g0 += GT) {
             const int gn = (n_tok - g0) < GT ? (n_tok - g0) : GT;
-            __syncthreads();   // the previous group's vectors are no longer read
-            {   // thread (half, c): channel c of tokens half, half + 2, ...  -- all loads first, then the stores
+            {   // thread (half, c): channel c of tokens half, half + 2, ...
                 const int c = t & (kD - 1), half = t >> 7;
-                float la[GT / 2], kk[GT / 2], qq[GT / 2], vv[GT / 2];
+                if (g0 == 0) {   // from the prefetched raw vectors
 #pragma unroll
-                for (int j = 0; j < GT / 2; ++j) {
-                    const int tok = half + 2 * j;
-                    if (tok < gn) {
-                        const size_t vec = vec_of(g0 + tok) + c;
-                        la[j] = log_alpha[vec];
-                        kk[j] = to_f<T>(k[vec]);
-                        qq[j] = to_f<T>(q[vec]);
-                        vv[j] = to_f<T>(v[vec]);
+                    for (int j = 0; j < GT / 2; ++j) {
+                        const int tok = half + 2 * j;
+                        if (tok < gn) {
+                            const float kk = to_f<T>(r_k[tok][c]), bb = r_b[tok];
+                            s_akq[tok][c] = make_float4(expf(r_a[tok][c]), kk, to_f<T>(r_q[tok][c]), bb * kk);
+                            s_v[tok][c] = to_f<T>(r_v[tok][c]);
+                            if (c == 0) s_b[tok] = bb;
+                        }
+                    }
+                } else {         // later groups of a long call: straight from global memory, loads first
+                    __syncthreads();   // the previous group's vectors are no longer read
+                    float la[GT / 2], kk[GT / 2], qq[GT / 2], vv[GT / 2], bb[GT / 2];
+#pragma unroll
+                    for (int j = 0; j < GT / 2; ++j) {
+                        const int tok = half + 2 * j;
+                        if (tok < gn) {
+                            const size_t vec = vec_of(g0 + tok) + c;
+                            la[j] = log_alpha[vec];
+                            kk[j] = to_f<T>(k[vec]);
+                            qq[j] = to_f<T>(q[vec]);
+                            vv[j] = to_f<T>(v[vec]);
+                            bb[j] = beta[(size_t)(n * n_tok + g0 + tok) * H + h];
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < GT / 2; ++j) {
+                        const int tok = half + 2 * j;
+                        if (tok < gn) {
+                            s_akq[tok][c] = make_float4(expf(la[j]), kk[j], qq[j], bb[j] * kk[j]);
+                            s_v[tok][c] = vv[j];
+                            if (c == 0) s_b[tok] = bb[j];
+                        }
                     }
                 }
-#pragma unroll
-                for (int j = 0; j < GT / 2; ++j) {
-                    const int tok = half + 2 * j;
-                    if (tok < gn) {
-                        s_a[tok][c] = expf(la[j]);
-                        s_k[tok][c] = kk[j];
-                        s_q[tok][c] = qq[j];
-                        s_v[tok][c] = vv[j];
-                    }
-                }
-                if (t < gn) s_b[t] = beta[(size_t)(n * n_tok + g0 + t) * H + h];
             }
             __syncthreads();
+            // the raw buffers and the state buffer are free: the next item's data may stream in
+            if (g0 == 0 && item + (int)gridDim.x < n_items) fetch(item + gridDim.x);
             if (warp < gn) {   // q.k of token `warp` (4 channels per lane, butterfly reduce)
                 float qk = 0.f;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) qk += s_q[warp][lane * 4 + i] * s_k[warp][lane * 4 + i];
+                for (int i = 0; i < 4; ++i) {
+                    const float4 e = s_akq[warp][lane * 4 + i];
+                    qk += e.z * e.y;
+                }
 #pragma unroll
                 for (int ofs = 16; ofs > 0; ofs >>= 1) qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
                 if (lane == 0) s_qk[warp] = qk;
             }
             __syncthreads();
             for (int tok = 0; tok < gn; ++tok) {
-                const float bt = s_b[tok];
                 float4 p = make_float4(0.f, 0.f, 0.f, 0.f), s = p;
 #pragma unroll
-                for (int m = 0; m < 16; ++m) {
-                    const int row = rg + 8 * m;
-                    mul4(x[m], s_a[tok][row]);
-                    fma4(p, s_k[tok][row], x[m]);
-                    fma4(s, s_q[tok][row], x[m]);
+                for (int m4 = 0; m4 < 16; m4 += 4) {
+                    float4 e[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) e[j] = s_akq[tok][rg + 8 * (m4 + j)];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        mul4(x[m4 + j], e[j].x);
+                        fma4(p, e[j].y, x[m4 + j]);
+                        fma4(s, e[j].z, x[m4 + j]);
+                    }
+                    asm volatile("" ::: "memory");   // keeps the loads of later rows from being hoisted (registers)
                 }
                 // the eight row groups of a column group: lanes that differ in bits 2..4 (fixed order)
 #pragma unroll
@@ -235,13 +296,20 @@ kda_decode_multi_kernel(const T* __restrict__ q, const T* __restrict__ k, const 
                 const float4 vv = *reinterpret_cast<const float4*>(&s_v[tok][col]);
                 const float4 r = make_float4(vv.x - p.x, vv.y - p.y, vv.z - p.z, vv.w - p.w);
                 if (rg == 0) {
-                    const float c = bt * s_qk[tok];
+                    const float c = s_b[tok] * s_qk[tok];
                     IO<T>::store4(o + vec_of(g0 + tok) + col,
                                   make_float4(scale * (s.x + c * r.x), scale * (s.y + c * r.y),
                                               scale * (s.z + c * r.z), scale * (s.w + c * r.w)));
                 }
 #pragma unroll
-                for (int m = 0; m < 16; ++m) fma4(x[m], bt * s_k[tok][rg + 8 * m], r);
+                for (int m4 = 0; m4 < 16; m4 += 4) {
+                    float bk[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) bk[j] = s_akq[tok][rg + 8 * (m4 + j)].w;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) fma4(x[m4 + j], bk[j], r);
+                    asm volatile("" ::: "memory");
+                }
             }
         }
 #pragma unroll
@@ -277,16 +345,17 @@ kda_status_t launch_decode_multi(const void* q, const void* k, const void* v, co
                                  int n_tok, int H, float scale, kda_dtype_t dt, cudaStream_t st)
 {
     if (n_seqs == 0 || n_tok == 0) return KDA_OK;
-    constexpr int kNextBytes = 16 * 256 * 16;   // the prefetched state
     int n_sm = 0;
     {
         DeviceLock lk;
         if (!lk.st) return lk.rc;
         if (!lk.st->attr_done[6]) {
             KDA_CUDA_TRY(cudaFuncSetAttribute(kda_decode_multi_kernel<__nv_bfloat16>,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kNextBytes));
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              MultiSmem<__nv_bfloat16>::kTotal));
             KDA_CUDA_TRY(cudaFuncSetAttribute(kda_decode_multi_kernel<float>,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kNextBytes));
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              MultiSmem<float>::kTotal));
             lk.st->attr_done[6] = true;
         }
         if (lk.st->n_sm == 0) {
@@ -301,10 +370,10 @@ kda_status_t launch_decode_multi(const void* q, const void* k, const void* v, co
     ProfScope ps(PROF_DECODE, st);
     if (dt == KDA_BF16) {
         using T = __nv_bfloat16;
-        kda_decode_multi_kernel<T><<<grid, 256, kNextBytes, st>>>((const T*)q, (const T*)k, (const T*)v, log_alpha,
+        kda_decode_multi_kernel<T><<<grid, 256, MultiSmem<T>::kTotal, st>>>((const T*)q, (const T*)k, (const T*)v, log_alpha,
                                                                   beta, S, slot, (T*)o, H, n_tok, scale, n_items);
     } else {
-        kda_decode_multi_kernel<float><<<grid, 256, kNextBytes, st>>>((const float*)q, (const float*)k,
+        kda_decode_multi_kernel<float><<<grid, 256, MultiSmem<float>::kTotal, st>>>((const float*)q, (const float*)k,
                                                                       (const float*)v, log_alpha, beta, S, slot,
                                                                       (float*)o, H, n_tok, scale, n_items);
     }
