@@ -509,7 +509,11 @@ def test_gate_range_stress_and_flag(oracle_mod):
 
 
 @pytest.mark.parametrize("lens,H", [([4096], 32), ([300, 77, 1, 640], 4), ([512, 2000, 100], 32),
-                                    ([100, 0, 300, 64, 65], 8), ([1000], 2)])
+                                    ([100, 0, 300, 64, 65], 8), ([1000], 2),
+                                    # several sequences of different lengths per round (indices without a tile)
+                                    ([100, 700, 64, 300, 1, 900, 250, 130, 65, 0, 410], 5),
+                                    # more heads than chain slots: a sequence's heads spread over rounds
+                                    ([300, 200], 40)])
 def test_fused_kernel_matches_two_kernel_path(oracle_mod, lens, H):
     """The fused cooperative kernel (engines + chains in one launch, tiles through a ring in L2)
     and the two-kernel schedule do the same arithmetic per tile: bit-identical results, for one
