@@ -248,6 +248,19 @@ kda_status_t kda_profile_read(int kind, double *total_ms, int *launches);
  */
 int kda_selftest_device_table(void);
 
+/*
+ * The schedule that the fused bf16 prefill kernel of kda_chunk_fwd would use for a batch whose
+ * sequence n has chunks_per_seq[n] chunks (HOST array of n_seqs entries), with H heads, room for
+ * avail_tiles tiles in the workspace and n_sm multiprocessors: out[0] = Q, the (sequence, head)
+ * chains that run side by side in one round; out[1] = R, the tiles per chain that the intra-chunk
+ * stage (Section 3.1, the WY / UT part) may run ahead of the state recurrence; out[2] = rounds;
+ * out[3] = production indices handed out in total (a round takes its longest chain times its number
+ * of chains).  Host arithmetic only: no CUDA call, runs without a GPU.  Returns 0, or 1 on a bad
+ * argument; Q = 0 in out[] means that no schedule exists (fewer than two tiles, or too few SMs).
+ */
+int kda_selftest_fused_plan(const int32_t *chunks_per_seq, int n_seqs, int H, int64_t avail_tiles,
+                            int n_sm, int64_t out[4]);
+
 /* Description of the calling thread's last error ("" if none); static storage, never NULL. */
 const char *kda_last_error(void);
 

@@ -2,11 +2,13 @@
 // of the computation runs in the kernels of the other translation units; this file only decides
 // what to launch.
 #include <atomic>
+#include <chrono>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <random>
 #include <vector>
 
 #include "kda_common.cuh"
@@ -134,7 +136,49 @@ FusedLayout fused_layout(int64_t J)
     L.off_ring = L.off_table + align_up((size_t)(J + 1) * sizeof(uint32_t));
     return L;
 }
-std::atomic<uint32_t> g_epoch{0};
+// Call counter that tags the flag words of the fused kernel.  It starts at a value drawn per process:
+// device memory handed from one process to the next may still hold the flag words of the earlier
+// one, and a counter that restarted at 1 could meet its own tags there.
+uint32_t epoch_seed()
+{
+    std::random_device rd;
+    const uint64_t t = (uint64_t)std::chrono::steady_clock::now().time_since_epoch().count();
+    return (uint32_t)rd() ^ (uint32_t)(t * 0x9E3779B97F4A7C15ull >> 32);
+}
+std::atomic<uint32_t> g_epoch{epoch_seed()};
+
+// Schedule of the fused kernel: Q chains run side by side (one round), each with a ring of R tiles;
+// n_prod counts the production indices, a round taking (longest chain) x (chains of the round).
+struct FusedPlan {
+    int64_t Q, R, n_rounds;
+    uint64_t n_prod;
+};
+FusedPlan fused_plan(const std::vector<int64_t>& chunk_cu, int n_seqs, int H, int64_t avail_tiles, int n_sm)
+{
+    FusedPlan P{0, 0, 0, 0};
+    const int64_t J = (int64_t)n_seqs * H;
+    int Qmax = fused_max_slots(n_sm);
+    if (Qmax > kSlotCap) Qmax = kSlotCap;
+    if (Qmax < 1 || avail_tiles < 2 || J < 1) return P;
+    // whole sequences per round when the heads of one fit, so that the chains of a round have
+    // equal lengths
+    int64_t Q = (H <= Qmax) ? (int64_t)H * (Qmax / H) : Qmax;
+    if (Q > J) Q = J;
+    if (Q * 2 > avail_tiles) Q = avail_tiles / 2;
+    int64_t R = avail_tiles / Q;
+    if (R > kRingMax) R = kRingMax;
+    P.Q = Q; P.R = R; P.n_rounds = (J + Q - 1) / Q;
+    for (int64_t r = 0; r < P.n_rounds; ++r) {
+        const int64_t j0 = r * Q, j1 = (j0 + Q < J ? j0 + Q : J) - 1;
+        int64_t maxlen = 0;
+        for (int64_t n = j0 / H; n <= j1 / H; ++n) {
+            const int64_t len = chunk_cu[n + 1] - chunk_cu[n];
+            maxlen = len > maxlen ? len : maxlen;
+        }
+        P.n_prod += (uint64_t)maxlen * (uint64_t)(j1 - j0 + 1);
+    }
+    return P;
+}
 std::atomic<int> g_chunk_path{0};   // 0 = automatic, 1 = always two kernels, 2 = always the fused kernel
 
 }  // namespace
@@ -164,6 +208,17 @@ int kda_selftest_device_table(void)
     s1->attr_done[5] = false;
     if (!g_dev_mu.try_lock()) return 5;     // (not held by this thread)
     g_dev_mu.unlock();
+    return 0;
+}
+
+int kda_selftest_fused_plan(const int32_t* chunks_per_seq, int n_seqs, int H, int64_t avail_tiles,
+                            int n_sm, int64_t out[4])
+{
+    if (!chunks_per_seq || !out || n_seqs < 1 || H < 1) return 1;
+    std::vector<int64_t> chunk_cu((size_t)n_seqs + 1, 0);
+    for (int n = 0; n < n_seqs; ++n) chunk_cu[n + 1] = chunk_cu[n] + chunks_per_seq[n];
+    const FusedPlan P = fused_plan(chunk_cu, n_seqs, H, avail_tiles, n_sm);
+    out[0] = P.Q; out[1] = P.R; out[2] = P.n_rounds; out[3] = (int64_t)P.n_prod;
     return 0;
 }
 
@@ -299,27 +354,10 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
             n_sm = lk.st->n_sm;
         }
         const int64_t avail = (int64_t)((workspace_bytes - FL.off_ring) / tbf);
-        int Qmax = fused_max_slots(n_sm);
-        if (Qmax > kSlotCap) Qmax = kSlotCap;
-        if (Qmax < 1) return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: the device has too few SMs");
-        // whole sequences per round when the heads of one fit, so that the chains of a round have
-        // equal lengths
-        int64_t Q = (H <= Qmax) ? (int64_t)H * (Qmax / H) : Qmax;
-        if (Q > J) Q = J;
-        if (Q * 2 > avail) Q = avail / 2;
-        int64_t R = avail / Q;
-        if (R > kRingMax) R = kRingMax;
-        const int64_t n_rounds = (J + Q - 1) / Q;
-        uint64_t n_prod = 0;
-        for (int64_t r = 0; r < n_rounds; ++r) {
-            const int64_t j0 = r * Q, j1 = (j0 + Q < J ? j0 + Q : J) - 1;
-            int64_t maxlen = 0;
-            for (int64_t n = j0 / H; n <= j1 / H; ++n) {
-                const int64_t len = chunk_cu[n + 1] - chunk_cu[n];
-                maxlen = len > maxlen ? len : maxlen;
-            }
-            n_prod += (uint64_t)maxlen * (uint64_t)(j1 - j0 + 1);
-        }
+        const FusedPlan P = fused_plan(chunk_cu, n_seqs, H, avail, n_sm);
+        if (P.Q < 1) return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: the device has too few SMs");
+        const int64_t Q = P.Q, R = P.R, n_rounds = P.n_rounds;
+        const uint64_t n_prod = P.n_prod;
         if (n_prod > 0x7fffffffull)
             return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: too many (chunk, head) tiles in one call");
         FusedArgs f;

@@ -115,3 +115,52 @@ def test_chunk_path_switch(lib):
     for mode in (2, 1, 0):
         K.kda_set_chunk_path(mode)
     assert lib.kda_set_chunk_path(3) == 1 and lib.kda_set_chunk_path(-1) == 1
+
+
+def _plan(lib, chunks, H, avail, n_sm):
+    arr = (ctypes.c_int32 * len(chunks))(*chunks)
+    out = (ctypes.c_int64 * 4)()
+    lib.kda_selftest_fused_plan.restype = ctypes.c_int
+    lib.kda_selftest_fused_plan.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                            ctypes.c_int64, ctypes.c_int, ctypes.c_void_p]
+    rc = lib.kda_selftest_fused_plan(ctypes.cast(arr, ctypes.c_void_p), len(chunks), H, avail, n_sm,
+                                     ctypes.cast(out, ctypes.c_void_p))
+    assert rc == 0
+    return tuple(out)
+
+
+def test_fused_schedule_plan(lib):
+    """Host side of the fused prefill kernel: how many (sequence, head) chains run side by side, how
+    deep their tile rings are, and how many production indices the call hands out.  Checked against
+    the constraints the kernel relies on and against a count by enumeration."""
+    import random
+    rng = random.Random(7)
+    cases = [([64], 32, 1024, 148), ([3, 11, 1, 5, 0, 14, 4, 3, 2, 0, 7], 5, 40, 148),
+             ([5, 4], 40, 1024, 148), ([1], 1, 2, 148), ([9] * 7, 3, 7, 148), ([2, 2], 2, 1000, 8)]
+    for _ in range(200):
+        n = rng.randint(1, 12)
+        cases.append(([rng.randint(0, 20) for _ in range(n)], rng.randint(1, 70),
+                      rng.randint(2, 1200), rng.choice([4, 16, 132, 148, 160, 400])))
+    for chunks, H, avail, n_sm in cases:
+        Q, R, n_rounds, n_prod = _plan(lib, chunks, H, avail, n_sm)
+        J = len(chunks) * H
+        q_max = min(n_sm // 4, 64)          # two CTAs per chain, as many CTAs again for the tiles
+        assert 1 <= Q <= min(J, q_max), (chunks, H, avail, n_sm, Q)
+        assert 2 <= R <= 16 and Q * R <= avail          # the rings fit the workspace
+        assert n_rounds == -(-J // Q)
+        if H <= q_max and Q * 2 <= avail and Q < J and (H * (q_max // H)) * 2 <= avail:
+            assert Q % H == 0                           # whole sequences per round
+        # enumeration: every round takes (its longest chain) x (its chains) indices, and each
+        # (chain, chunk) pair of the batch gets exactly one of them
+        total, tiles = 0, 0
+        for r in range(n_rounds):
+            js = range(r * Q, min((r + 1) * Q, J))
+            longest = max(chunks[j // H] for j in js)
+            for c in range(longest):
+                for j in js:
+                    total += 1
+                    tiles += c < chunks[j // H]
+        assert total == n_prod and tiles == sum(chunks) * H
+    # no schedule: fewer than two tiles of room, or a device with fewer than four SMs
+    assert _plan(lib, [4], 2, 1, 148)[0] == 0
+    assert _plan(lib, [4], 2, 64, 3)[0] == 0
