@@ -4,6 +4,8 @@ A plain, slow CPU statement of what the KDA hot path computes, in fp64:
 
 * ``recurrence`` / ``decode_step`` call ``kda_oracle.c``, the token-by-token recurrence of
   Section 3, Eq. 1 of the Kimi Linear paper.  This is the oracle.
+* ``dplr_recurrence`` is the general diagonal-plus-low-rank recurrence of Section 6.1 ("Relation
+  to DPLR"), the paper's comparison workload, in the same plain form (``kda_oracle.c``).
 * ``chunkwise.chunk_kda_np`` is a second, independent numpy statement of the chunkwise algorithm of
   Section 3.1 (WY representation + UT transform + chunk state update + output equation).  It is a
   cross-check of the oracle, not the oracle.
@@ -55,6 +57,11 @@ def _load():
                 f32p, f32p, f32p, f32p, f32p, f64p, ctypes.POINTER(ctypes.c_int32), f64p,
                 ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double,
                 ctypes.c_int]
+            lib.kda_oracle_dplr_recurrence.restype = ctypes.c_int
+            lib.kda_oracle_dplr_recurrence.argtypes = [
+                f32p, f32p, f32p, f32p, f32p, f32p, f64p, f64p, f64p,
+                ctypes.POINTER(ctypes.c_int64), ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                ctypes.c_int, ctypes.c_double, ctypes.c_int]
             lib.kda_oracle_max_threads.restype = ctypes.c_int
             _lib = lib
     return _lib
@@ -115,6 +122,46 @@ def recurrence(q, k, v, log_alpha, beta, S0=None, cu_seqlens=None, scale=1.0,
         _ptr(cu, ctypes.c_int64), N, H, dk, dv, float(scale), int(n_threads))
     if rc != 0:
         raise RuntimeError("kda_oracle_recurrence failed")
+    return o, S_T
+
+
+def dplr_recurrence(q, k, v, a, b, g, S0=None, cu_seqlens=None, scale=1.0, want_o=True,
+                    want_state=True, n_threads=0):
+    """The general diagonal-plus-low-rank recurrence (Section 6.1, "Relation to DPLR") token by
+    token in fp64:  S_t = (Diag(exp(g_t)) + b_t a_t^T) S_{t-1} + k_t v_t^T,  o_t = scale S_t^T q_t.
+
+    q, k, a, b, g: [T,H,dk]; v: [T,H,dv]; S0: [N,H,dk,dv] or None; cu_seqlens as in
+    ``recurrence``.  Returns (o or None, S_T or None) in fp64.
+    """
+    k = _f32(k)
+    T, H, dk = k.shape
+    v = _f32(v)
+    dv = v.shape[-1]
+    q = _f32(q, (T, H, dk)) if q is not None else None
+    a = _f32(a, (T, H, dk))
+    b = _f32(b, (T, H, dk))
+    g = _f32(g, (T, H, dk))
+    if cu_seqlens is None:
+        cu = np.array([0, T], dtype=np.int64)
+    else:
+        cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int64))
+        assert cu[0] == 0 and cu[-1] == T and np.all(np.diff(cu) >= 0)
+    N = cu.shape[0] - 1
+    S0a = None
+    if S0 is not None:
+        S0a = np.ascontiguousarray(np.asarray(S0, dtype=np.float64))
+        assert S0a.shape == (N, H, dk, dv)
+    if want_o:
+        assert q is not None
+    o = np.empty((T, H, dv), dtype=np.float64) if want_o else None
+    S_T = np.empty((N, H, dk, dv), dtype=np.float64) if want_state else None
+    rc = _load().kda_oracle_dplr_recurrence(
+        _ptr(q, ctypes.c_float), _ptr(k, ctypes.c_float), _ptr(v, ctypes.c_float),
+        _ptr(a, ctypes.c_float), _ptr(b, ctypes.c_float), _ptr(g, ctypes.c_float),
+        _ptr(S0a, ctypes.c_double), _ptr(o, ctypes.c_double), _ptr(S_T, ctypes.c_double),
+        _ptr(cu, ctypes.c_int64), N, H, dk, dv, float(scale), int(n_threads))
+    if rc != 0:
+        raise RuntimeError("kda_oracle_dplr_recurrence failed")
     return o, S_T
 
 

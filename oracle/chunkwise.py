@@ -54,3 +54,51 @@ def chunk_kda_np(q, k, v, log_alpha, beta, S0=None, chunk=64, scale=1.0):
             S = np.exp(G[-1])[:, None] * S + (np.exp(G[-1][None, :] - G) * K).T @ Vn
         S_T[h] = S
     return o, S_T
+
+
+def chunk_dplr_np(q, k, v, a, b, g, S0=None, chunk=64, scale=1.0):
+    """Chunkwise form of the general diagonal-plus-low-rank recurrence (Section 6.1, "Relation to
+    DPLR"; the structure of the paper's chunkwise DPLR pseudo-code), one sequence, numpy fp64.  A
+    cross-check of ``dplr_recurrence``, not the oracle.
+
+    With G the cumulative log-decay inside the chunk, x_i = S_{i-1}^T a_i the contraction of a with
+    the state before token i, and S the state entering the chunk:
+
+      * four gated Gram matrices, the row factor of a stopping one token early:
+        Aab[i,j] = sum_d a_i exp(G_{i-1} - G_j) b_j,  Aak likewise with k_j      (j < i)
+        Aqb[i,j] = sum_d q_i exp(G_i - G_j) b_j,      Aqk likewise with k_j      (j <= i);
+      * X = (I - Aab)^-1 (Atil S + Aak V)  with  Atil_i = a_i exp(G_{i-1}), i.e. X = u + w S;
+      * O = (q . exp(G)) S + Aqb X + Aqk V;
+      * S <- Diag(exp(G_C)) S + (k . exp(G_C - G))^T V + (b . exp(G_C - G))^T X.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
+    T, H, dk = k.shape
+    dv = v.shape[-1]
+    o = np.zeros((T, H, dv))
+    S_T = np.zeros((H, dk, dv))
+    for h in range(H):
+        S = np.zeros((dk, dv)) if S0 is None else np.array(S0[h], dtype=np.float64)
+        for c0 in range(0, T, chunk):
+            c1 = min(T, c0 + chunk)
+            L = c1 - c0
+            Q, K, V = q[c0:c1, h] * scale, k[c0:c1, h], v[c0:c1, h]
+            A, B, gg = a[c0:c1, h], b[c0:c1, h], g[c0:c1, h]
+            G = np.cumsum(gg, axis=0)
+            Gm = G - gg                                            # G_{i-1}
+            Dq = np.exp(np.clip(G[:, None, :] - G[None, :, :], None, 0.0))     # exp(G_i - G_j), j <= i
+            Da = np.exp(np.clip(Gm[:, None, :] - G[None, :, :], None, 0.0))    # exp(G_{i-1} - G_j), j < i
+            Aqk = np.tril(np.einsum("id,jd,ijd->ij", Q, K, Dq))
+            Aqb = np.tril(np.einsum("id,jd,ijd->ij", Q, B, Dq))
+            Aab = np.tril(np.einsum("id,jd,ijd->ij", A, B, Da), -1)
+            Aak = np.tril(np.einsum("id,jd,ijd->ij", A, K, Da), -1)
+            X = np.linalg.solve(np.eye(L) - Aab, (A * np.exp(Gm)) @ S + Aak @ V)
+            o[c0:c1, h] = (Q * np.exp(G)) @ S + Aqb @ X + Aqk @ V
+            dec = np.exp(G[-1][None, :] - G)
+            S = np.exp(G[-1])[:, None] * S + (K * dec).T @ V + (B * dec).T @ X
+        S_T[h] = S
+    return o, S_T

@@ -151,6 +151,87 @@ int kda_oracle_decode_step(const float *q, const float *k, const float *v, const
     return failed ? -1 : 0;
 }
 
+/*
+ * General diagonal-plus-low-rank recurrence (Section 3.2 and Section 6.1, "Relation to DPLR"), the
+ * comparison workload of the paper's kernel-time figure.  Per sequence and head, with S a dk x dv
+ * matrix, g the per-channel log-decay and a, b the two low-rank vectors:
+ *
+ *     S_t = (Diag(exp(g_t)) + b_t a_t^T) S_{t-1} + k_t v_t^T ,      o_t = scale * S_t^T q_t
+ *
+ * i.e. a_t is contracted with the state as the previous token left it (x = S_{t-1}^T a_t), and the
+ * state then receives the decay, the rank-one term b_t x^T and the new key/value pair.  This is the
+ * reading of the paper's chunkwise DPLR pseudo-code taken here: its decay factor between the row of
+ * a and the column of b or k stops one token before the row, and its state update adds b-weighted
+ * and k-weighted terms.  With a = alpha . k, b = -beta k and the key replaced by beta k it is Eq. 1
+ * (the correspondence the paper states, up to the sign convention of the low-rank term).
+ *
+ * Layouts as above; a, b, g are [T_total,H,dk].
+ */
+int kda_oracle_dplr_recurrence(const float *q, const float *k, const float *v, const float *a,
+                               const float *b, const float *g, const double *S0, double *o,
+                               double *S_T, const int64_t *cu_seqlens, int n_seqs, int H, int dk,
+                               int dv, double scale, int n_threads)
+{
+    if (!k || !v || !a || !b || !g || !cu_seqlens || n_seqs < 0 || H <= 0 || dk <= 0 || dv <= 0)
+        return -1;
+    if (o && !q) return -1;
+    int failed = 0;
+    long n_items = (long)n_seqs * H;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+    (void)n_threads;
+#endif
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long item = 0; item < n_items; ++item) {
+        int n = (int)(item / H), h = (int)(item % H);
+        double *S = (double *)malloc(sizeof(double) * dk * dv);
+        double *x = (double *)malloc(sizeof(double) * dv);
+        if (!S || !x) {
+            failed = 1;
+            free(S);
+            free(x);
+            continue;
+        }
+        size_t sofs = ((size_t)n * H + h) * dk * dv;
+        if (S0) memcpy(S, S0 + sofs, sizeof(double) * dk * dv);
+        else memset(S, 0, sizeof(double) * dk * dv);
+        for (int64_t t = cu_seqlens[n]; t < cu_seqlens[n + 1]; ++t) {
+            size_t th = (size_t)t * H + h;
+            const float *at = a + th * dk, *bt = b + th * dk, *gt = g + th * dk, *kt = k + th * dk;
+            const float *vt = v + th * dv;
+            /* x = S_{t-1}^T a_t */
+            for (int j = 0; j < dv; ++j) x[j] = 0.0;
+            for (int i = 0; i < dk; ++i) {
+                double ai = (double)at[i];
+                const double *Si = S + (size_t)i * dv;
+                for (int j = 0; j < dv; ++j) x[j] += ai * Si[j];
+            }
+            /* S_t = Diag(exp(g_t)) S_{t-1} + b_t x^T + k_t v_t^T */
+            for (int i = 0; i < dk; ++i) {
+                double d = exp((double)gt[i]), bi = (double)bt[i], ki = (double)kt[i];
+                double *Si = S + (size_t)i * dv;
+                for (int j = 0; j < dv; ++j) Si[j] = d * Si[j] + bi * x[j] + ki * (double)vt[j];
+            }
+            if (o) {
+                const float *qt = q + th * dk;
+                double *ot = o + th * dv;
+                for (int j = 0; j < dv; ++j) ot[j] = 0.0;
+                for (int i = 0; i < dk; ++i) {
+                    double qi = (double)qt[i];
+                    const double *Si = S + (size_t)i * dv;
+                    for (int j = 0; j < dv; ++j) ot[j] += qi * Si[j];
+                }
+                for (int j = 0; j < dv; ++j) ot[j] *= scale;
+            }
+        }
+        if (S_T) memcpy(S_T + sofs, S, sizeof(double) * dk * dv);
+        free(S);
+        free(x);
+    }
+    return failed ? -1 : 0;
+}
+
 int kda_oracle_max_threads(void)
 {
 #ifdef _OPENMP

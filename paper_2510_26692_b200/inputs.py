@@ -16,7 +16,8 @@ from typing import Dict, Optional, Sequence
 
 import torch
 
-_ORDER = {"q": 0, "k": 1, "v": 2, "x": 3, "beta": 4, "S0": 5, "S": 6, "lens": 7}
+_ORDER = {"q": 0, "k": 1, "v": 2, "x": 3, "beta": 4, "S0": 5, "S": 6, "lens": 7, "a": 8, "b": 9, "eta": 10,
+          "do": 11, "dS": 12}
 
 
 def _gen(seed: int, name: str, device) -> torch.Generator:
@@ -122,4 +123,33 @@ def decode_inputs(n_seqs: int, H: int, steps: int, dk: int = 128, dv: int = 128,
     out["log_alpha"] = torch.nn.functional.logsigmoid(x)
     out["beta"] = torch.sigmoid(_randn((steps, n_seqs, H), seed, "beta", device))
     out["S"] = _randn((n_seqs, H, dk, dv), seed, "S", device) * s_std
+    return out
+
+
+def dplr_inputs(lengths: Sequence[int], H: int, dk: int = 128, dv: int = 128, seed: int = 0,
+                gate_mean: float = 4.0, s0_std: float = 0.0, device="cpu") -> Dict[str, Optional[torch.Tensor]]:
+    """Inputs of one call of the general diagonal-plus-low-rank workload (the paper's comparison
+    kernel): q, k, v, the decay g = logsigmoid(N(gate_mean, 1)) as in ``chunk_inputs``, and two
+    independent low-rank vectors: a = a unit vector times a factor in (0.5, 1), b = minus another
+    unit vector (correlated with a's) times a factor in (0, 1), so that the transition
+    Diag(exp(g)) + b a^T stays close to a contraction and long sequences neither blow up nor die
+    out.  Everything fp32.
+    """
+    T = int(sum(lengths))
+    N = len(lengths)
+    out: Dict[str, Optional[torch.Tensor]] = {}
+    out["q"] = _l2norm(_randn((T, H, dk), seed, "q", device)) * (dk ** -0.5)
+    out["k"] = _l2norm(_randn((T, H, dk), seed, "k", device))
+    out["v"] = _randn((T, H, dv), seed, "v", device)
+    x = _randn((T, H, dk), seed, "x", device)
+    x += gate_mean
+    out["g"] = torch.nn.functional.logsigmoid(x)
+    del x
+    ra = _randn((T, H, dk), seed, "a", device)
+    rb = _randn((T, H, dk), seed, "b", device)
+    eta = torch.sigmoid(_randn((T, H, 2), seed, "eta", device))
+    out["a"] = _l2norm(ra) * (0.5 + 0.5 * eta[..., 0:1])
+    out["b"] = -_l2norm(ra + 0.5 * rb) * eta[..., 1:2]
+    out["S0"] = (_randn((N, H, dk, dv), seed, "S0", device) * s0_std) if s0_std > 0 else None
+    out["cu_seqlens"] = cu_seqlens_of(lengths)
     return out
