@@ -230,6 +230,66 @@ def extra_workloads(K, inputs, torch, dev, peaks):
     return out
 
 
+def dplr_comparison(K, inputs, torch, dev, peaks):
+    """The paper's one kernel-level experiment (Section 3.2 kernel-time figure; Section 6.1): the
+    general diagonal-plus-low-rank chunk forward against KDA at batch 1, 16 heads.  Both in the
+    library's fp32 FMA style (same chunk length, same two-kernel structure), so the ratio shows what
+    binding a and b to k saves; the tensor-core bf16 KDA path is listed beside them."""
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps=5):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    T, Hh = 16384, 16
+    out = {"workload": "B=1, T=16384, H=16, dk=dv=128, chunk=64 (inputs 134 MB per tensor > L2); paper figure: "
+                       "DPLR 14.89 ms / KDA 7.60 ms = 1.96 at this length (other hardware)"}
+    d = inputs.dplr_inputs([T], H=Hh, seed=5, s0_std=0.02, device=dev)
+    nb = K.kda_dplr_chunk_fwd_workspace_bytes(T, 1, Hh)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    o = torch.empty((T, Hh, D), dtype=torch.float32, device=dev)
+    S_T = torch.empty((1, Hh, D, D), dtype=torch.float32, device=dev)
+    ms_dplr = timed(lambda: K.kda_dplr_chunk_fwd(d["q"], d["k"], d["v"], d["a"], d["b"], d["g"], d["S0"], o, S_T,
+                                                 None, None, 1, T, Hh, D, D, CHUNK, 1.0, ws, nb, stream))
+    K.kda_check_status(ws)
+    nbytes = T * Hh * 7 * 512 + Hh * STATE_BYTES
+    out["dplr_fp32"] = {"ms": ms_dplr, "algorithmic_bytes": nbytes,
+                        "frac": nbytes / (ms_dplr * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    del d, ws
+    torch.cuda.empty_cache()
+    d = inputs.chunk_inputs([T], H=Hh, dtype=torch.float32, seed=5, s0_std=0.02, device=dev)
+    nb = K.kda_chunk_fwd_workspace_bytes(T, 1, Hh, D, D, CHUNK, K.KDA_F32)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    ms_kda = timed(lambda: K.kda_chunk_fwd(d["q"], d["k"], d["v"], d["log_alpha"], d["beta"], d["S0"], o, S_T,
+                                           None, None, 1, T, Hh, D, D, CHUNK, 1.0, K.KDA_F32, ws, nb, stream))
+    K.kda_check_status(ws)
+    nbytes = T * Hh * (5 * 512 + 4) + Hh * STATE_BYTES
+    out["kda_fp32"] = {"ms": ms_kda, "algorithmic_bytes": nbytes,
+                       "frac": nbytes / (ms_kda * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    out["dplr_over_kda_fp32"] = ms_dplr / ms_kda
+    del d, ws, o
+    torch.cuda.empty_cache()
+    d = inputs.chunk_inputs([T], H=Hh, dtype=torch.bfloat16, seed=5, s0_std=0.02, device=dev)
+    nb = K.kda_chunk_fwd_workspace_bytes(T, 1, Hh, D, D, CHUNK, K.KDA_BF16)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    o = torch.empty((T, Hh, D), dtype=torch.bfloat16, device=dev)
+    ms_tc = timed(lambda: K.kda_chunk_fwd(d["q"], d["k"], d["v"], d["log_alpha"], d["beta"], d["S0"], o, S_T,
+                                          None, None, 1, T, Hh, D, D, CHUNK, 1.0, K.KDA_BF16, ws, nb, stream), 20)
+    K.kda_check_status(ws)
+    out["kda_bf16_tensor_core"] = {"ms": ms_tc}
+    del d, ws, o, S_T
+    torch.cuda.empty_cache()
+    return out
+
+
 def decode_only(args, K, inputs, torch, dev, peaks):
     """Short decode-only run (used under a profiler): one block of 64 in-place steps, timed."""
     dd = inputs.decode_inputs(DEC_SEQS, H, DEC_STEPS, seed=4)
@@ -513,6 +573,7 @@ def main():
     if world == 1 and not args.no_other_workloads:
         if free_b >= 80 * (1 << 30):
             other = extra_workloads(K, inputs, torch, dev, peaks)
+            other["dplr_comparison"] = dplr_comparison(K, inputs, torch, dev, peaks)
         else:
             other = {"skipped": "needs about 70 GB of free device memory, %.0f GB free" % (free_b / 2 ** 30)}
 

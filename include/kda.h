@@ -145,6 +145,37 @@ kda_status_t kda_chunk_fwd_static(const void *q, const void *k, const void *v,
                                   void *cuda_stream);
 
 /*
+ * Comparison workload: chunkwise forward of the GENERAL diagonal-plus-low-rank recurrence (paper
+ * Section 6.1 "Relation to DPLR" and its chunkwise DPLR pseudo-code; the kernel-time comparison of
+ * Section 3.2), per sequence and head:
+ *
+ *     S_t = (Diag(exp(g_t)) + b_t a_t^T) S_{t-1} + k_t v_t^T ,      o_t = scale * S_t^T q_t
+ *
+ * (a_t is contracted with the state the previous token left; with a = alpha . k, b = -beta k and
+ * the key beta k this is Eq. 1).  fp32 storage and arithmetic only, in the same two-kernel FMA
+ * style as kda_chunk_fwd with dt = KDA_F32, so that the two run times compare like with like.
+ *
+ *   q, k, a, b, g  [T_total, H, dk] fp32 device;  v, o [T_total, H, dv] fp32 device
+ *   S0, S_T, cu_seqlens_dev, cu_seqlens_host, n_seqs, total_tokens, H, scale: as in kda_chunk_fwd
+ *   workspace: device memory, 256-byte aligned, at least ..._min_workspace_bytes (the call then
+ *              walks the chunks in several passes); ..._workspace_bytes gives room for one pass.
+ *              Its first 256 bytes hold the status word that kda_check_status reads.
+ * Only dk = dv = 128 and chunk = 64.  Asynchronous on `cuda_stream`; nothing is allocated.  Errors
+ * as for kda_chunk_fwd (KDA_ERR_INVALID_ARG, KDA_ERR_UNSUPPORTED, KDA_ERR_WORKSPACE, KDA_ERR_CUDA);
+ * a channel that decays by more than e^-160 inside one chunk raises the KDA_ERR_GATE_RANGE flag.
+ */
+size_t kda_dplr_chunk_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
+                                              int chunk);
+size_t kda_dplr_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv,
+                                          int chunk);
+kda_status_t kda_dplr_chunk_fwd(const float *q, const float *k, const float *v, const float *a,
+                                const float *b, const float *g, const float *S0, float *o,
+                                float *S_T, const int32_t *cu_seqlens_dev,
+                                const int32_t *cu_seqlens_host, int n_seqs, int64_t total_tokens,
+                                int H, int dk, int dv, int chunk, float scale, void *workspace,
+                                size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Chooses how kda_chunk_fwd schedules a bf16 call (process-wide; no counterpart in the paper).
  *   0  automatic (default): when the workspace has room for every (chunk, head) tile of the call,
  *      the intra-chunk stage (Section 3.1: gates, UT transform) runs as one kernel and the

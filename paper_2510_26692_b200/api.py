@@ -59,6 +59,13 @@ def load():
     lib.kda_chunk_fwd_static.restype = i32
     lib.kda_chunk_fwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32,
                                          i32, i32, f32, i32, vp]
+    lib.kda_dplr_chunk_fwd_workspace_bytes.restype = sz
+    lib.kda_dplr_chunk_fwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
+    lib.kda_dplr_chunk_fwd_min_workspace_bytes.restype = sz
+    lib.kda_dplr_chunk_fwd_min_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
+    lib.kda_dplr_chunk_fwd.restype = i32
+    lib.kda_dplr_chunk_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32,
+                                       i32, i32, f32, vp, sz, vp]
     lib.kda_decode_step.restype = i32
     lib.kda_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp]
     lib.kda_decode_multi.restype = i32
@@ -174,6 +181,33 @@ def kda_chunk_fwd(q, k, v, log_alpha, beta, S0, o, S_T, cu_seqlens_dev, cu_seqle
         _ptr(cu_seqlens_dev, True, torch.int32, "cu_seqlens_dev"),
         _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
         int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale), int(dt),
+        _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
+    _check(rc)
+
+
+def kda_dplr_chunk_fwd_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64) -> int:
+    return int(load().kda_dplr_chunk_fwd_workspace_bytes(int(total_tokens), int(n_seqs), int(H), dk, dv, chunk))
+
+
+def kda_dplr_chunk_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64) -> int:
+    return int(load().kda_dplr_chunk_fwd_min_workspace_bytes(int(total_tokens), int(n_seqs), int(H), dk, dv,
+                                                             chunk))
+
+
+def kda_dplr_chunk_fwd(q, k, v, a, b, g, S0, o, S_T, cu_seqlens_dev, cu_seqlens_host, n_seqs,
+                       total_tokens, H, dk, dv, chunk, scale, workspace, workspace_bytes=None, stream=None):
+    """``kda_dplr_chunk_fwd`` of ``include/kda.h`` (the general diagonal-plus-low-rank comparison
+    workload, fp32 device tensors).  Asynchronous on ``stream``."""
+    f32 = torch.float32
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    rc = load().kda_dplr_chunk_fwd(
+        _ptr(q, True, f32, "q"), _ptr(k, True, f32, "k"), _ptr(v, True, f32, "v"),
+        _ptr(a, True, f32, "a"), _ptr(b, True, f32, "b"), _ptr(g, True, f32, "g"),
+        _ptr(S0, True, f32, "S0"), _ptr(o, True, f32, "o"), _ptr(S_T, True, f32, "S_T"),
+        _ptr(cu_seqlens_dev, True, torch.int32, "cu_seqlens_dev"),
+        _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
+        int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale),
         _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
     _check(rc)
 
