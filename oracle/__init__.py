@@ -6,6 +6,7 @@ A plain, slow CPU statement of what the KDA hot path computes, in fp64:
   Section 3, Eq. 1 of the Kimi Linear paper.  This is the oracle.
 * ``dplr_recurrence`` is the general diagonal-plus-low-rank recurrence of Section 6.1 ("Relation
   to DPLR"), the paper's comparison workload, in the same plain form (``kda_oracle.c``).
+* ``backward`` is the adjoint of that recurrence (gradients of Eq. 1), also in ``kda_oracle.c``.
 * ``chunkwise.chunk_kda_np`` is a second, independent numpy statement of the chunkwise algorithm of
   Section 3.1 (WY representation + UT transform + chunk state update + output equation).  It is a
   cross-check of the oracle, not the oracle.
@@ -60,6 +61,11 @@ def _load():
             lib.kda_oracle_dplr_recurrence.restype = ctypes.c_int
             lib.kda_oracle_dplr_recurrence.argtypes = [
                 f32p, f32p, f32p, f32p, f32p, f32p, f64p, f64p, f64p,
+                ctypes.POINTER(ctypes.c_int64), ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                ctypes.c_int, ctypes.c_double, ctypes.c_int]
+            lib.kda_oracle_backward.restype = ctypes.c_int
+            lib.kda_oracle_backward.argtypes = [
+                f32p, f32p, f32p, f32p, f32p, f64p, f64p, f64p, f64p, f64p, f64p, f64p, f64p, f64p,
                 ctypes.POINTER(ctypes.c_int64), ctypes.c_int, ctypes.c_int, ctypes.c_int,
                 ctypes.c_int, ctypes.c_double, ctypes.c_int]
             lib.kda_oracle_max_threads.restype = ctypes.c_int
@@ -163,6 +169,48 @@ def dplr_recurrence(q, k, v, a, b, g, S0=None, cu_seqlens=None, scale=1.0, want_
     if rc != 0:
         raise RuntimeError("kda_oracle_dplr_recurrence failed")
     return o, S_T
+
+
+def backward(q, k, v, log_alpha, beta, d_o=None, dS_T=None, S0=None, cu_seqlens=None, scale=1.0,
+             n_threads=0):
+    """Gradients of Eq. 1 for L = sum_t <d_o_t, o_t> + <dS_T, S_T>, by the adjoint of the
+    token-by-token recurrence in fp64 (``kda_oracle_backward``).  Shapes as in ``recurrence``; d_o
+    [T,H,dv] and dS_T [N,H,dk,dv] may be None (zeros).  Returns a dict with dq, dk, dlog_alpha
+    [T,H,dk], dv [T,H,dv], dbeta [T,H], dS0 [N,H,dk,dv], all fp64."""
+    k = _f32(k)
+    T, H, dk = k.shape
+    v = _f32(v)
+    dv = v.shape[-1]
+    q = _f32(q, (T, H, dk))
+    log_alpha = _f32(log_alpha, (T, H, dk))
+    beta = _f32(beta, (T, H))
+    if cu_seqlens is None:
+        cu = np.array([0, T], dtype=np.int64)
+    else:
+        cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int64))
+        assert cu[0] == 0 and cu[-1] == T and np.all(np.diff(cu) >= 0)
+    N = cu.shape[0] - 1
+
+    def f64(x, shape):
+        if x is None:
+            return None
+        a = np.ascontiguousarray(np.asarray(x, dtype=np.float64))
+        assert a.shape == tuple(shape), (a.shape, shape)
+        return a
+    S0a, doa, dSa = f64(S0, (N, H, dk, dv)), f64(d_o, (T, H, dv)), f64(dS_T, (N, H, dk, dv))
+    out = {"dq": np.empty((T, H, dk)), "dk": np.empty((T, H, dk)), "dv": np.empty((T, H, dv)),
+           "dlog_alpha": np.empty((T, H, dk)), "dbeta": np.empty((T, H)), "dS0": np.empty((N, H, dk, dv))}
+    rc = _load().kda_oracle_backward(
+        _ptr(q, ctypes.c_float), _ptr(k, ctypes.c_float), _ptr(v, ctypes.c_float),
+        _ptr(log_alpha, ctypes.c_float), _ptr(beta, ctypes.c_float), _ptr(S0a, ctypes.c_double),
+        _ptr(doa, ctypes.c_double), _ptr(dSa, ctypes.c_double),
+        _ptr(out["dq"], ctypes.c_double), _ptr(out["dk"], ctypes.c_double), _ptr(out["dv"], ctypes.c_double),
+        _ptr(out["dlog_alpha"], ctypes.c_double), _ptr(out["dbeta"], ctypes.c_double),
+        _ptr(out["dS0"], ctypes.c_double), _ptr(cu, ctypes.c_int64), N, H, dk, dv, float(scale),
+        int(n_threads))
+    if rc != 0:
+        raise RuntimeError("kda_oracle_backward failed")
+    return out
 
 
 def decode_step(q, k, v, log_alpha, beta, S, state_slot=None, scale=1.0, n_threads=0):

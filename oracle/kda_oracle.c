@@ -232,6 +232,134 @@ int kda_oracle_dplr_recurrence(const float *q, const float *k, const float *v, c
     return failed ? -1 : 0;
 }
 
+/*
+ * Gradients of Eq. 1 (backward pass; the paper trains with the recurrence, Section 5, but prints no
+ * backward algorithm, so this is Eq. 1 differentiated by hand).  For the scalar
+ *
+ *     L = sum_t <d_o_t, o_t> + <dS_T, S_T>
+ *
+ * it returns dL/dq, dL/dk, dL/dv, dL/dlog_alpha, dL/dbeta and dL/dS0.  With the forward step
+ * written as  S' = Diag(alpha_t) S_{t-1},  r = v_t - S'^T k_t,  S_t = S' + beta_t k_t r^T,
+ * o_t = scale S_t^T q_t,  and Lam the adjoint of the state, the steps are taken in reverse order:
+ *
+ *     Lam  += scale q_t d_o_t^T                 dq_t = scale S_t d_o_t
+ *     dbeta_t = k_t^T Lam r                     dk_t  = beta_t Lam r
+ *     dr = beta_t Lam^T k_t                     dv_t  = dr
+ *     Lam' = Lam - k_t dr^T                     dk_t -= S' dr
+ *     dlog_alpha_t = rowsum(Lam' . S')          Lam  <- Diag(alpha_t) Lam'          (for t-1)
+ *
+ * (dlog_alpha uses alpha_t dS'/dalpha_t = S', so nothing is divided by alpha.)  The forward states
+ * of one sequence and head are all kept in memory: sizes are for tests (T * dk * dv doubles).
+ *
+ * Layouts as above; d_o [T_total,H,dv] may be NULL (= zeros), dS_T [n_seqs,H,dk,dv] may be NULL
+ * (= zeros); every output pointer may be NULL.
+ */
+int kda_oracle_backward(const float *q, const float *k, const float *v, const float *log_alpha,
+                        const float *beta, const double *S0, const double *d_o, const double *dS_T,
+                        double *dq, double *dk_out, double *dv_out, double *dg, double *dbeta,
+                        double *dS0, const int64_t *cu_seqlens, int n_seqs, int H, int dk, int dv,
+                        double scale, int n_threads)
+{
+    if (!q || !k || !v || !log_alpha || !beta || !cu_seqlens || n_seqs < 0 || H <= 0 || dk <= 0 || dv <= 0)
+        return -1;
+    int failed = 0;
+    long n_items = (long)n_seqs * H;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+    (void)n_threads;
+#endif
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long item = 0; item < n_items; ++item) {
+        int n = (int)(item / H), h = (int)(item % H);
+        int64_t t0 = cu_seqlens[n], t1 = cu_seqlens[n + 1];
+        size_t len = (size_t)(t1 - t0), sz = (size_t)dk * dv;
+        /* Sd[t] = decayed state S' of token t, Sp[t] = state S_t after token t, R[t] = residual r */
+        double *Sd = (double *)malloc(sizeof(double) * sz * (len ? len : 1));
+        double *Sp = (double *)malloc(sizeof(double) * sz * (len ? len : 1));
+        double *R = (double *)malloc(sizeof(double) * dv * (len ? len : 1));
+        double *Lam = (double *)malloc(sizeof(double) * sz);
+        double *S = (double *)malloc(sizeof(double) * sz);
+        double *dr = (double *)malloc(sizeof(double) * dv);
+        double *lr = (double *)malloc(sizeof(double) * dk);
+        if (!Sd || !Sp || !R || !Lam || !S || !dr || !lr) {
+            failed = 1;
+            free(Sd); free(Sp); free(R); free(Lam); free(S); free(dr); free(lr);
+            continue;
+        }
+        size_t sofs = ((size_t)n * H + h) * sz;
+        if (S0) memcpy(S, S0 + sofs, sizeof(double) * sz);
+        else memset(S, 0, sizeof(double) * sz);
+        /* forward, keeping every intermediate */
+        for (size_t s = 0; s < len; ++s) {
+            size_t th = (size_t)(t0 + (int64_t)s) * H + h;
+            const float *kt = k + th * dk, *vt = v + th * dv, *gt = log_alpha + th * dk;
+            double b = (double)beta[th];
+            double *Sds = Sd + s * sz, *Sps = Sp + s * sz, *r = R + s * dv;
+            for (int i = 0; i < dk; ++i) {
+                double al = exp((double)gt[i]);
+                for (int j = 0; j < dv; ++j) Sds[(size_t)i * dv + j] = al * S[(size_t)i * dv + j];
+            }
+            for (int j = 0; j < dv; ++j) r[j] = (double)vt[j];
+            for (int i = 0; i < dk; ++i)
+                for (int j = 0; j < dv; ++j) r[j] -= (double)kt[i] * Sds[(size_t)i * dv + j];
+            for (int i = 0; i < dk; ++i)
+                for (int j = 0; j < dv; ++j)
+                    Sps[(size_t)i * dv + j] = Sds[(size_t)i * dv + j] + b * (double)kt[i] * r[j];
+            memcpy(S, Sps, sizeof(double) * sz);
+        }
+        /* reverse */
+        if (dS_T) memcpy(Lam, dS_T + sofs, sizeof(double) * sz);
+        else memset(Lam, 0, sizeof(double) * sz);
+        for (size_t s = len; s-- > 0;) {
+            size_t th = (size_t)(t0 + (int64_t)s) * H + h;
+            const float *qt = q + th * dk, *kt = k + th * dk, *gt = log_alpha + th * dk;
+            double b = (double)beta[th];
+            const double *Sds = Sd + s * sz, *Sps = Sp + s * sz, *r = R + s * dv;
+            const double *dot = d_o ? d_o + th * dv : NULL;
+            /* o_t = scale S_t^T q_t */
+            for (int i = 0; i < dk; ++i) {
+                double acc = 0.0;
+                for (int j = 0; j < dv; ++j) {
+                    double g_o = dot ? dot[j] : 0.0;
+                    Lam[(size_t)i * dv + j] += scale * (double)qt[i] * g_o;
+                    acc += Sps[(size_t)i * dv + j] * g_o;
+                }
+                if (dq) dq[th * dk + i] = scale * acc;
+            }
+            /* S_t = S' + beta k r^T */
+            double db = 0.0;
+            for (int i = 0; i < dk; ++i) {
+                double acc = 0.0;
+                for (int j = 0; j < dv; ++j) acc += Lam[(size_t)i * dv + j] * r[j];
+                lr[i] = acc;                       /* (Lam r)_i */
+                db += (double)kt[i] * acc;
+            }
+            if (dbeta) dbeta[th] = db;
+            for (int j = 0; j < dv; ++j) {
+                double acc = 0.0;
+                for (int i = 0; i < dk; ++i) acc += Lam[(size_t)i * dv + j] * (double)kt[i];
+                dr[j] = b * acc;
+                if (dv_out) dv_out[th * dv + j] = dr[j];   /* r = v - S'^T k */
+            }
+            for (int i = 0; i < dk; ++i) {
+                double sdr = 0.0, gsum = 0.0, al = exp((double)gt[i]);
+                for (int j = 0; j < dv; ++j) {
+                    double lp = Lam[(size_t)i * dv + j] - (double)kt[i] * dr[j];   /* Lam' */
+                    sdr += Sds[(size_t)i * dv + j] * dr[j];
+                    gsum += lp * Sds[(size_t)i * dv + j];
+                    Lam[(size_t)i * dv + j] = al * lp;                             /* adjoint of S_{t-1} */
+                }
+                if (dk_out) dk_out[th * dk + i] = b * lr[i] - sdr;
+                if (dg) dg[th * dk + i] = gsum;
+            }
+        }
+        if (dS0) memcpy(dS0 + sofs, Lam, sizeof(double) * sz);
+        free(Sd); free(Sp); free(R); free(Lam); free(S); free(dr); free(lr);
+    }
+    return failed ? -1 : 0;
+}
+
 int kda_oracle_max_threads(void)
 {
 #ifdef _OPENMP
