@@ -290,6 +290,45 @@ def dplr_comparison(K, inputs, torch, dev, peaks):
     return out
 
 
+def backward_figure(K, inputs, torch, dev, peaks):
+    """Gradients of the prefill operator (kda_chunk_bwd) on the headline prefill workload: d_o and
+    dS_T random, forward recomputed inside the call."""
+    stream = torch.cuda.current_stream()
+    T = T_PREFILL
+    d = inputs.chunk_inputs([T], H=H, dtype=torch.bfloat16, seed=1, s0_std=0.02, device=dev)
+    g = torch.Generator(device=dev).manual_seed(77)
+    d_o = torch.randn((T, H, D), generator=g, device=dev).to(torch.bfloat16)
+    dS_T = torch.randn((1, H, D, D), generator=g, device=dev)
+    nb = K.kda_chunk_bwd_workspace_bytes(T, 1, H)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    outs = [torch.empty((T, H, D), dtype=torch.float32, device=dev) for _ in range(4)]
+    db = torch.empty((T, H), dtype=torch.float32, device=dev)
+    dS0 = torch.empty_like(dS_T)
+
+    def call():
+        K.kda_chunk_bwd(d["q"], d["k"], d["v"], d["log_alpha"], d["beta"], d["S0"], d_o, dS_T, outs[0], outs[1],
+                        outs[2], outs[3], db, dS0, None, None, 1, T, H, D, D, CHUNK, 1.0, K.KDA_BF16, ws, nb,
+                        stream)
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(5):
+        call()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    K.kda_check_status(ws)
+    ms = e0.elapsed_time(e1) / 5
+    # q, k, v, d_o bf16 + log alpha, beta fp32 read; dq, dk, dv, dlog_alpha, dbeta fp32 written; states
+    nbytes = T * H * (4 * 256 + 512 + 4 + 4 * 512 + 4) + 4 * H * D * D * 4
+    return {"workload": "gradients of the prefill workload (B=1 T=4096 H=32, bf16 q/k/v/d_o, fp32 gradients)",
+            "ms": ms, "tokens_per_s": T / (ms * 1e-3), "algorithmic_bytes": nbytes,
+            "achieved_gbs": nbytes / (ms * 1e-3) / 1e9, "frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "note": "token-sequential adjoint in fp32 FMA (one CTA per sequence, head and 32-column slice): "
+                    "bound by the 4096 dependent steps, not by memory"}
+
+
 def decode_only(args, K, inputs, torch, dev, peaks):
     """Short decode-only run (used under a profiler): one block of 64 in-place steps, timed."""
     dd = inputs.decode_inputs(DEC_SEQS, H, DEC_STEPS, seed=4)
@@ -574,6 +613,7 @@ def main():
         if free_b >= 80 * (1 << 30):
             other = extra_workloads(K, inputs, torch, dev, peaks)
             other["dplr_comparison"] = dplr_comparison(K, inputs, torch, dev, peaks)
+            other["backward"] = backward_figure(K, inputs, torch, dev, peaks)
         else:
             other = {"skipped": "needs about 70 GB of free device memory, %.0f GB free" % (free_b / 2 ** 30)}
 

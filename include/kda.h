@@ -145,6 +145,40 @@ kda_status_t kda_chunk_fwd_static(const void *q, const void *k, const void *v,
                                   void *cuda_stream);
 
 /*
+ * Backward pass of kda_chunk_fwd: gradients of Eq. 1 (the operator is trained end to end, Section 5;
+ * the paper prints no backward algorithm, so this is the adjoint of Eq. 1 itself).  For
+ *
+ *     L = sum_t <d_o_t, o_t> + <dS_T, S_T>
+ *
+ * it returns dL/dq, dL/dk, dL/dv, dL/dlog_alpha, dL/dbeta and dL/dS0.  The forward pass is
+ * recomputed inside (nothing has to be kept from kda_chunk_fwd): a first sweep stores the state at
+ * every chunk boundary, a reverse sweep recomputes one chunk at a time and runs the adjoint through
+ * it token by token; fp32 arithmetic throughout.
+ *
+ *   q, k [T_total,H,dk], v, d_o [T_total,H,dv]   device, element type `dt` (KDA_F32 or KDA_BF16)
+ *   log_alpha [T_total,H,dk], beta [T_total,H]   fp32 device
+ *   S0, dS_T  [n_seqs,H,dk,dv] fp32 device or NULL (= zeros);  d_o may be NULL (= zeros)
+ *   dq, dk, dlog_alpha [T_total,H,dk], dv [T_total,H,dv], dbeta [T_total,H]   fp32 device, written
+ *   dS0 [n_seqs,H,dk,dv] fp32 device, written, or NULL
+ *   cu_seqlens_dev / cu_seqlens_host, n_seqs, total_tokens, H, scale: as in kda_chunk_fwd
+ *   workspace: device memory, 256-byte aligned, at least kda_chunk_bwd_workspace_bytes(...) (chunk
+ *              boundary states, one chunk of recomputed states per (sequence, head), and the
+ *              per-slice shares of the gradients that are summed over dv; about 0.26 MB per token
+ *              at H = 32).  Its first 256 bytes hold the status word that kda_check_status reads.
+ * Only dk = dv = 128 and chunk = 64.  Asynchronous on `cuda_stream`; nothing is allocated; results
+ * are deterministic (fixed summation order).  Errors: KDA_ERR_INVALID_ARG, KDA_ERR_UNSUPPORTED,
+ * KDA_ERR_WORKSPACE, KDA_ERR_CUDA.
+ */
+size_t kda_chunk_bwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv, int chunk);
+kda_status_t kda_chunk_bwd(const void *q, const void *k, const void *v, const float *log_alpha,
+                           const float *beta, const float *S0, const void *d_o, const float *dS_T,
+                           float *dq, float *dk_out, float *dv_out, float *dlog_alpha, float *dbeta,
+                           float *dS0, const int32_t *cu_seqlens_dev, const int32_t *cu_seqlens_host,
+                           int n_seqs, int64_t total_tokens, int H, int dk, int dv, int chunk,
+                           float scale, kda_dtype_t dt, void *workspace, size_t workspace_bytes,
+                           void *cuda_stream);
+
+/*
  * Comparison workload: chunkwise forward of the GENERAL diagonal-plus-low-rank recurrence (paper
  * Section 6.1 "Relation to DPLR" and its chunkwise DPLR pseudo-code; the kernel-time comparison of
  * Section 3.2), per sequence and head:

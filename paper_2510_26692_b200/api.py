@@ -66,6 +66,10 @@ def load():
     lib.kda_dplr_chunk_fwd.restype = i32
     lib.kda_dplr_chunk_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32,
                                        i32, i32, f32, vp, sz, vp]
+    lib.kda_chunk_bwd_workspace_bytes.restype = sz
+    lib.kda_chunk_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
+    lib.kda_chunk_bwd.restype = i32
+    lib.kda_chunk_bwd.argtypes = [vp] * 16 + [i32, i64, i32, i32, i32, i32, f32, i32, vp, sz, vp]
     lib.kda_decode_step.restype = i32
     lib.kda_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp]
     lib.kda_decode_multi.restype = i32
@@ -208,6 +212,32 @@ def kda_dplr_chunk_fwd(q, k, v, a, b, g, S0, o, S_T, cu_seqlens_dev, cu_seqlens_
         _ptr(cu_seqlens_dev, True, torch.int32, "cu_seqlens_dev"),
         _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
         int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale),
+        _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
+    _check(rc)
+
+
+def kda_chunk_bwd_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64) -> int:
+    return int(load().kda_chunk_bwd_workspace_bytes(int(total_tokens), int(n_seqs), int(H), dk, dv, chunk))
+
+
+def kda_chunk_bwd(q, k, v, log_alpha, beta, S0, d_o, dS_T, dq, dk_out, dv_out, dlog_alpha, dbeta, dS0,
+                  cu_seqlens_dev, cu_seqlens_host, n_seqs, total_tokens, H, dk, dv, chunk, scale, dt,
+                  workspace, workspace_bytes=None, stream=None):
+    """``kda_chunk_bwd`` of ``include/kda.h``: gradients of the prefill operator (fp32 outputs).
+    Asynchronous on ``stream``."""
+    f32 = torch.float32
+    et = torch.bfloat16 if dt == KDA_BF16 else torch.float32
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    rc = load().kda_chunk_bwd(
+        _ptr(q, True, et, "q"), _ptr(k, True, et, "k"), _ptr(v, True, et, "v"),
+        _ptr(log_alpha, True, f32, "log_alpha"), _ptr(beta, True, f32, "beta"), _ptr(S0, True, f32, "S0"),
+        _ptr(d_o, True, et, "d_o"), _ptr(dS_T, True, f32, "dS_T"),
+        _ptr(dq, True, f32, "dq"), _ptr(dk_out, True, f32, "dk"), _ptr(dv_out, True, f32, "dv"),
+        _ptr(dlog_alpha, True, f32, "dlog_alpha"), _ptr(dbeta, True, f32, "dbeta"), _ptr(dS0, True, f32, "dS0"),
+        _ptr(cu_seqlens_dev, True, torch.int32, "cu_seqlens_dev"),
+        _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
+        int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale), int(dt),
         _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
     _check(rc)
 
