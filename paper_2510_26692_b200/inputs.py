@@ -17,7 +17,7 @@ from typing import Dict, Optional, Sequence
 import torch
 
 _ORDER = {"q": 0, "k": 1, "v": 2, "x": 3, "beta": 4, "S0": 5, "S": 6, "lens": 7, "a": 8, "b": 9, "eta": 10,
-          "do": 11, "dS": 12}
+          "do": 11, "dS": 12, "go": 13, "w": 14, "bias": 15}
 
 
 def _gen(seed: int, name: str, device) -> torch.Generator:
@@ -150,6 +150,35 @@ def dplr_inputs(lengths: Sequence[int], H: int, dk: int = 128, dv: int = 128, se
     eta = torch.sigmoid(_randn((T, H, 2), seed, "eta", device))
     out["a"] = _l2norm(ra) * (0.5 + 0.5 * eta[..., 0:1])
     out["b"] = -_l2norm(ra + 0.5 * rb) * eta[..., 1:2]
+    out["S0"] = (_randn((N, H, dk, dv), seed, "S0", device) * s0_std) if s0_std > 0 else None
+    out["cu_seqlens"] = cu_seqlens_of(lengths)
+    return out
+
+
+def layer_inputs(lengths: Sequence[int], H: int, dk: int = 128, dv: int = 128, seed: int = 0,
+                 gate_mean: float = 4.0, s0_std: float = 0.0, device="cpu") -> Dict[str, Optional[torch.Tensor]]:
+    """Pre-activations of one KDA layer call (Section 4, "Neural Parameterization"): q_c, k_c (what
+    leaves the short convolution and Swish, before L2Norm; N(0,1) times a per-token factor so that
+    the norms vary), v, the decay pre-activation g_a (N(-gate_mean, 1): after the softplus and a
+    per-head rate exp(A_log) of about one this gives the same decay range as ``chunk_inputs``), the
+    beta pre-activation b_pre ~ N(0,1) (fp32), the output-gate pre-activation g_o ~ N(0,1), and the
+    layer's parameters A_log [H] ~ N(0, 0.3), dt_bias [H,dk] ~ N(0, 0.3), RMSNorm weight w [dv] ~
+    1 + N(0, 0.1).  Activations bf16, parameters fp32.
+    """
+    T = int(sum(lengths))
+    N = len(lengths)
+    bf = torch.bfloat16
+    out: Dict[str, Optional[torch.Tensor]] = {}
+    fac = 0.5 + torch.rand((T, H, 2), generator=_gen(seed, "eta", device), device=device) * 3.0
+    out["q_c"] = (_randn((T, H, dk), seed, "q", device) * fac[..., 0:1]).to(bf)
+    out["k_c"] = (_randn((T, H, dk), seed, "k", device) * fac[..., 1:2]).to(bf)
+    out["v"] = _randn((T, H, dv), seed, "v", device).to(bf)
+    out["g_a"] = (_randn((T, H, dk), seed, "x", device) - gate_mean).to(bf)
+    out["b_pre"] = _randn((T, H), seed, "beta", device)
+    out["g_o"] = _randn((T, H, dv), seed, "go", device).to(bf)
+    out["A_log"] = _randn((H,), seed, "a", device) * 0.3
+    out["dt_bias"] = _randn((H, dk), seed, "bias", device) * 0.3
+    out["w"] = 1.0 + _randn((dv,), seed, "w", device) * 0.1
     out["S0"] = (_randn((N, H, dk, dv), seed, "S0", device) * s0_std) if s0_std > 0 else None
     out["cu_seqlens"] = cu_seqlens_of(lengths)
     return out
