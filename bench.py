@@ -329,6 +329,40 @@ def backward_figure(K, inputs, torch, dev, peaks):
                     "bound by the 4096 dependent steps, not by memory"}
 
 
+def layer_figure(K, inputs, torch, dev, peaks):
+    """kda_layer_fwd on the headline prefill shape: L2Norm, decay function and beta sigmoid inside the
+    intra-chunk kernel, RMSNorm and output gate as a pass over the bf16 output."""
+    stream = torch.cuda.current_stream()
+    T = T_PREFILL
+    sets = [inputs.layer_inputs([T], H=H, seed=60 + i, s0_std=0.02, device=dev) for i in range(3)]   # > L2 in total
+    nb = K.kda_layer_fwd_workspace_bytes(T, 1, H)
+    ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+    y = torch.empty((T, H, D), dtype=torch.bfloat16, device=dev)
+    S_T = torch.empty((1, H, D, D), dtype=torch.float32, device=dev)
+
+    def call(d):
+        K.kda_layer_fwd(d["q_c"], d["k_c"], d["v"], d["g_a"], d["b_pre"], d["g_o"], d["A_log"], d["dt_bias"], d["w"],
+                        1e-6, 1e-5, d["S0"], y, S_T, None, None, 1, T, H, D, D, CHUNK, D ** -0.5, ws, nb, stream)
+    for i in range(5):
+        call(sets[i % 3])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 60
+    e0.record(stream)
+    for i in range(reps):
+        call(sets[i % 3])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    K.kda_check_status(ws)
+    ms = e0.elapsed_time(e1) / reps
+    # q_c, k_c, v, g_a, g_o read and y written in bf16, b_pre fp32; the states in and out
+    nbytes = T * H * (6 * 256 + 4) + H * STATE_BYTES
+    return {"workload": "B=1 T=4096 H=32, bf16 pre-activations (q_c, k_c, v, g_a, g_o), fp32 b_pre; inputs rotate over 3 copies",
+            "ms": ms, "tokens_per_s": T / (ms * 1e-3), "algorithmic_bytes": nbytes,
+            "achieved_gbs": nbytes / (ms * 1e-3) / 1e9, "frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "note": "three kernels per call: intra-chunk (with the prologue), inter-chunk, output stage"}
+
+
 def decode_only(args, K, inputs, torch, dev, peaks):
     """Short decode-only run (used under a profiler): one block of 64 in-place steps, timed."""
     dd = inputs.decode_inputs(DEC_SEQS, H, DEC_STEPS, seed=4)
@@ -614,6 +648,7 @@ def main():
             other = extra_workloads(K, inputs, torch, dev, peaks)
             other["dplr_comparison"] = dplr_comparison(K, inputs, torch, dev, peaks)
             other["backward"] = backward_figure(K, inputs, torch, dev, peaks)
+            other["layer_fwd"] = layer_figure(K, inputs, torch, dev, peaks)
         else:
             other = {"skipped": "needs about 70 GB of free device memory, %.0f GB free" % (free_b / 2 ** 30)}
 

@@ -145,6 +145,43 @@ kda_status_t kda_chunk_fwd_static(const void *q, const void *k, const void *v,
                                   void *cuda_stream);
 
 /*
+ * The KDA operator with the layer's surrounding element-wise stages (paper Section 4, "Neural
+ * Parameterization"), from the activations that leave the short convolutions to the input of the
+ * output projection, bf16 tensor-core path:
+ *
+ *     q, k      = L2Norm(q_c), L2Norm(k_c)                      x / sqrt(sum x^2 + l2_eps), over dk
+ *     log alpha = -exp(A_log[h]) * softplus(g_a + dt_bias[h,:])  (the decay function f; the paper
+ *                 names its family only -- "similar to GDN and Mamba" -- this is that form)
+ *     beta      = sigmoid(b_pre)
+ *     o         = KDA(q, k, v, alpha, beta)                      Eq. 1, with `scale` on q
+ *     y         = sigmoid(g_o) . RMSNorm(o) . rms_weight         o / sqrt(mean o^2 + rms_eps), over dv
+ *
+ * The normalisation, the decay function and the sigmoid of beta are computed inside the
+ * intra-chunk kernel from the half-precision pre-activations (no fp32 gate tensor and no
+ * normalised copy of q and k ever exists in memory); the output stage runs as a separate pass over
+ * the bf16 output, in place.
+ *
+ *   q_c, k_c, g_a [T_total,H,dk], v, g_o, y [T_total,H,dv]   bf16 device
+ *   b_pre [T_total,H]                                        fp32 device
+ *   A_log [H], dt_bias [H,dk], rms_weight [dv]               fp32 device
+ *   S0, S_T, cu_seqlens_dev, cu_seqlens_host, n_seqs, total_tokens, H, scale: as in kda_chunk_fwd;
+ *   y may be NULL (final state only; q_c, g_o, rms_weight are then unused)
+ *   workspace: as for kda_chunk_fwd with dt = KDA_BF16, at least kda_layer_fwd_min_workspace_bytes
+ *              (the call always runs the two-kernel schedule, in several passes if need be).
+ * Only dk = dv = 128 and chunk = 64.  Asynchronous; nothing is allocated; errors and the status
+ * word as for kda_chunk_fwd.
+ */
+size_t kda_layer_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv, int chunk);
+size_t kda_layer_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv, int chunk);
+kda_status_t kda_layer_fwd(const void *q_c, const void *k_c, const void *v, const void *g_a,
+                           const float *b_pre, const void *g_o, const float *A_log,
+                           const float *dt_bias, const float *rms_weight, float l2_eps, float rms_eps,
+                           const float *S0, void *y, float *S_T, const int32_t *cu_seqlens_dev,
+                           const int32_t *cu_seqlens_host, int n_seqs, int64_t total_tokens, int H,
+                           int dk, int dv, int chunk, float scale, void *workspace,
+                           size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Backward pass of kda_chunk_fwd: gradients of Eq. 1 (the operator is trained end to end, Section 5;
  * the paper prints no backward algorithm, so this is the adjoint of Eq. 1 itself).  For
  *

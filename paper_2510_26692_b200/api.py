@@ -70,6 +70,13 @@ def load():
     lib.kda_chunk_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
     lib.kda_chunk_bwd.restype = i32
     lib.kda_chunk_bwd.argtypes = [vp] * 16 + [i32, i64, i32, i32, i32, i32, f32, i32, vp, sz, vp]
+    lib.kda_layer_fwd_workspace_bytes.restype = sz
+    lib.kda_layer_fwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
+    lib.kda_layer_fwd_min_workspace_bytes.restype = sz
+    lib.kda_layer_fwd_min_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
+    lib.kda_layer_fwd.restype = i32
+    lib.kda_layer_fwd.argtypes = [vp] * 9 + [f32, f32, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32,
+                                             vp, sz, vp]
     lib.kda_decode_step.restype = i32
     lib.kda_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp]
     lib.kda_decode_multi.restype = i32
@@ -238,6 +245,34 @@ def kda_chunk_bwd(q, k, v, log_alpha, beta, S0, d_o, dS_T, dq, dk_out, dv_out, d
         _ptr(cu_seqlens_dev, True, torch.int32, "cu_seqlens_dev"),
         _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
         int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale), int(dt),
+        _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
+    _check(rc)
+
+
+def kda_layer_fwd_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64) -> int:
+    return int(load().kda_layer_fwd_workspace_bytes(int(total_tokens), int(n_seqs), int(H), dk, dv, chunk))
+
+
+def kda_layer_fwd_min_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64) -> int:
+    return int(load().kda_layer_fwd_min_workspace_bytes(int(total_tokens), int(n_seqs), int(H), dk, dv, chunk))
+
+
+def kda_layer_fwd(q_c, k_c, v, g_a, b_pre, g_o, A_log, dt_bias, rms_weight, l2_eps, rms_eps, S0, y, S_T,
+                  cu_seqlens_dev, cu_seqlens_host, n_seqs, total_tokens, H, dk, dv, chunk, scale, workspace,
+                  workspace_bytes=None, stream=None):
+    """``kda_layer_fwd`` of ``include/kda.h``: the operator with L2Norm, decay function, beta
+    sigmoid, head-wise RMSNorm and output gate, from bf16 pre-activations.  Asynchronous."""
+    f32, bf = torch.float32, torch.bfloat16
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    rc = load().kda_layer_fwd(
+        _ptr(q_c, True, bf, "q_c"), _ptr(k_c, True, bf, "k_c"), _ptr(v, True, bf, "v"), _ptr(g_a, True, bf, "g_a"),
+        _ptr(b_pre, True, f32, "b_pre"), _ptr(g_o, True, bf, "g_o"), _ptr(A_log, True, f32, "A_log"),
+        _ptr(dt_bias, True, f32, "dt_bias"), _ptr(rms_weight, True, f32, "rms_weight"), float(l2_eps),
+        float(rms_eps), _ptr(S0, True, f32, "S0"), _ptr(y, True, bf, "y"), _ptr(S_T, True, f32, "S_T"),
+        _ptr(cu_seqlens_dev, True, torch.int32, "cu_seqlens_dev"),
+        _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
+        int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale),
         _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
     _check(rc)
 

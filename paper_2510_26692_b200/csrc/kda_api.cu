@@ -256,12 +256,23 @@ size_t kda_chunk_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, in
     return want < lo ? lo : want;
 }
 
-kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const float* log_alpha,
-                           const float* beta, const float* S0, void* o, float* S_T,
-                           const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host,
-                           int n_seqs, int64_t total_tokens, int H, int dk, int dv, int chunk,
-                           float scale, kda_dtype_t dt, void* workspace, size_t workspace_bytes,
-                           void* cuda_stream)
+}  // extern "C"
+
+namespace kda {
+namespace {
+// decay-function parameters of a layer-mode call (kda_layer_fwd); rate == nullptr = plain call
+struct LayerMode {
+    const float* rate = nullptr;
+    const float* bias = nullptr;
+    float l2_eps = 0.f;
+};
+
+kda_status_t chunk_fwd_impl(const void* q, const void* k, const void* v, const float* log_alpha,
+                            const float* beta, const float* S0, void* o, float* S_T,
+                            const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host,
+                            int n_seqs, int64_t total_tokens, int H, int dk, int dv, int chunk,
+                            float scale, kda_dtype_t dt, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream, const LayerMode& lm)
 {
     if (!shape_ok(dk, dv, chunk, dt))
         return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: only dk=dv=128, chunk=64, dt in {f32,bf16} "
@@ -324,7 +335,7 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
         const WsLayout L2p = ws_layout(n_seqs, H);
         const bool one_pass = workspace_bytes >= L2p.fixed &&
                               (int64_t)((workspace_bytes - L2p.fixed) / ((size_t)H * tc_tile_bytes())) >= total_chunks;
-        fused = mode == 2 || (mode == 0 && !one_pass);
+        fused = !lm.rate && (mode == 2 || (mode == 0 && !one_pass));
     }
     if (fused) {
         // ---- one fused cooperative kernel ----
@@ -412,6 +423,7 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
     a.n_seqs = n_seqs; a.H = H; a.total_tokens = total_tokens; a.seq_len = seq_len;
     a.chunks_per_seq = chunks_per_seq; a.scale = scale;
     a.S_out = state;
+    a.gate_rate = lm.rate; a.gate_bias = lm.bias; a.l2_eps = lm.l2_eps;
 
     int64_t g0 = 0;
     bool first = true;
@@ -436,6 +448,60 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
         first = false;
     } while (g0 < total_chunks);
     return KDA_OK;
+}
+
+}  // namespace
+}  // namespace kda
+
+extern "C" {
+
+kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const float* log_alpha,
+                           const float* beta, const float* S0, void* o, float* S_T,
+                           const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host,
+                           int n_seqs, int64_t total_tokens, int H, int dk, int dv, int chunk,
+                           float scale, kda_dtype_t dt, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream)
+{
+    return chunk_fwd_impl(q, k, v, log_alpha, beta, S0, o, S_T, cu_seqlens_dev, cu_seqlens_host, n_seqs,
+                          total_tokens, H, dk, dv, chunk, scale, dt, workspace, workspace_bytes, cuda_stream,
+                          LayerMode());
+}
+
+size_t kda_layer_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv, int chunk)
+{
+    return kda_chunk_fwd_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, KDA_BF16);
+}
+
+size_t kda_layer_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv, int chunk)
+{
+    if (!shape_ok(dk, dv, chunk, KDA_BF16) || total_tokens < 0 || n_seqs < 0 || H <= 0) return 0;
+    return ws_layout(n_seqs, H).fixed + align_up((size_t)H * tc_tile_bytes());
+}
+
+kda_status_t kda_layer_fwd(const void* q_c, const void* k_c, const void* v, const void* g_a,
+                           const float* b_pre, const void* g_o, const float* A_log, const float* dt_bias,
+                           const float* rms_weight, float l2_eps, float rms_eps, const float* S0, void* y,
+                           float* S_T, const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host,
+                           int n_seqs, int64_t total_tokens, int H, int dk, int dv, int chunk, float scale,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!A_log || !dt_bias)
+        return fail(KDA_ERR_INVALID_ARG, "kda_layer_fwd: A_log and dt_bias must not be NULL");
+    if (y && total_tokens > 0 && (!g_o || !rms_weight))
+        return fail(KDA_ERR_INVALID_ARG, "kda_layer_fwd: g_o and rms_weight must not be NULL when y is "
+                    "requested");
+    const void* ptrs[] = {g_o, A_log, dt_bias, rms_weight};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return fail(KDA_ERR_INVALID_ARG, "kda_layer_fwd: pointer %p is not 16-byte "
+                                       "aligned", p);
+    LayerMode lm;
+    lm.rate = A_log; lm.bias = dt_bias; lm.l2_eps = l2_eps;
+    kda_status_t rc = chunk_fwd_impl(q_c, k_c, v, reinterpret_cast<const float*>(g_a), b_pre, S0, y, S_T,
+                                     cu_seqlens_dev, cu_seqlens_host, n_seqs, total_tokens, H, dk, dv, chunk,
+                                     scale, KDA_BF16, workspace, workspace_bytes, cuda_stream, lm);
+    if (rc != KDA_OK || !y || total_tokens == 0 || n_seqs == 0) return rc;
+    return launch_layer_epilogue(y, g_o, rms_weight, rms_eps, total_tokens * H,
+                                 static_cast<cudaStream_t>(cuda_stream));
 }
 
 kda_status_t kda_decode_step(const void* q, const void* k, const void* v, const float* log_alpha,

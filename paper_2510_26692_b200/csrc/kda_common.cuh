@@ -63,6 +63,13 @@ struct ChunkArgs {
     int64_t chunks_per_seq;   // equal-length case
     int64_t g0, g1;           // global chunk range of this pass
     float scale;
+    // Layer mode (kda_layer_fwd, bf16 tensor-core path only), off when gate_rate is nullptr: q and k
+    // arrive un-normalised, `log_alpha` points to the bf16 pre-activations of the decay function and
+    // `beta` to the fp32 pre-activations of beta; the intra-chunk kernel applies L2Norm, the decay
+    // function -exp(gate_rate[h]) * softplus(x + gate_bias[h, d]) and the sigmoid itself.
+    const float* gate_rate = nullptr;   // [H]
+    const float* gate_bias = nullptr;   // [H, dk]
+    float l2_eps = 0.f;
 };
 
 // Work description of the fused bf16 chunk-forward kernel (one cooperative launch per call).
@@ -194,6 +201,10 @@ struct DeviceLock {
 };
 // The slot table itself, without any CUDA call (unit-testable on a machine without a GPU).
 DeviceState* device_slot(int ordinal);
+
+// output stage of the layer wrap: y = sigmoid(g_o) . RMSNorm(y) . w in place, rows of kD bf16 values
+kda_status_t launch_layer_epilogue(void* y, const void* g_o, const float* w, float eps, int64_t n_rows,
+                                   cudaStream_t st);
 
 kda_status_t launch_wait_selftest(WsHeader* hdr, uint64_t limit_ns, cudaStream_t st);
 

@@ -80,7 +80,8 @@ constexpr uint32_t E_DESC = E_BETA + 256;         // two tile descriptors
 constexpr uint32_t E_BAR = E_DESC + 128;          // 8-byte words: mma barrier, K barrier, abort word, Q barrier,
                                                   // (first engine) TMEM slot, V barrier
 constexpr uint32_t E_KS = (E_BAR + 64 + 1023) / 1024 * 1024;   // raw k of the NEXT tile [2 K-halves][64][64] bf16
-constexpr uint32_t E_BYTES = E_KS + 16384;
+constexpr uint32_t E_NORM = E_KS + 16384;         // layer mode: 1 / |k_i|, 1 / |q_i| (64 fp32 each)
+constexpr uint32_t E_BYTES = E_NORM + 1024;
 static_assert(E_TD_BYTES >= 8 * 128 * 4 && E_TD_BYTES >= 4 * 16 * LDD * 4, "scan exchange and diagonal blocks fit");
 
 // ---- shared-memory map of a chain CTA (bytes from the 1024-aligned base) -----------------------------
@@ -345,7 +346,7 @@ __device__ bool static_tile(const FusedArgs& f, uint32_t idx, TileDesc* d)
     return true;
 }
 
-template <bool kHasQ, bool kFused>
+template <bool kHasQ, bool kFused, bool kLayer = false>
 __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, int bar_id, int te,
                            uint32_t first, uint32_t stride, const CUtensorMap* tm_k,
                            const CUtensorMap* tm_q, const CUtensorMap* tm_v)
@@ -373,7 +374,29 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
     // thread (w, c4) owns rows 8w..8w+7 and channels 4c4..4c4+3 in the gating phase
     const int c4 = lane, d0 = c4 * 4, i0 = warp * kRPT;
     float G[kRPT][4];
+    float rate = 0.f, bias[4] = {0.f, 0.f, 0.f, 0.f};   // layer mode: decay-function parameters of the tile's head
     auto prefetch_regs = [&](const TileDesc& D) {
+        if (kLayer) {
+            // bf16 pre-activations of the decay function; the function itself is applied at the top of
+            // the tile, when the registers are next looked at
+            const __nv_bfloat16* gp = reinterpret_cast<const __nv_bfloat16*>(a.log_alpha) +
+                                      ((size_t)D.tok0 * a.H + D.h) * kD + d0;
+#pragma unroll
+            for (int r = 0; r < kRPT; ++r) {
+                const int i = i0 + r;
+                uint32_t lo = 0u, hi = 0u;
+                if (i < D.len)
+                    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];"
+                                 : "=r"(lo), "=r"(hi)
+                                 : "l"(gp + (size_t)i * a.H * kD));
+                G[r][0] = __uint_as_float(lo << 16); G[r][1] = __uint_as_float(lo & 0xffff0000u);
+                G[r][2] = __uint_as_float(hi << 16); G[r][3] = __uint_as_float(hi & 0xffff0000u);
+            }
+            rate = a.gate_rate[D.h];
+            const float4 b4 = *reinterpret_cast<const float4*>(a.gate_bias + (size_t)D.h * kD + d0);
+            bias[0] = b4.x; bias[1] = b4.y; bias[2] = b4.z; bias[3] = b4.w;
+            return;
+        }
         const float* gp = a.log_alpha + ((size_t)D.tok0 * a.H + D.h) * kD + d0;
 #pragma unroll
         for (int r = 0; r < kRPT; ++r) {
@@ -454,6 +477,18 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         char* tile = D.tile;
         KT_MARK(te == 0, 0);   // loop overhead
 
+        if (kLayer) {
+            // log alpha = -exp(rate) * softplus(x + bias); rows past the end of the sequence do not decay
+            const float nr = -__expf(rate);
+#pragma unroll
+            for (int r = 0; r < kRPT; ++r)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float x = G[r][e] + bias[e];
+                    const float sp = fmaxf(x, 0.f) + __logf(1.f + __expf(-fabsf(x)));
+                    G[r][e] = (i0 + r < D.len) ? nr * sp : 0.f;
+                }
+        }
         // ---- a1: cumulative log-decay, in the log2 domain (exponentials below are bare ex2) ---------
 #pragma unroll
         for (int e = 0; e < 4; ++e) G[0][e] *= kLog2e;
@@ -482,6 +517,8 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         if (te == kSchedThread) atomicAdd(&f.hdr->pad[11], (int)((ptx::globaltimer_ns() - ts0_) >> 4));
 #endif
         ptx::cp_async_wait_all();             // beta
+        if (kLayer && te < kC)                // (each of these threads copied its own element)
+            sBeta[te] = te < D.len ? 1.f / (1.f + __expf(-sBeta[te])) : 0.f;
         ebar();
         KT_MARK(te == 0, 1);   // scan + publish + slot wait
         if (*abort_word) break;
@@ -526,6 +563,41 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
         // ---- gated operands ---------------------------------------------------------------------------
         // (two copies of the loop, chosen per warp: without the clamp when no channel of the warp's
         // share of the tile can reach it, since |G_i - G_m| <= |G_C| / 2)
+        float* sNorm = reinterpret_cast<float*>(smem + E_NORM);
+        if (kLayer) {
+            // L2Norm of k and q: the warp owns its eight rows whole (32 lanes x 4 channels)
+            const int hf = c4 >> 4;
+            float ssk[kRPT], ssq[kRPT];
+#pragma unroll
+            for (int r = 0; r < kRPT; ++r) {
+                const int i = i0 + r;
+                const uint32_t o2 = (uint32_t)(i * 128 + ((((c4 >> 1) & 7) ^ (i & 7)) << 4) + (c4 & 1) * 8);
+                const uint2 k2 = *reinterpret_cast<const uint2*>(smem + E_KS + hf * 8192 + o2);
+                uint2 q2 = make_uint2(0u, 0u);
+                if (has_q) q2 = *reinterpret_cast<const uint2*>(smem + E_KQ + hf * E_KQ_HALF + o2 + 8192);
+                const float k0 = __uint_as_float(k2.x << 16), k1 = __uint_as_float(k2.x & 0xffff0000u);
+                const float k2f = __uint_as_float(k2.y << 16), k3 = __uint_as_float(k2.y & 0xffff0000u);
+                const float q0 = __uint_as_float(q2.x << 16), q1 = __uint_as_float(q2.x & 0xffff0000u);
+                const float q2f = __uint_as_float(q2.y << 16), q3 = __uint_as_float(q2.y & 0xffff0000u);
+                ssk[r] = k0 * k0 + k1 * k1 + k2f * k2f + k3 * k3;
+                ssq[r] = q0 * q0 + q1 * q1 + q2f * q2f + q3 * q3;
+            }
+#pragma unroll
+            for (int s = 16; s >= 1; s >>= 1)
+#pragma unroll
+                for (int r = 0; r < kRPT; ++r) {
+                    ssk[r] += __shfl_xor_sync(0xffffffffu, ssk[r], s);
+                    ssq[r] += __shfl_xor_sync(0xffffffffu, ssq[r], s);
+                }
+#pragma unroll
+            for (int r = 0; r < kRPT; ++r)
+                if (lane == r) {   // (rows past the end of the sequence are zeroed below: keep their factor finite)
+                    const bool in = i0 + r < D.len;
+                    sNorm[i0 + r] = in ? rsqrtf(ssk[r] + a.l2_eps) : 0.f;
+                    sNorm[kC + i0 + r] = in ? rsqrtf(ssq[r] + a.l2_eps) : 0.f;
+                }
+            __syncwarp();
+        }
         auto gate_rows = [&](auto clamp_tag) {
             constexpr bool kClamp = decltype(clamp_tag)::value;
             const int hf = c4 >> 4;                       // K-half (channels 0-63 / 64-127)
@@ -546,15 +618,25 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                 const float qf[4] = {__uint_as_float(q2.x << 16), __uint_as_float(q2.x & 0xffff0000u),
                                      __uint_as_float(q2.y << 16), __uint_as_float(q2.y & 0xffff0000u)};
                 float okg[4], oqg[4], oki[4];
+                float rk = 1.f, rq = a.scale;
+                if (kLayer) {
+                    rk = sNorm[i];
+                    rq = a.scale * sNorm[kC + i];
+                }
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     float x = G[r][e] + off[e];
                     if (kClamp) x = fminf(fmaxf(x, -kClamp2), kClamp2);
                     const float e1 = ex2(x);                     // exp(G - G_m)
                     const float e2 = ex2(-x);                    // exp(G_m - G)
-                    okg[e] = kf[e] * e1;
-                    oqg[e] = a.scale * qf[e] * e1;
-                    oki[e] = kf[e] * e2;
+                    if (kLayer) {
+                        okg[e] = kf[e] * (e1 * rk);
+                        oki[e] = kf[e] * (e2 * rk);
+                    } else {
+                        okg[e] = kf[e] * e1;
+                        oki[e] = kf[e] * e2;
+                    }
+                    oqg[e] = rq * qf[e] * e1;
                 }
                 *reinterpret_cast<uint2*>(pk) = make_uint2(pack_bf16(okg[0], okg[1]), pack_bf16(okg[2], okg[3]));
                 if (has_q)
@@ -1386,7 +1468,7 @@ kda_fused_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtens
 
 // ---- the intra-chunk stage alone (first kernel of the two-kernel schedule) --------------------------------
 // Persistent CTAs of one engine each, two per SM; the tiles of the pass go to a plain array.
-template <bool kHasQ>
+template <bool kHasQ, bool kLayer>
 __global__ void __launch_bounds__(kEngThreads, 2)
 kda_intra_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtensorMap tm_k,
              const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_v,
@@ -1424,7 +1506,7 @@ kda_intra_tc(const __grid_constant__ FusedArgs f, const __grid_constant__ CUtens
     if ((ptx::smem_u32(smem) & 1023u) != 0) {
         if (t == 0) report_timeout(f, 90);   // the operand images need 1024-byte alignment
     } else {
-        engine_run<kHasQ, false>(f, smem, tmem_base, 1, t, blockIdx.x, gridDim.x, &tm_k, &tm_q, &tm_v);
+        engine_run<kHasQ, false, kLayer>(f, smem, tmem_base, 1, t, blockIdx.x, gridDim.x, &tm_k, &tm_q, &tm_v);
     }
     ptx::tc_fence_before();
     __syncthreads();
@@ -1534,9 +1616,13 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, boo
         DeviceLock lk;
         if (!lk.st) return lk.rc;
         if (!lk.st->attr_done[1]) {
-            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)E_BYTES));
-            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)E_BYTES));
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)E_BYTES));
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_intra_tc<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)E_BYTES));
             lk.st->attr_done[1] = true;
         }
@@ -1565,10 +1651,15 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, boo
     const int64_t resident = 2 * (int64_t)n_sm;   // two CTAs per SM
     const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
     ProfScope ps(PROF_INTRA, st);
-    if (has_q)
-        kda_intra_tc<true><<<grid, kEngThreads, E_BYTES, st>>>(f, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
+    const bool layer = a.gate_rate != nullptr;
+    if (layer && has_q)
+        kda_intra_tc<true, true><<<grid, kEngThreads, E_BYTES, st>>>(f, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
+    else if (layer)
+        kda_intra_tc<false, true><<<grid, kEngThreads, E_BYTES, st>>>(f, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
+    else if (has_q)
+        kda_intra_tc<true, false><<<grid, kEngThreads, E_BYTES, st>>>(f, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
     else
-        kda_intra_tc<false><<<grid, kEngThreads, E_BYTES, st>>>(f, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
+        kda_intra_tc<false, false><<<grid, kEngThreads, E_BYTES, st>>>(f, tm_k, tm_q, tm_v, clear_status ? 1 : 0);
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;
