@@ -158,8 +158,13 @@ kda_status_t kda_chunk_fwd_static(const void *q, const void *k, const void *v,
  *
  * The normalisation, the decay function and the sigmoid of beta are computed inside the
  * intra-chunk kernel from the half-precision pre-activations (no fp32 gate tensor and no
- * normalised copy of q and k ever exists in memory); the output stage runs as a separate pass over
- * the bf16 output, in place.
+ * normalised copy of q and k ever exists in memory).  The output stage runs inside the inter-chunk
+ * kernel: the CTAs that hold the column slices of one (sequence, head) are launched as a thread-block
+ * cluster and exchange each row's sums of squares through distributed shared memory.  Where the
+ * device cannot keep as many clusters resident as the call has work for (or after
+ * kda_layer_set_fused_output(0)), the stage runs as a separate pass over the bf16 output, in place;
+ * the results of the two forms differ by rounding only (the separate pass normalises the rounded
+ * bf16 output).
  *
  *   q_c, k_c, g_a [T_total,H,dk], v, g_o, y [T_total,H,dv]   bf16 device
  *   b_pre [T_total,H]                                        fp32 device
@@ -171,6 +176,8 @@ kda_status_t kda_chunk_fwd_static(const void *q, const void *k, const void *v,
  * Only dk = dv = 128 and chunk = 64.  Asynchronous; nothing is allocated; errors and the status
  * word as for kda_chunk_fwd.
  */
+/* Process-wide switch (default 1): 0 makes kda_layer_fwd always run its output stage as a pass of its own. */
+kda_status_t kda_layer_set_fused_output(int on);
 size_t kda_layer_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv, int chunk);
 size_t kda_layer_fwd_min_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv, int chunk);
 kda_status_t kda_layer_fwd(const void *q_c, const void *k_c, const void *v, const void *g_a,

@@ -74,6 +74,8 @@ def load():
     lib.kda_layer_fwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
     lib.kda_layer_fwd_min_workspace_bytes.restype = sz
     lib.kda_layer_fwd_min_workspace_bytes.argtypes = [i64, i32, i32, i32, i32, i32]
+    lib.kda_layer_set_fused_output.restype = i32
+    lib.kda_layer_set_fused_output.argtypes = [i32]
     lib.kda_layer_fwd.restype = i32
     lib.kda_layer_fwd.argtypes = [vp] * 9 + [f32, f32, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32,
                                              vp, sz, vp]
@@ -247,6 +249,12 @@ def kda_chunk_bwd(q, k, v, log_alpha, beta, S0, d_o, dS_T, dq, dk_out, dv_out, d
         int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale), int(dt),
         _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
     _check(rc)
+
+
+def kda_layer_set_fused_output(on: bool) -> None:
+    """False: ``kda_layer_fwd`` runs its output stage as a separate pass (default: inside the
+    inter-chunk kernel when the device can hold the clusters this needs)."""
+    _check(load().kda_layer_set_fused_output(1 if on else 0))
 
 
 def kda_layer_fwd_workspace_bytes(total_tokens, n_seqs, H, dk=128, dv=128, chunk=64) -> int:

@@ -179,7 +179,8 @@ FusedPlan fused_plan(const std::vector<int64_t>& chunk_cu, int n_seqs, int H, in
     }
     return P;
 }
-std::atomic<int> g_chunk_path{0};   // 0 = automatic, 1 = always two kernels, 2 = always the fused kernel
+std::atomic<int> g_chunk_path{0};
+std::atomic<int> g_fuse_output{1};  // kda_layer_fwd: 1 = output stage inside the inter-chunk kernel when possible   // 0 = automatic, 1 = always two kernels, 2 = always the fused kernel
 
 }  // namespace
 }  // namespace kda
@@ -265,6 +266,9 @@ struct LayerMode {
     const float* rate = nullptr;
     const float* bias = nullptr;
     float l2_eps = 0.f;
+    const void* out_gate = nullptr;     // non-null: the output stage runs inside the inter-chunk kernel
+    const float* rms_weight = nullptr;
+    float rms_eps = 0.f;
 };
 
 kda_status_t chunk_fwd_impl(const void* q, const void* k, const void* v, const float* log_alpha,
@@ -424,6 +428,7 @@ kda_status_t chunk_fwd_impl(const void* q, const void* k, const void* v, const f
     a.chunks_per_seq = chunks_per_seq; a.scale = scale;
     a.S_out = state;
     a.gate_rate = lm.rate; a.gate_bias = lm.bias; a.l2_eps = lm.l2_eps;
+    a.out_gate = lm.out_gate; a.rms_weight = lm.rms_weight; a.rms_eps = lm.rms_eps;
 
     int64_t g0 = 0;
     bool first = true;
@@ -467,6 +472,12 @@ kda_status_t kda_chunk_fwd(const void* q, const void* k, const void* v, const fl
                           LayerMode());
 }
 
+kda_status_t kda_layer_set_fused_output(int on)
+{
+    g_fuse_output.store(on ? 1 : 0, std::memory_order_relaxed);
+    return KDA_OK;
+}
+
 size_t kda_layer_fwd_workspace_bytes(int64_t total_tokens, int n_seqs, int H, int dk, int dv, int chunk)
 {
     return kda_chunk_fwd_workspace_bytes(total_tokens, n_seqs, H, dk, dv, chunk, KDA_BF16);
@@ -496,10 +507,17 @@ kda_status_t kda_layer_fwd(const void* q_c, const void* k_c, const void* v, cons
                                        "aligned", p);
     LayerMode lm;
     lm.rate = A_log; lm.bias = dt_bias; lm.l2_eps = l2_eps;
+    // The output stage runs inside the inter-chunk kernel when the device can hold the clusters this
+    // needs (the slices of a row exchange their sums of squares), else as a pass of its own.
+    const bool fuse_out = y && total_tokens > 0 && n_seqs > 0 && g_fuse_output.load(std::memory_order_relaxed) &&
+                          inter_can_fuse_epilogue((int64_t)n_seqs * H);
+    if (fuse_out) {
+        lm.out_gate = g_o; lm.rms_weight = rms_weight; lm.rms_eps = rms_eps;
+    }
     kda_status_t rc = chunk_fwd_impl(q_c, k_c, v, reinterpret_cast<const float*>(g_a), b_pre, S0, y, S_T,
                                      cu_seqlens_dev, cu_seqlens_host, n_seqs, total_tokens, H, dk, dv, chunk,
                                      scale, KDA_BF16, workspace, workspace_bytes, cuda_stream, lm);
-    if (rc != KDA_OK || !y || total_tokens == 0 || n_seqs == 0) return rc;
+    if (rc != KDA_OK || !y || total_tokens == 0 || n_seqs == 0 || fuse_out) return rc;
     return launch_layer_epilogue(y, g_o, rms_weight, rms_eps, total_tokens * H,
                                  static_cast<cudaStream_t>(cuda_stream));
 }

@@ -22,6 +22,8 @@
 // TMEM, read back with tcgen05.ld.
 // Every wait is bounded: on a timeout the CTA records KDA_ERR_TIMEOUT in the workspace header,
 // drains its copies, frees its TMEM and returns.
+#include <cstring>
+
 #include "kda_common.cuh"
 #include "kda_ptx.cuh"
 #include "kda_tiles.cuh"
@@ -50,7 +52,10 @@ template <int NS> struct InterCfg {
     static constexpr uint32_t kSbf = kStages * kStage;      // B operand of MMA1, MN-major: [128 dk rows][128 B]
     static constexpr uint32_t kVn = kSbf + 128 * 128;       // B operand of MMA2, MN-major: [64 token rows][128 B]
     static constexpr uint32_t kBars = kVn + 64 * 128;
-    static constexpr uint32_t kTotal = kBars + 128;
+    static constexpr uint32_t kSsq = kBars + 256;           // output stage: [2][slices][64] fp32 row sums of squares
+    static constexpr uint32_t kWgt = kSsq + 2 * (128 / NS) * 64 * 4;   // output stage: this slice's NS RMSNorm weights
+    static constexpr uint32_t kGate = (kWgt + NS * 4 + 127) / 128 * 128;   // output stage: four [32 rows][NS] bf16 gate blocks
+    static constexpr uint32_t kTotal = kGate + (NS == 32 ? 4 * 32 * NS * 2 : 0);   // (the output stage runs with 32-column slices only)
     static constexpr uint32_t kSmem = kTotal + 1024;        // slack for manual 1024-byte alignment
     static constexpr uint32_t kTxBytes = kMainBytes + kUBytes;
     static constexpr uint32_t kTmemCols = 3 * kNCtrl * NS <= 256 ? 256 : 512;   // 2 kNCtrl x D1 + kNCtrl x D3, NS columns each
@@ -69,6 +74,12 @@ __device__ __forceinline__ void tmem_ld_sum(uint32_t taddr, float (&acc)[NS]) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) acc[blk * 32 + j] = __uint_as_float(r[j]) + __uint_as_float(r2[j]);
     }
+}
+// 1 / x by the special-function unit alone (no rounding fix-up, no branches: 32 of them interleave)
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
     __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
@@ -91,11 +102,19 @@ __device__ __forceinline__ void store_row(uint8_t* img, int row, const float (&x
 // the MMAs (and, in warp 4, the bulk copies).  The roles meet only on mbarriers, so issue
 // latencies never sit on the compute warps' path and the output conversion overlaps the next
 // chunk's first MMA.
-template <int NS>
-__global__ void __launch_bounds__(128 + 32 * kNCtrl, 1)
-kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader* hdr)
+//
+// kEpi (launched as clusters of the kD / NS slice CTAs of one (sequence, head)): the output stage of
+// the layer wrap runs on the output rows before they are stored.  The mean square of a row spans
+// the slices, so every CTA writes its share of the row's sum of squares into the shared memory of
+// all CTAs of the cluster and arrives on their barriers; two buffers used alternately suffice,
+// because nobody can send chunk g + 2 before everybody has finished reading chunk g.
+template <int NS, bool kEpi>
+__global__ void __launch_bounds__(kEpi ? 384 : 128 + 32 * kNCtrl, 1)
+kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader* hdr,
+             const __grid_constant__ CUtensorMap tm_g)
 {
     using Cfg = InterCfg<NS>;
+    constexpr int NSL = kD / NS;   // slices = CTAs of a cluster
     constexpr int NSTG = Cfg::kStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(
@@ -110,6 +129,11 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     uint64_t* vn_ready = sbf_ready + 1;    // 2 warp arrivals: V_new written
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(vn_ready + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint64_t* ssq_bar = vn_ready + 2;      // [2] the sums of squares of every slice's 64 rows have landed
+    uint64_t* o_done = ssq_bar + 2;        // [2] (kEpi) the output warps have read a chunk's accumulator
+    uint64_t* gate_bar = o_done + 2;       // [4] (kEpi) an output warp's block of gate pre-activations has landed
+    float* ssq = reinterpret_cast<float*>(smem + Cfg::kSsq);
+    float* s_wgt = reinterpret_cast<float*>(smem + Cfg::kWgt);
     uint8_t* sbf = smem + Cfg::kSbf;
     uint8_t* vn = smem + Cfg::kVn;
 
@@ -140,6 +164,12 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         ptx::mbar_init(&out_bar[1], 1);
         ptx::mbar_init(sbf_ready, 4);    // one arrival per compute warp (after a warp-level sync)
         ptx::mbar_init(vn_ready, 2);
+        ptx::mbar_init(&ssq_bar[0], 1);
+        ptx::mbar_init(&ssq_bar[1], 1);
+        ptx::mbar_init(&o_done[0], 2);
+        ptx::mbar_init(&o_done[1], 2);
+#pragma unroll
+        for (int w4 = 0; w4 < 4; ++w4) ptx::mbar_init(&gate_bar[w4], 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -147,8 +177,10 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         ptx::tmem_alloc(tmem_slot, Cfg::kTmemCols);
         ptx::tmem_relinquish();
     }
+    if (kEpi && tid < NS) s_wgt[tid] = a.rms_weight[slice * NS + tid];
     ptx::tc_fence_before();
     __syncthreads();
+    if (kEpi) ptx::cluster_sync_all();   // every CTA's barriers exist before anybody arrives on them
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t d3 = 2 * kNCtrl * NS;   // TMEM columns: D1 {parity 0,1} x {part} first, then the D3 parts
@@ -161,7 +193,89 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
         }
     };
 
-    if (warp >= 4) {
+    // a7: O = (Gamma.Q) S + Aqk V_new for token row i of chunk `it` (a thread of TMEM lanes 64-127);
+    // kEpi: followed by the output stage of the layer wrap
+    auto output_row = [&](int it, int i, uint32_t tmem_lane, const uint4 (&gq)[NS / 8]) {
+        const uint32_t d1 = (uint32_t)(it & 1) * kNCtrl * NS;
+        const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
+        const int len = (tok_end - tok0) < kC ? (int)(tok_end - tok0) : kC;
+        __nv_bfloat16* orow = op + ((tok0 + i) * a.H + h) * kD + col0;
+        wait(&out_bar[it & 1], (uint32_t)(it >> 1) & 1u, 6);
+        ptx::tc_fence_after();
+        float ov[NS];
+        tmem_ld_sum<NS>(tmem_lane + d1, ov);
+        ptx::tc_fence_before();
+        if (kEpi) {
+            // the accumulator may be written again; this slice's share of the row's sum of squares
+            // goes to every CTA of the cluster
+            __syncwarp();
+            if ((tid & 31) == 0) ptx::mbar_arrive(&o_done[it & 1]);
+            const int b = it & 1;
+            const uint32_t rank = ptx::cluster_ctarank();
+            float part = 0.f;
+#pragma unroll
+            for (int j = 0; j < NS; ++j) part = fmaf(ov[j], ov[j], part);
+            // (asynchronous stores that report their bytes to the receiver's barrier: nothing to fence)
+            const uint32_t slot = ptx::smem_u32(ssq + (b * NSL + (int)rank) * kC + i);
+            const uint32_t bar = ptx::smem_u32(&ssq_bar[b]);
+#pragma unroll
+            for (int r = 0; r < NSL; ++r)
+                ptx::st_async_cluster_f32(ptx::map_to_cta(slot, (uint32_t)r), part, ptx::map_to_cta(bar, (uint32_t)r));
+            // one thread per CTA and chunk arms the own barrier: the 64 rows of every slice, 4 bytes each
+            if (i == 0) ptx::mbar_expect_tx(&ssq_bar[b], NSL * kC * 4);
+            if (!*abort_flag && !ptx::mbar_wait_cluster(&ssq_bar[b], (uint32_t)(it >> 1) & 1u, kWaitLimitNs)) {
+                *abort_flag = 1;
+                if (atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = 9;
+            }
+            float tot = 0.f;
+#pragma unroll
+            for (int r = 0; r < NSL; ++r) tot += ssq[(b * NSL + r) * kC + i];
+            const float rstd = rsqrtf(tot * (1.f / kD) + a.rms_eps);
+            const __nv_bfloat16* G = reinterpret_cast<const __nv_bfloat16*>(gq);
+#pragma unroll
+            for (int j = 0; j < NS; ++j)
+                ov[j] = ov[j] * (rstd * s_wgt[j]) * rcp_approx(1.f + __expf(-__bfloat162float(G[j])));
+        }
+        if (i < len) {
+#pragma unroll
+            for (int j = 0; j < NS; j += 8)
+                *reinterpret_cast<uint4*>(orow + j) =
+                    make_uint4(pack2(ov[j], ov[j + 1]), pack2(ov[j + 2], ov[j + 3]),
+                               pack2(ov[j + 4], ov[j + 5]), pack2(ov[j + 6], ov[j + 7]));
+        }
+    };
+
+    if (warp >= 6) {
+        // ================= output warps (kEpi launches only) =================
+        // Warps 6, 7 take the even chunks, warps 10, 11 the odd ones (TMEM lanes 64-127 belong to warps
+        // with index 2 or 3 modulo 4), so each has two steps of the chain for one chunk's rows.  Each
+        // fetches its own 32 rows of gate pre-activations one chunk ahead with a 2-D tiled TMA load.
+        if (kEpi && op && (warp & 3) >= 2) {
+            const int lane = tid & 31, q2 = (warp & 3) - 2, set = warp >= 10 ? 1 : 0;
+            const uint32_t tmem_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+            uint8_t* gbuf = smem + Cfg::kGate + (set * 2 + q2) * (32 * NS * 2);
+            uint64_t* gbar = &gate_bar[set * 2 + q2];
+            auto request_gate = [&](int it) {
+                const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
+                ptx::mbar_expect_tx(gbar, 32 * NS * 2);
+                ptx::tma_load_2d(gbuf, &tm_g, h * kD + col0, (int)(tok0 + q2 * 32), gbar);
+            };
+            if (lane == 0 && set < nchunks) request_gate(set);
+            uint32_t k = 0;
+            for (int it = set; it < nchunks; it += 2, ++k) {
+                uint4 gq[NS / 8];
+                wait(gbar, k & 1u, 11);
+#pragma unroll
+                for (int c = 0; c < NS / 8; ++c) gq[c] = *reinterpret_cast<const uint4*>(gbuf + lane * (NS * 2) + c * 16);
+                __syncwarp();
+                if (lane == 0 && it + 2 < nchunks) {
+                    ptx::fence_async_smem();   // the rows were read before the next block lands over them
+                    request_gate(it + 2);
+                }
+                output_row(it, q2 * 32 + lane, tmem_lane, gq);
+            }
+        }
+    } else if (warp >= 4) {
         // ================= control warps: lane 0 of each issues MMAs =================
         // Issuing one tcgen05.mma costs the issuing thread several tens of cycles whatever the tile
         // size, and both products on the sequential chain are tiny, so each is split along its
@@ -196,6 +310,9 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 // MMA1(it): D1 = [W ; Gamma.Q] S, this thread's half of the sum over dk
                 wait(&full[s], (uint32_t)(it / NSTG) & 1u, 1);
                 wait(sbf_ready, (uint32_t)it & 1u, 4);
+                // (kEpi: the output rows are read by warps of their own, which may lag: this chunk's
+                // accumulator is the one of chunk it - 2)
+                if (kEpi && op && it >= 2) wait(&o_done[it & 1], (uint32_t)((it >> 1) - 1) & 1u, 10);
                 ptx::tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < 8 / kNCtrl; ++k) {
@@ -318,23 +435,9 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::tc_fence_before();
                 warp_arrive(sbf_ready);
             }
-            if (warp >= 2 && op) {   // a7: O = (Gamma.Q) S + Aqk V_new  (token row = tid - 64)
-                const int i = tid - 64;
-                const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
-                const int len = (tok_end - tok0) < kC ? (int)(tok_end - tok0) : kC;
-                __nv_bfloat16* orow = op + ((tok0 + i) * a.H + h) * kD + col0;
-                wait(&out_bar[it & 1], (uint32_t)(it >> 1) & 1u, 6);
-                ptx::tc_fence_after();
-                float ov[NS];
-                tmem_ld_sum<NS>(tmem_lane + d1, ov);
-                if (i < len) {
-#pragma unroll
-                    for (int j = 0; j < NS; j += 8)
-                        *reinterpret_cast<uint4*>(orow + j) =
-                            make_uint4(pack2(ov[j], ov[j + 1]), pack2(ov[j + 2], ov[j + 3]),
-                                       pack2(ov[j + 4], ov[j + 5]), pack2(ov[j + 6], ov[j + 7]));
-                }
-                ptx::tc_fence_before();
+            if (!kEpi && warp >= 2 && op) {
+                const uint4 no_gate[NS / 8] = {};
+                output_row(it, tid - 64, tmem_lane, no_gate);
             }
         }
         if (*abort_flag == 0) {
@@ -346,6 +449,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (kEpi) ptx::cluster_sync_all();   // no CTA leaves while another may still write into its shared memory
     if (warp == 0) ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
 }
 
@@ -354,15 +458,29 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
                                WsHeader* hdr, bool after_intra, cudaStream_t st)
 {
     using Cfg = InterCfg<NS>;
+    const bool want_epi = NS == 32 && a.out_gate != nullptr && a.o != nullptr;
+    if (a.out_gate != nullptr && a.o != nullptr && !want_epi)
+        return fail(KDA_ERR_UNSUPPORTED, "the fused output stage runs with 32-column slices only");
     {
         DeviceLock lk;
         if (!lk.st) return lk.rc;
         const int slot = NS == 32 ? 2 : 3;
         if (!lk.st->attr_done[slot]) {
-            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_tc<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_tc<NS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)Cfg::kSmem));
+            if (NS == 32)
+                KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_tc<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                  (int)InterCfg<32>::kSmem));
             lk.st->attr_done[slot] = true;
         }
+    }
+    CUtensorMap tm_g;
+    memset(&tm_g, 0, sizeof(tm_g));
+    if (want_epi) {
+        if (a.total_tokens > 0x7fffffff)
+            return fail(KDA_ERR_UNSUPPORTED, "kda_layer_fwd: more than 2^31 tokens in one call");
+        kda_status_t rc = make_plain_tmap(&tm_g, a.out_gate, a.total_tokens, a.H, NS, 32);
+        if (rc != KDA_OK) return rc;
     }
     ProfScope ps(PROF_INTER, st);
     cudaLaunchConfig_t cfg = {};
@@ -370,14 +488,31 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
     cfg.blockDim = dim3(128 + 32 * kNCtrl);
     cfg.dynamicSmemBytes = Cfg::kSmem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
     // only overlap with this library's own intra-chunk kernel, never with a caller's kernel that may
     // still be producing S0
-    cfg.numAttrs = after_intra ? 1 : 0;
-    KDA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kda_inter_tc<NS>, a, tiles, n_begin, hdr));
+    if (after_intra) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
+    if (want_epi) {
+        // the slice CTAs of one (sequence, head) form a cluster (the caller has checked that enough
+        // of them fit the device at once: inter_can_fuse_epilogue)
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = kD / NS;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        cfg.numAttrs = na + 1;
+        cfg.blockDim = dim3(384);   // warps 6, 7, 10, 11: the output rows
+        KDA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kda_inter_tc<32, true>, a, tiles, n_begin, hdr, tm_g));
+        count_launch();
+        return KDA_OK;
+    }
+    KDA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kda_inter_tc<NS, false>, a, tiles, n_begin, hdr, tm_g));
     count_launch();
     return KDA_OK;
 }
@@ -405,6 +540,49 @@ kda_status_t launch_wait_selftest(WsHeader* hdr, uint64_t limit_ns, cudaStream_t
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;
+}
+
+namespace {
+bool clusters_fit(int64_t groups, int n_sm)
+{
+    using Cfg = InterCfg<32>;
+    if (cudaFuncSetAttribute(kda_inter_tc<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Cfg::kSmem) != cudaSuccess)
+        return false;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kD / 32, 1, 1);
+    cfg.blockDim = dim3(384);
+    cfg.dynamicSmemBytes = Cfg::kSmem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kD / 32;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kda_inter_tc<32, true>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    const int64_t plain = n_sm / (kD / 32);   // groups of slice CTAs that a launch without clusters holds
+    return n >= (groups < plain ? groups : plain);
+}
+}  // namespace
+
+// Whether the output stage of the layer wrap can run inside the inter-chunk kernel for a call with
+// `groups` (sequence, head) pairs: its slice CTAs then form clusters, and a GPC holds fewer clusters
+// than its SM count suggests; if the device cannot keep as many (sequence, head) pairs in flight as
+// without clusters, or the call is large enough for 64-column slices, the stage runs as a separate
+// pass instead.
+bool inter_can_fuse_epilogue(int64_t groups)
+{
+    int n_sm = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return false;
+    if (groups * 4 > 2 * (int64_t)n_sm) return false;   // the launcher picks 64-column slices there
+    return clusters_fit(groups, n_sm);
 }
 
 size_t tc_tile_bytes() { return tc::TILE_BYTES; }

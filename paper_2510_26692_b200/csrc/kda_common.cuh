@@ -1,6 +1,7 @@
 // Internal helpers shared by the translation units of the KDA library (host side error plumbing,
 // launch accounting, workspace header layout, small device utilities).  Not part of the C ABI.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -70,6 +71,11 @@ struct ChunkArgs {
     const float* gate_rate = nullptr;   // [H]
     const float* gate_bias = nullptr;   // [H, dk]
     float l2_eps = 0.f;
+    // Output stage of the layer wrap inside the inter-chunk kernel (off when out_gate is nullptr):
+    // o is replaced by sigmoid(out_gate) . RMSNorm(o) . rms_weight before it is stored.
+    const void* out_gate = nullptr;     // bf16 [T_total, H, dv]
+    const float* rms_weight = nullptr;  // [dv]
+    float rms_eps = 0.f;
 };
 
 // Work description of the fused bf16 chunk-forward kernel (one cooperative launch per call).
@@ -171,6 +177,8 @@ kda_status_t launch_chunk_simt(const ChunkArgs& a, kda_dtype_t dt, void* tiles, 
 size_t tc_tile_bytes();
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
                              WsHeader* hdr, bool clear_status, cudaStream_t st);
+bool inter_can_fuse_epilogue(int64_t groups);
+kda_status_t make_plain_tmap(CUtensorMap* tm, const void* base, int64_t total_tokens, int H, int cols, int rows);
 
 // fused bf16 path: workspace bytes besides the ring (flags and round table), and the launcher
 size_t fused_fixed_bytes(int n_seqs, int H);

@@ -1595,6 +1595,23 @@ kda_status_t make_tmap(CUtensorMap* tm, const void* base, int64_t total_tokens, 
 
 }  // namespace
 
+// [total_tokens, H*128] bf16 matrix, boxes of `rows` tokens x `cols` channels, no swizzle (rows of the
+// box land back to back); used for the output-gate blocks of the layer wrap
+kda_status_t make_plain_tmap(CUtensorMap* tm, const void* base, int64_t total_tokens, int H, int cols, int rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return fail(KDA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    const cuuint64_t dims[2] = {(cuuint64_t)H * kD, (cuuint64_t)total_tokens};
+    const cuuint64_t strides[1] = {(cuuint64_t)H * kD * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)cols, (cuuint32_t)rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(KDA_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return KDA_OK;
+}
+
 // (tc_tile_bytes is defined beside the two-kernel path)
 
 kda_status_t launch_fused_prep(WsHeader* hdr, const int32_t* cu_seqlens, uint32_t* round_base, int n_seqs,

@@ -87,3 +87,24 @@ def test_layer_equals_plain_call_on_precomputed_inputs(oracle_mod):
              "S0": d["S0"], "cu_seqlens": d["cu_seqlens"]}
     _, S_plain = run_chunk(plain)
     assert rel_l2(to_np32(S_layer), to_np32(S_plain)) <= 5e-3
+
+
+def test_layer_output_stage_fused_and_separate_agree(oracle_mod):
+    """The output stage inside the inter-chunk kernel (clusters exchanging the rows' sums of squares)
+    against the same stage as a separate pass: both within tolerance of the oracle, and close to each
+    other (the separate pass normalises the bf16-rounded output)."""
+    scale = 128 ** -0.5
+    for lens, H in (([700, 130, 64], 4), ([2048], 40)):      # 40 heads: more chains than 32-column slices fit
+        d = inputs.layer_inputs(lens, H=H, seed=44, s0_std=0.02)
+        try:
+            K.kda_layer_set_fused_output(False)
+            y_sep, S_sep = run_layer(d, scale)
+        finally:
+            K.kda_layer_set_fused_output(True)
+        y_fus, S_fus = run_layer(d, scale)
+        y_ref, S_ref, _ = oracle_layer(oracle_mod, d, scale)
+        assert torch.equal(S_sep, S_fus)
+        e_sep, e_fus = rel_l2(to_np32(y_sep), y_ref), rel_l2(to_np32(y_fus), y_ref)
+        print("output stage", lens, H, "separate", e_sep, "fused", e_fus)
+        assert e_sep <= TOL and e_fus <= TOL
+        assert rel_l2(to_np32(y_fus), to_np32(y_sep)) <= 1e-2
