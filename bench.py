@@ -407,6 +407,9 @@ def main():
                     help="kda_set_chunk_path mode for the timed prefill: 0 automatic, 1 two kernels, 2 fused kernel")
     ap.add_argument("--prefill-only", action="store_true",
                     help="time only the device-resident prefill loop (short runs under a profiler)")
+    ap.add_argument("--only", default=None, choices=["layer", "backward", "dplr"],
+                    help="run one of the side figures alone (layer wrap, backward pass, DPLR comparison) and "
+                         "print it as a partial JSON line; for profiling")
     ap.add_argument("--decode-only", action="store_true",
                     help="time only the decode loop (short runs under a profiler)")
     args = ap.parse_args()
@@ -442,6 +445,12 @@ def main():
 
     if args.decode_only:
         return decode_only(args, K, inputs, torch, dev, peaks)
+    if args.only:
+        fn = {"layer": layer_figure, "backward": backward_figure, "dplr": dplr_comparison}[args.only]
+        out = fn(K, inputs, torch, dev, peaks)
+        if rank == 0:
+            print(json.dumps({"partial": args.only, "gpu_launches": K.kda_launch_count(), args.only: out}))
+        return 0
     K.kda_set_chunk_path(args.chunk_path)
 
     # ---- prefill workload: 3 input copies (each 206 MB > L2) rotated between steps ---------------

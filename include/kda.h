@@ -196,7 +196,8 @@ kda_status_t kda_layer_fwd(const void *q_c, const void *k_c, const void *v, cons
  *
  * it returns dL/dq, dL/dk, dL/dv, dL/dlog_alpha, dL/dbeta and dL/dS0.  The forward pass is
  * recomputed inside (nothing has to be kept from kda_chunk_fwd): a first sweep stores the state at
- * every chunk boundary, a reverse sweep recomputes one chunk at a time and runs the adjoint through
+ * the start of every block of 8 tokens, a reverse sweep recomputes one block at a time (in shared
+ * memory) and runs the adjoint through
  * it token by token; fp32 arithmetic throughout.
  *
  *   q, k [T_total,H,dk], v, d_o [T_total,H,dv]   device, element type `dt` (KDA_F32 or KDA_BF16)
@@ -206,8 +207,8 @@ kda_status_t kda_layer_fwd(const void *q_c, const void *k_c, const void *v, cons
  *   dS0 [n_seqs,H,dk,dv] fp32 device, written, or NULL
  *   cu_seqlens_dev / cu_seqlens_host, n_seqs, total_tokens, H, scale: as in kda_chunk_fwd
  *   workspace: device memory, 256-byte aligned, at least kda_chunk_bwd_workspace_bytes(...) (chunk
- *              boundary states, one chunk of recomputed states per (sequence, head), and the
- *              per-slice shares of the gradients that are summed over dv; about 0.26 MB per token
+ *              states at the start of every block of 8 tokens and the
+ *              per-slice shares of the gradients that are summed over dv; about 0.45 MB per token
  *              at H = 32).  Its first 256 bytes hold the status word that kda_check_status reads.
  * Only dk = dv = 128 and chunk = 64.  Asynchronous on `cuda_stream`; nothing is allocated; results
  * are deterministic (fixed summation order).  Errors: KDA_ERR_INVALID_ARG, KDA_ERR_UNSUPPORTED,

@@ -13,8 +13,9 @@
 // per (sequence, head, slice), thread = (column, block of 32 rows), both matrices in registers.  The
 // sums over columns (dq, dk, dlog_alpha, dbeta) are formed per slice and added by a second kernel,
 // in a fixed order.  Forward states are not stored for the whole sequence: a first sweep keeps the
-// state at every chunk boundary (64 tokens), the reverse sweep recomputes one chunk at a time into
-// a scratch area that stays in L2.  All arithmetic is fp32 FMA; q, k, v, d_o may be stored as bf16.
+// state at the start of every block of 8 tokens, the reverse sweep recomputes one block at a time into
+// shared memory (8 decayed states of this slice, 128 KB) and runs the adjoint through it.  All
+// arithmetic is fp32 FMA; q, k, v, d_o may be stored as bf16.
 #include <vector>
 
 #include "kda_common.cuh"
@@ -25,6 +26,8 @@ namespace {
 constexpr int NS = 32;                 // state columns per CTA
 constexpr int kSlices = kD / NS;
 constexpr int kThreads = 128;
+constexpr int kB = 8;                  // tokens per recomputation block
+constexpr int kBlocksPerChunk = kC / kB;
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -35,8 +38,7 @@ struct BwdArgs {
     const float* S0; const float* dS_T;
     float* dv; float* dS0;
     const int32_t* cu_seqlens; const int32_t* chunk_cu;
-    float* ckpt;        // [total_chunks][H][128][128]: state at the start of every chunk
-    float* scratch;     // [n_seqs*H*kSlices][64][128][NS]: decayed states S' of the chunk in flight
+    float* ckpt;        // [total_chunks * 8][H][128][128]: state at the start of every block of 8 tokens
     float* part_q; float* part_k; float* part_g;   // [kSlices][T][H][128]
     float* part_b;      // [kSlices][T][H]
     int n_seqs, H;
@@ -45,17 +47,19 @@ struct BwdArgs {
 };
 
 // shared memory of the sweep kernel (floats)
-constexpr int M_K = 0;                       // [64][128] k
-constexpr int M_Q = M_K + kC * kD;           // [64][128] q
-constexpr int M_A = M_Q + kC * kD;           // [64][128] alpha = exp(log alpha)
-constexpr int M_V = M_A + kC * kD;           // [64][NS] v slice
-constexpr int M_DO = M_V + kC * NS;          // [64][NS] d_o slice
-constexpr int M_R = M_DO + kC * NS;          // [64][NS] residuals r_t
-constexpr int M_B = M_R + kC * NS;           // [64] beta
-constexpr int M_RED = M_B + kC;              // [2][4][NS] cross-warp column sums
-constexpr int M_DB = M_RED + 2 * 4 * NS;     // [64][4] dbeta per warp
-constexpr int M_FLOATS = M_DB + kC * 4;
+constexpr int M_SD = 0;                      // [8][128][NS] decayed states S' of the block in flight
+constexpr int M_K = M_SD + kB * kD * NS;     // [8][128] k
+constexpr int M_Q = M_K + kB * kD;           // [8][128] q
+constexpr int M_A = M_Q + kB * kD;           // [8][128] alpha = exp(log alpha)
+constexpr int M_V = M_A + kB * kD;           // [8][NS] v slice
+constexpr int M_DO = M_V + kB * NS;          // [8][NS] d_o slice
+constexpr int M_R = M_DO + kB * NS;          // [8][NS] residuals r_t
+constexpr int M_B = M_R + kB * NS;           // [8] beta
+constexpr int M_RED = M_B + kB;              // [2][4][NS] cross-warp column sums
+constexpr int M_DB = M_RED + 2 * 4 * NS;     // [8][4] dbeta per warp
+constexpr int M_FLOATS = M_DB + kB * 4;
 constexpr size_t kSweepSmem = (size_t)M_FLOATS * sizeof(float);
+static_assert(kSweepSmem <= 232448, "fits the shared memory of one SM");
 
 // sum over the 32 lanes of 32 per-lane values each: afterwards lane l holds the total of x[l]
 __device__ __forceinline__ float lane_transpose_sum(float (&x)[32], int lane) {
@@ -93,23 +97,23 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
         tok_begin = (int64_t)n * a.seq_len; tok_end = tok_begin + a.seq_len;
         chunk0 = (int64_t)n * a.chunks_per_seq;
     }
-    const int nch = (int)((tok_end - tok_begin + kC - 1) / kC);
+    const int nblk = (int)((tok_end - tok_begin + kB - 1) / kB);
     const T* qp = reinterpret_cast<const T*>(a.q);
     const T* kp = reinterpret_cast<const T*>(a.k);
     const T* vp = reinterpret_cast<const T*>(a.v);
     const T* gp = reinterpret_cast<const T*>(a.d_o);
     const size_t sbase = ((size_t)n * a.H + h) * (size_t)(kD * kD);
-    float* scratch = a.scratch + ((size_t)((size_t)n * a.H + h) * kSlices + slice) * (size_t)(kC * kD * NS);
+    float* sSd = sm + M_SD;
 
     float S[32], Lam[32];
 #pragma unroll
     for (int r = 0; r < 32; ++r) S[r] = a.S0 ? a.S0[sbase + (size_t)(i0 + r) * kD + col] : 0.f;
 
-    // loads the vectors of chunk c into shared memory; returns its number of tokens
-    auto load_chunk = [&](int c, bool with_q) {
-        const int64_t tok0 = tok_begin + (int64_t)c * kC;
-        const int len = (tok_end - tok0) < kC ? (int)(tok_end - tok0) : kC;
-        __syncthreads();   // the previous chunk's readers are done
+    // loads the vectors of block b into shared memory; returns its number of tokens
+    auto load_block = [&](int b, bool with_q) {
+        const int64_t tok0 = tok_begin + (int64_t)b * kB;
+        const int len = (tok_end - tok0) < kB ? (int)(tok_end - tok0) : kB;
+        __syncthreads();   // the previous block's readers are done
         for (int idx = t; idx < len * kD; idx += kThreads) {
             const int j = idx >> 7, d = idx & 127;
             const size_t off = ((size_t)(tok0 + j) * a.H + h) * kD + d;
@@ -127,22 +131,23 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
         __syncthreads();
         return len;
     };
-    // one forward token on the register state; optionally keeps S' (global scratch) and r (shared)
+    // one forward token on the register state; optionally keeps S' and r in shared memory
     auto forward_token = [&](int j, bool keep) {
         const float* kj = sm + M_K + j * kD + i0;
         const float* aj = sm + M_A + j * kD + i0;
-        float part = 0.f;
+        float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
 #pragma unroll
-        for (int r = 0; r < 32; ++r) {
-            S[r] *= aj[r];
-            part = fmaf(kj[r], S[r], part);
+        for (int r = 0; r < 32; r += 4) {
+            S[r] *= aj[r]; S[r + 1] *= aj[r + 1]; S[r + 2] *= aj[r + 2]; S[r + 3] *= aj[r + 3];
+            p0 = fmaf(kj[r], S[r], p0); p1 = fmaf(kj[r + 1], S[r + 1], p1);
+            p2 = fmaf(kj[r + 2], S[r + 2], p2); p3 = fmaf(kj[r + 3], S[r + 3], p3);
         }
         if (keep) {
 #pragma unroll
-            for (int r = 0; r < 32; ++r) scratch[((size_t)j * kD + i0 + r) * NS + lane] = S[r];
+            for (int r = 0; r < 32; ++r) sSd[((size_t)j * kD + i0 + r) * NS + lane] = S[r];
         }
         float* red = sm + M_RED + (j & 1) * 4 * NS;
-        red[rg * NS + lane] = part;
+        red[rg * NS + lane] = (p0 + p1) + (p2 + p3);
         __syncthreads();
         const float res = sm[M_V + j * NS + lane] - (red[lane] + red[NS + lane] + red[2 * NS + lane] + red[3 * NS + lane]);
         if (keep && rg == 0) sm[M_R + j * NS + lane] = res;
@@ -150,27 +155,30 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
 #pragma unroll
         for (int r = 0; r < 32; ++r) S[r] = fmaf(kj[r], br, S[r]);
     };
+    auto ckpt_of = [&](int b) {   // (a chunk of 64 tokens owns eight block slots)
+        return a.ckpt + ((size_t)(chunk0 * kBlocksPerChunk + b) * a.H + h) * (size_t)(kD * kD);
+    };
 
-    // ---- sweep 1: forward, keeping the state at every chunk start ------------------------------------
-    for (int c = 0; c < nch; ++c) {
-        float* ck = a.ckpt + ((size_t)(chunk0 + c) * a.H + h) * (size_t)(kD * kD);
+    // ---- sweep 1: forward, keeping the state at every block start -----------------------------------
+    for (int b = 0; b < nblk; ++b) {
+        float* ck = ckpt_of(b);
 #pragma unroll
         for (int r = 0; r < 32; ++r) ck[(size_t)(i0 + r) * kD + col] = S[r];
-        const int len = load_chunk(c, false);
+        const int len = load_block(b, false);
         for (int j = 0; j < len; ++j) forward_token(j, false);
     }
 
-    // ---- sweep 2: chunks in reverse; recompute the chunk, then run the adjoint through it -----------
+    // ---- sweep 2: blocks in reverse; recompute the block, then run the adjoint through it ------------
 #pragma unroll
     for (int r = 0; r < 32; ++r) Lam[r] = a.dS_T ? a.dS_T[sbase + (size_t)(i0 + r) * kD + col] : 0.f;
-    for (int c = nch - 1; c >= 0; --c) {
-        const int64_t tok0 = tok_begin + (int64_t)c * kC;
-        const float* ck = a.ckpt + ((size_t)(chunk0 + c) * a.H + h) * (size_t)(kD * kD);
+    for (int b = nblk - 1; b >= 0; --b) {
+        const int64_t tok0 = tok_begin + (int64_t)b * kB;
+        const float* ck = ckpt_of(b);
 #pragma unroll
         for (int r = 0; r < 32; ++r) S[r] = ck[(size_t)(i0 + r) * kD + col];
-        const int len = load_chunk(c, true);
+        const int len = load_block(b, true);
         for (int j = 0; j < len; ++j) forward_token(j, true);
-        __syncthreads();   // r_t of every token is in shared memory (this thread's own S' stores are its own)
+        __syncthreads();   // r_t of every token is in shared memory (a thread reads back its own S' only)
         for (int j = len - 1; j >= 0; --j) {
             const float* kj = sm + M_K + j * kD + i0;
             const float* qj = sm + M_Q + j * kD + i0;
@@ -179,7 +187,7 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
             const float bt = sm[M_B + j];
             float Sd[32], x[32];
 #pragma unroll
-            for (int r = 0; r < 32; ++r) Sd[r] = scratch[((size_t)j * kD + i0 + r) * NS + lane];
+            for (int r = 0; r < 32; ++r) Sd[r] = sSd[((size_t)j * kD + i0 + r) * NS + lane];
             // o_t = scale S_t^T q_t
             const float sgo = a.scale * go, br = bt * res;
 #pragma unroll
@@ -189,15 +197,16 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
             }
             const float dq_i = lane_transpose_sum(x, lane);
             // S_t = S' + beta k r^T
-            float part = 0.f;
+            float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
 #pragma unroll
-            for (int r = 0; r < 32; ++r) {
-                x[r] = Lam[r] * res;
-                part = fmaf(Lam[r], kj[r], part);
+            for (int r = 0; r < 32; r += 4) {
+                x[r] = Lam[r] * res; x[r + 1] = Lam[r + 1] * res; x[r + 2] = Lam[r + 2] * res; x[r + 3] = Lam[r + 3] * res;
+                p0 = fmaf(Lam[r], kj[r], p0); p1 = fmaf(Lam[r + 1], kj[r + 1], p1);
+                p2 = fmaf(Lam[r + 2], kj[r + 2], p2); p3 = fmaf(Lam[r + 3], kj[r + 3], p3);
             }
             const float lr_i = lane_transpose_sum(x, lane);    // (Lam r)_i
             float* red = sm + M_RED + (j & 1) * 4 * NS;
-            red[rg * NS + lane] = part;
+            red[rg * NS + lane] = (p0 + p1) + (p2 + p3);
             __syncthreads();
             const float dr = bt * (red[lane] + red[NS + lane] + red[2 * NS + lane] + red[3 * NS + lane]);
             if (rg == 0) a.dv[((size_t)(tok0 + j) * a.H + h) * kD + col] = dr;
@@ -267,7 +276,7 @@ __global__ void kda_bwd_reduce(const float* __restrict__ part_q, const float* __
 }
 
 struct BwdLayout {
-    size_t off_table, off_ckpt, off_scratch, off_pq, off_pk, off_pg, off_pb, total;
+    size_t off_table, off_ckpt, off_pq, off_pk, off_pg, off_pb, total;
 };
 BwdLayout bwd_layout(int64_t T, int n_seqs, int H)
 {
@@ -276,8 +285,7 @@ BwdLayout bwd_layout(int64_t T, int n_seqs, int H)
     const size_t vec = (size_t)T * H * kD * sizeof(float);
     L.off_table = sizeof(WsHeader);
     L.off_ckpt = L.off_table + align_up((size_t)(n_seqs + 1) * sizeof(int32_t));
-    L.off_scratch = L.off_ckpt + align_up(chunks * H * kD * kD * sizeof(float));
-    L.off_pq = L.off_scratch + align_up((size_t)n_seqs * H * kSlices * kC * kD * NS * sizeof(float));
+    L.off_pq = L.off_ckpt + align_up(chunks * kBlocksPerChunk * H * kD * kD * sizeof(float));
     L.off_pk = L.off_pq + align_up(kSlices * vec);
     L.off_pg = L.off_pk + align_up(kSlices * vec);
     L.off_pb = L.off_pg + align_up(kSlices * vec);
@@ -370,7 +378,6 @@ kda_status_t kda_chunk_bwd(const void* q, const void* k, const void* v, const fl
     a.S0 = S0; a.dS_T = dS_T; a.dv = dv_out; a.dS0 = dS0;
     a.cu_seqlens = cu_seqlens_dev; a.chunk_cu = cu_seqlens_dev ? chunk_cu_dev : nullptr;
     a.ckpt = reinterpret_cast<float*>(ws + L.off_ckpt);
-    a.scratch = reinterpret_cast<float*>(ws + L.off_scratch);
     a.part_q = reinterpret_cast<float*>(ws + L.off_pq);
     a.part_k = reinterpret_cast<float*>(ws + L.off_pk);
     a.part_g = reinterpret_cast<float*>(ws + L.off_pg);
