@@ -9,8 +9,8 @@
 //     dr = beta_t Lam^T k_t = dv_t      Lam' = Lam - k_t dr^T
 //     dlog_alpha_t = rowsum(Lam' . S')  Lam <- Diag(alpha_t) Lam'
 //
-// Columns of S and of Lam never mix, so dv is cut into four 32-column slices: one CTA of four warps
-// per (sequence, head, slice), thread = (column, block of 32 rows), both matrices in registers.  The
+// Columns of S and of Lam never mix, so dv is cut into four 32-column slices: one CTA of eight warps
+// per (sequence, head, slice), thread = (column, block of 16 rows), both matrices in registers.  The
 // sums over columns (dq, dk, dlog_alpha, dbeta) are formed per slice and added by a second kernel,
 // in a fixed order.  Forward states are not stored for the whole sequence: a first sweep keeps the
 // state at the start of every block of 8 tokens, the reverse sweep recomputes one block at a time into
@@ -25,7 +25,9 @@ namespace {
 
 constexpr int NS = 32;                 // state columns per CTA
 constexpr int kSlices = kD / NS;
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kRows = kD / kWarps;      // state rows per thread (the warp's block of rows)
 constexpr int kB = 8;                  // tokens per recomputation block
 constexpr int kBlocksPerChunk = kC / kB;
 constexpr size_t kAlign = 256;
@@ -55,16 +57,16 @@ constexpr int M_V = M_A + kB * kD;           // [8][NS] v slice
 constexpr int M_DO = M_V + kB * NS;          // [8][NS] d_o slice
 constexpr int M_R = M_DO + kB * NS;          // [8][NS] residuals r_t
 constexpr int M_B = M_R + kB * NS;           // [8] beta
-constexpr int M_RED = M_B + kB;              // [2][4][NS] cross-warp column sums
-constexpr int M_DB = M_RED + 2 * 4 * NS;     // [8][4] dbeta per warp
-constexpr int M_FLOATS = M_DB + kB * 4;
+constexpr int M_RED = M_B + kB;              // [2][warps][NS] cross-warp column sums
+constexpr int M_DB = M_RED + 2 * kWarps * NS;   // [8][warps] dbeta per warp
+constexpr int M_FLOATS = M_DB + kB * kWarps;
 constexpr size_t kSweepSmem = (size_t)M_FLOATS * sizeof(float);
 static_assert(kSweepSmem <= 232448, "fits the shared memory of one SM");
 
-// sum over the 32 lanes of 32 per-lane values each: afterwards lane l holds the total of x[l]
-__device__ __forceinline__ float lane_transpose_sum(float (&x)[32], int lane) {
+// sum over the 32 lanes of kRows per-lane values each: afterwards lane l holds the total of x[l % kRows]
+__device__ __forceinline__ float lane_transpose_sum(float (&x)[kRows], int lane) {
 #pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) {
+    for (int s = kRows / 2; s >= 1; s >>= 1) {
         const bool up = (lane & s) != 0;
 #pragma unroll
         for (int j = 0; j < s; ++j) {
@@ -73,7 +75,22 @@ __device__ __forceinline__ float lane_transpose_sum(float (&x)[32], int lane) {
             x[j] = keep + __shfl_xor_sync(0xffffffffu, send, s);
         }
     }
-    return x[0];
+    float v = x[0];
+#pragma unroll
+    for (int s = kRows; s < 32; s <<= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+    return v;
+}
+__device__ __forceinline__ float sum_db(const float* p) {
+    float v = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) v += p[w];
+    return v;
+}
+__device__ __forceinline__ float sum_partials(const float* red, int lane) {
+    float v = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) v += red[w * NS + lane];
+    return v;
 }
 
 template <typename T> __device__ __forceinline__ float ldf(const T* p);
@@ -87,7 +104,7 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
     const int t = threadIdx.x, lane = t & 31, rg = t >> 5;
     const int slice = blockIdx.x, h = blockIdx.y, n = blockIdx.z;
     const int col = slice * NS + lane;
-    const int i0 = rg * 32;                    // first of this thread's 32 rows
+    const int i0 = rg * kRows;                 // first of this thread's rows
 
     int64_t tok_begin, tok_end, chunk0;
     if (a.cu_seqlens) {
@@ -105,9 +122,9 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
     const size_t sbase = ((size_t)n * a.H + h) * (size_t)(kD * kD);
     float* sSd = sm + M_SD;
 
-    float S[32], Lam[32];
+    float S[kRows], Lam[kRows];
 #pragma unroll
-    for (int r = 0; r < 32; ++r) S[r] = a.S0 ? a.S0[sbase + (size_t)(i0 + r) * kD + col] : 0.f;
+    for (int r = 0; r < kRows; ++r) S[r] = a.S0 ? a.S0[sbase + (size_t)(i0 + r) * kD + col] : 0.f;
 
     // loads the vectors of block b into shared memory; returns its number of tokens
     auto load_block = [&](int b, bool with_q) {
@@ -137,23 +154,23 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
         const float* aj = sm + M_A + j * kD + i0;
         float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
 #pragma unroll
-        for (int r = 0; r < 32; r += 4) {
+        for (int r = 0; r < kRows; r += 4) {
             S[r] *= aj[r]; S[r + 1] *= aj[r + 1]; S[r + 2] *= aj[r + 2]; S[r + 3] *= aj[r + 3];
             p0 = fmaf(kj[r], S[r], p0); p1 = fmaf(kj[r + 1], S[r + 1], p1);
             p2 = fmaf(kj[r + 2], S[r + 2], p2); p3 = fmaf(kj[r + 3], S[r + 3], p3);
         }
         if (keep) {
 #pragma unroll
-            for (int r = 0; r < 32; ++r) sSd[((size_t)j * kD + i0 + r) * NS + lane] = S[r];
+            for (int r = 0; r < kRows; ++r) sSd[((size_t)j * kD + i0 + r) * NS + lane] = S[r];
         }
-        float* red = sm + M_RED + (j & 1) * 4 * NS;
+        float* red = sm + M_RED + (j & 1) * kWarps * NS;
         red[rg * NS + lane] = (p0 + p1) + (p2 + p3);
         __syncthreads();
-        const float res = sm[M_V + j * NS + lane] - (red[lane] + red[NS + lane] + red[2 * NS + lane] + red[3 * NS + lane]);
+        const float res = sm[M_V + j * NS + lane] - sum_partials(red, lane);
         if (keep && rg == 0) sm[M_R + j * NS + lane] = res;
         const float br = sm[M_B + j] * res;
 #pragma unroll
-        for (int r = 0; r < 32; ++r) S[r] = fmaf(kj[r], br, S[r]);
+        for (int r = 0; r < kRows; ++r) S[r] = fmaf(kj[r], br, S[r]);
     };
     auto ckpt_of = [&](int b) {   // (a chunk of 64 tokens owns eight block slots)
         return a.ckpt + ((size_t)(chunk0 * kBlocksPerChunk + b) * a.H + h) * (size_t)(kD * kD);
@@ -163,19 +180,19 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
     for (int b = 0; b < nblk; ++b) {
         float* ck = ckpt_of(b);
 #pragma unroll
-        for (int r = 0; r < 32; ++r) ck[(size_t)(i0 + r) * kD + col] = S[r];
+        for (int r = 0; r < kRows; ++r) ck[(size_t)(i0 + r) * kD + col] = S[r];
         const int len = load_block(b, false);
         for (int j = 0; j < len; ++j) forward_token(j, false);
     }
 
     // ---- sweep 2: blocks in reverse; recompute the block, then run the adjoint through it ------------
 #pragma unroll
-    for (int r = 0; r < 32; ++r) Lam[r] = a.dS_T ? a.dS_T[sbase + (size_t)(i0 + r) * kD + col] : 0.f;
+    for (int r = 0; r < kRows; ++r) Lam[r] = a.dS_T ? a.dS_T[sbase + (size_t)(i0 + r) * kD + col] : 0.f;
     for (int b = nblk - 1; b >= 0; --b) {
         const int64_t tok0 = tok_begin + (int64_t)b * kB;
         const float* ck = ckpt_of(b);
 #pragma unroll
-        for (int r = 0; r < 32; ++r) S[r] = ck[(size_t)(i0 + r) * kD + col];
+        for (int r = 0; r < kRows; ++r) S[r] = ck[(size_t)(i0 + r) * kD + col];
         const int len = load_block(b, true);
         for (int j = 0; j < len; ++j) forward_token(j, true);
         __syncthreads();   // r_t of every token is in shared memory (a thread reads back its own S' only)
@@ -185,13 +202,13 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
             const float* aj = sm + M_A + j * kD + i0;
             const float res = sm[M_R + j * NS + lane], go = sm[M_DO + j * NS + lane];
             const float bt = sm[M_B + j];
-            float Sd[32], x[32];
+            float Sd[kRows], x[kRows];
 #pragma unroll
-            for (int r = 0; r < 32; ++r) Sd[r] = sSd[((size_t)j * kD + i0 + r) * NS + lane];
+            for (int r = 0; r < kRows; ++r) Sd[r] = sSd[((size_t)j * kD + i0 + r) * NS + lane];
             // o_t = scale S_t^T q_t
             const float sgo = a.scale * go, br = bt * res;
 #pragma unroll
-            for (int r = 0; r < 32; ++r) {
+            for (int r = 0; r < kRows; ++r) {
                 Lam[r] = fmaf(qj[r], sgo, Lam[r]);
                 x[r] = fmaf(kj[r], br, Sd[r]) * sgo;          // S_t[i][c] * scale * d_o[c]
             }
@@ -199,49 +216,52 @@ __global__ void __launch_bounds__(kThreads, 1) kda_bwd_sweep(BwdArgs a)
             // S_t = S' + beta k r^T
             float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
 #pragma unroll
-            for (int r = 0; r < 32; r += 4) {
+            for (int r = 0; r < kRows; r += 4) {
                 x[r] = Lam[r] * res; x[r + 1] = Lam[r + 1] * res; x[r + 2] = Lam[r + 2] * res; x[r + 3] = Lam[r + 3] * res;
                 p0 = fmaf(Lam[r], kj[r], p0); p1 = fmaf(Lam[r + 1], kj[r + 1], p1);
                 p2 = fmaf(Lam[r + 2], kj[r + 2], p2); p3 = fmaf(Lam[r + 3], kj[r + 3], p3);
             }
             const float lr_i = lane_transpose_sum(x, lane);    // (Lam r)_i
-            float* red = sm + M_RED + (j & 1) * 4 * NS;
+            float* red = sm + M_RED + (j & 1) * kWarps * NS;
             red[rg * NS + lane] = (p0 + p1) + (p2 + p3);
             __syncthreads();
-            const float dr = bt * (red[lane] + red[NS + lane] + red[2 * NS + lane] + red[3 * NS + lane]);
+            const float dr = bt * sum_partials(red, lane);
             if (rg == 0) a.dv[((size_t)(tok0 + j) * a.H + h) * kD + col] = dr;
             // r = v - S'^T k ;  S' = Diag(alpha) S_{t-1}
 #pragma unroll
-            for (int r = 0; r < 32; ++r) {
+            for (int r = 0; r < kRows; ++r) {
                 Lam[r] = fmaf(-kj[r], dr, Lam[r]);             // Lam'
                 x[r] = Sd[r] * dr;
             }
             const float sdr_i = lane_transpose_sum(x, lane);   // (S' dr)_i
 #pragma unroll
-            for (int r = 0; r < 32; ++r) {
+            for (int r = 0; r < kRows; ++r) {
                 x[r] = Lam[r] * Sd[r];
                 Lam[r] *= aj[r];
             }
             const float dg_i = lane_transpose_sum(x, lane);
-            // lane l now holds the slice's share of row i0 + l
-            const float k_i = sm[M_K + j * kD + i0 + lane];
-            const size_t po = (((size_t)slice * a.total_tokens + (size_t)(tok0 + j)) * a.H + h) * kD + i0 + lane;
-            a.part_q[po] = dq_i;
-            a.part_k[po] = bt * lr_i - sdr_i;
-            a.part_g[po] = dg_i;
-            float db = k_i * lr_i;
+            // lanes l and l + 16 now hold the slice's share of row i0 + l
+            const int rl = lane & (kRows - 1);
+            const float k_i = sm[M_K + j * kD + i0 + rl];
+            if (lane < kRows) {
+                const size_t po = (((size_t)slice * a.total_tokens + (size_t)(tok0 + j)) * a.H + h) * kD + i0 + lane;
+                a.part_q[po] = dq_i;
+                a.part_k[po] = bt * lr_i - sdr_i;
+                a.part_g[po] = dg_i;
+            }
+            float db = lane < kRows ? k_i * lr_i : 0.f;
 #pragma unroll
             for (int s = 16; s >= 1; s >>= 1) db += __shfl_xor_sync(0xffffffffu, db, s);
-            if (lane == 0) sm[M_DB + j * 4 + rg] = db;
+            if (lane == 0) sm[M_DB + j * kWarps + rg] = db;
         }
         __syncthreads();
         if (t < len)
             a.part_b[((size_t)slice * a.total_tokens + (size_t)(tok0 + t)) * a.H + h] =
-                sm[M_DB + t * 4] + sm[M_DB + t * 4 + 1] + sm[M_DB + t * 4 + 2] + sm[M_DB + t * 4 + 3];
+                sum_db(sm + M_DB + t * kWarps);
     }
     if (a.dS0) {
 #pragma unroll
-        for (int r = 0; r < 32; ++r) a.dS0[sbase + (size_t)(i0 + r) * kD + col] = Lam[r];
+        for (int r = 0; r < kRows; ++r) a.dS0[sbase + (size_t)(i0 + r) * kD + col] = Lam[r];
     }
 }
 
