@@ -164,3 +164,45 @@ def test_fused_schedule_plan(lib):
     # no schedule: fewer than two tiles of room, or a device with fewer than four SMs
     assert _plan(lib, [4], 2, 1, 148)[0] == 0
     assert _plan(lib, [4], 2, 64, 3)[0] == 0
+
+
+def test_side_entry_points_reject_bad_arguments(lib):
+    """Layer wrap, backward pass and DPLR comparison: argument errors found before any CUDA call."""
+    import paper_2510_26692_b200 as K
+    one = ctypes.c_void_p(256)
+    f32, sz, i64, i32 = ctypes.c_float, ctypes.c_size_t, ctypes.c_int64, ctypes.c_int
+    # kda_dplr_chunk_fwd: head size, misaligned pointer, cu_seqlens on one side only
+    rc = lib.kda_dplr_chunk_fwd(one, one, one, one, one, one, None, one, one, None, None, 1, 64, 2, 64, 128, 64,
+                                1.0, one, 1 << 30, None)
+    assert rc == 2
+    rc = lib.kda_dplr_chunk_fwd(one, one, one, ctypes.c_void_p(260), one, one, None, one, one, None, None, 1, 64, 2,
+                                128, 128, 64, 1.0, one, 1 << 30, None)
+    assert rc == 1 and "aligned" in K.kda_last_error()
+    rc = lib.kda_dplr_chunk_fwd(one, one, one, one, one, one, None, one, one, one, None, 1, 64, 2, 128, 128, 64, 1.0,
+                                one, 1 << 30, None)
+    assert rc == 1
+    assert lib.kda_dplr_chunk_fwd_workspace_bytes(4096, 1, 2, 128, 128, 64) >= \
+        lib.kda_dplr_chunk_fwd_min_workspace_bytes(4096, 1, 2, 128, 128, 64) > 0
+    assert lib.kda_dplr_chunk_fwd_workspace_bytes(4096, 1, 2, 64, 128, 64) == 0
+    # kda_chunk_bwd: chunk length, missing gradient output, workspace too small
+    args = [one] * 6 + [one, one] + [one] * 5 + [one, None, None]
+    rc = lib.kda_chunk_bwd(*args, 1, 64, 2, 128, 128, 32, 1.0, K.KDA_BF16, one, 1 << 30, None)
+    assert rc == 2
+    bad = list(args)
+    bad[9] = None      # dk
+    rc = lib.kda_chunk_bwd(*bad, 1, 64, 2, 128, 128, 64, 1.0, K.KDA_BF16, one, 1 << 30, None)
+    assert rc == 1 and "NULL" in K.kda_last_error()
+    rc = lib.kda_chunk_bwd(*args, 1, 64, 2, 128, 128, 64, 1.0, K.KDA_BF16, one, 4096, None)
+    assert rc == 3
+    assert lib.kda_chunk_bwd_workspace_bytes(4096, 1, 32, 128, 128, 64) > 4096 * 32 * 128 * 4 * 12
+    # kda_layer_fwd: decay-function parameters are required; y needs its gate and weight
+    largs = [one] * 6 + [None, one, one]
+    rc = lib.kda_layer_fwd(*largs, 1e-6, 1e-5, None, one, one, None, None, 1, 64, 2, 128, 128, 64, 1.0, one,
+                           1 << 30, None)
+    assert rc == 1 and "A_log" in K.kda_last_error()
+    largs = [one] * 5 + [None, one, one, one]
+    rc = lib.kda_layer_fwd(*largs, 1e-6, 1e-5, None, one, one, None, None, 1, 64, 2, 128, 128, 64, 1.0, one,
+                           1 << 30, None)
+    assert rc == 1 and "g_o" in K.kda_last_error()
+    assert lib.kda_layer_fwd_workspace_bytes(4096, 1, 32, 128, 128, 64) >= \
+        lib.kda_layer_fwd_min_workspace_bytes(4096, 1, 32, 128, 128, 64) > 0

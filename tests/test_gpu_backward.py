@@ -65,7 +65,9 @@ def oracle_bwd(oracle_mod, d, d_o, dS_T, scale=1.0):
 @pytest.mark.parametrize("lens,H,dtype,s0", [([100], 2, torch.float32, 0.0),
                                              ([300], 3, torch.bfloat16, 0.05),
                                              ([64, 1, 200, 0, 130], 2, torch.bfloat16, 0.05),
-                                             ([1024], 4, torch.float32, 0.02)])
+                                             ([1024], 4, torch.float32, 0.02),
+                                             ([3, 0, 9, 64, 65, 1], 1, torch.float32, 0.05),
+                                             ([7, 8], 3, torch.bfloat16, 0.0)])
 def test_backward_matches_oracle(oracle_mod, lens, H, dtype, s0):
     d = inputs.chunk_inputs(lens, H=H, dtype=dtype, seed=31, s0_std=s0)
     d_o, dS_T = cotangents(d, 31, dtype)

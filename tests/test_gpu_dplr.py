@@ -45,7 +45,7 @@ def oracle_dplr(oracle_mod, d, scale=1.0):
 
 
 @pytest.mark.parametrize("lens,H,s0", [([256], 2, 0.0), ([1000], 3, 0.05), ([64, 1, 200, 0, 130], 4, 0.05),
-                                       ([2048], 16, 0.02)])
+                                       ([2048], 16, 0.02), ([1], 1, 0.05), ([63, 65, 0], 1, 0.0)])
 def test_dplr_matches_oracle(oracle_mod, lens, H, s0):
     d = inputs.dplr_inputs(lens, H=H, seed=21, s0_std=s0)
     o, S_T = run_dplr(d, scale=0.9)

@@ -50,7 +50,7 @@ def oracle_layer(oracle_mod, d, scale, l2_eps=1e-6, rms_eps=1e-5):
 
 
 @pytest.mark.parametrize("lens,H,s0", [([256], 2, 0.0), ([1000], 3, 0.02), ([64, 1, 200, 0, 130], 4, 0.02),
-                                       ([4096], 8, 0.02)])
+                                       ([4096], 8, 0.02), ([1, 63, 65], 1, 0.02), ([5], 3, 0.0)])
 def test_layer_matches_oracle(oracle_mod, lens, H, s0):
     d = inputs.layer_inputs(lens, H=H, seed=41, s0_std=s0)
     scale = 128 ** -0.5
