@@ -37,6 +37,7 @@ namespace {
 
 constexpr uint64_t kWaitLimitNs = 1000000000ull;   // 1 s per wait
 constexpr int kNCtrl = 2;                          // MMA-issuing threads (one per control warp)
+bool g_inter_wide = true;                          // (debug switch) use the 128-column form for large batches
 
 template <int NS> struct InterCfg {
     static_assert(NS == 32 || NS == 64, "state columns per CTA: one or two 32-column blocks");
@@ -453,6 +454,319 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
     if (warp == 0) ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
 }
 
+// ---- all 128 state columns in one CTA (throughput form, for calls with more chains than SMs) ------------
+// Sixteen compute warps (TMEM lane quadrant = warp & 3, 32-column group = warp >> 2) share one set of
+// operand images and one MMA per product with N = 128: per SM and step this moves four times the
+// columns of the 32-column form.  Two control threads issue the products (one the first product, the
+// other the state product and the output product); a loader thread requests every piece of a tile as
+// early as its buffer frees up: the [W' ; Q'] image (free once the first product has completed), the
+// K' / Aqk / U part (free once the last product of its chunk has completed and U has been read) and the
+// three gate vectors, each with its own ring and its own empty / full barriers.
+struct WideCfg {
+    static constexpr uint32_t kA = 0;                        // [2] x [W' ; Q'] images, 32 KB each
+    static constexpr uint32_t kABytes = 32768;
+    static constexpr uint32_t kB = 2 * kABytes;              // [2] x (K' 16 KB | Aqk 8 KB | U 16 KB)
+    static constexpr uint32_t kBBytes = 40960;
+    static constexpr uint32_t kBU = 24576;                   // U inside a B part
+    static constexpr uint32_t kG = kB + 2 * kBBytes;         // [3] x (gamma^C | exp(G_m) | exp(G_C - G_m))
+    static constexpr uint32_t kSbf = (kG + 3 * tc::GV_BYTES + 1023) / 1024 * 1024;   // B operand of MMA1: [2 column halves][128 dk rows][128 B]
+    static constexpr uint32_t kSbfHalf = 128 * 128;
+    static constexpr uint32_t kVn = kSbf + 2 * kSbfHalf;     // B operand of MMA2: [2 column halves][64 token rows][128 B]
+    static constexpr uint32_t kVnHalf = 64 * 128;
+    static constexpr uint32_t kBars = kVn + 2 * kVnHalf;
+    static constexpr uint32_t kTotal = kBars + 256;
+    static constexpr uint32_t kSmem = kTotal + 1024;
+    static constexpr int kThreads = 16 * 32 + 96;            // + two control warps and the loader warp
+    static_assert(kSmem <= 232448, "fits the shared memory of one SM");
+    static_assert(tc::OFF_AQ == tc::OFF_KI + 16384 && tc::OFF_GV == tc::OFF_AQ + 8192, "K' and Aqk are contiguous in a tile");
+};
+
+__device__ __forceinline__ void store_row32_at(uint8_t* img, int row, int c0, const float (&x)[32]) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        *reinterpret_cast<uint4*>(img + row * 128 + (((c0 + c) ^ (row & 7)) << 4)) =
+            make_uint4(pack2(x[8 * c], x[8 * c + 1]), pack2(x[8 * c + 2], x[8 * c + 3]),
+                       pack2(x[8 * c + 4], x[8 * c + 5]), pack2(x[8 * c + 6], x[8 * c + 7]));
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&acc)[32]) {
+    uint32_t r[32];
+    ptx::tmem_ld_32x32b_x32(taddr, r);
+    ptx::tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(r[j]);
+}
+
+__global__ void __launch_bounds__(WideCfg::kThreads, 1)
+kda_inter_tc_wide(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader* hdr)
+{
+    using Cfg = WideCfg;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* fullA = reinterpret_cast<uint64_t*>(smem + Cfg::kBars);   // [2]
+    uint64_t* fullB = fullA + 2;           // [2]
+    uint64_t* fullG = fullB + 2;           // [3]
+    uint64_t* emptyA = fullG + 3;          // [2] the first product of the chunk has completed
+    uint64_t* emptyB = emptyA + 2;         // [2] the last product of the chunk has completed and U has been read
+    uint64_t* emptyG = emptyB + 2;         // [3] all compute warps have read the vectors
+    uint64_t* mma1_bar = emptyG + 3;
+    uint64_t* mma2_bar = mma1_bar + 1;
+    uint64_t* out_bar = mma2_bar + 1;      // [2]
+    uint64_t* sbf_ready = out_bar + 2;     // 16 warp arrivals
+    uint64_t* vn_ready = sbf_ready + 1;    // 8 warp arrivals
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(vn_ready + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint8_t* sbf = smem + Cfg::kSbf;
+    uint8_t* vn = smem + Cfg::kVn;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int h = blockIdx.y, n = n_begin + blockIdx.z;
+    __nv_bfloat16* op = reinterpret_cast<__nv_bfloat16*>(a.o);
+
+    int64_t cb, ce, tok_begin, tok_end;
+    if (a.cu_seqlens) {
+        cb = a.chunk_cu[n]; ce = a.chunk_cu[n + 1];
+        tok_begin = a.cu_seqlens[n]; tok_end = a.cu_seqlens[n + 1];
+    } else {
+        cb = (int64_t)n * a.chunks_per_seq; ce = cb + a.chunks_per_seq;
+        tok_begin = (int64_t)n * a.seq_len; tok_end = tok_begin + a.seq_len;
+    }
+    const int64_t seq_c0 = cb;
+    if (cb < a.g0) cb = a.g0;
+    if (ce > a.g1) ce = a.g1;
+    const int nchunks = ce > cb ? (int)(ce - cb) : 0;
+
+    if (tid == 0) {
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(&fullA[s], 1);
+            ptx::mbar_init(&fullB[s], 1);
+            ptx::mbar_init(&emptyA[s], 1);                // commit of the first control thread
+            ptx::mbar_init(&emptyB[s], 1 + 8);            // commit of the second + the eight warps that read U
+            ptx::mbar_init(&out_bar[s], 1);
+        }
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+            ptx::mbar_init(&fullG[s], 1);
+            ptx::mbar_init(&emptyG[s], 16);
+        }
+        ptx::mbar_init(mma1_bar, 1);
+        ptx::mbar_init(mma2_bar, 1);
+        ptx::mbar_init(sbf_ready, 16);
+        ptx::mbar_init(vn_ready, 8);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 0) {
+        ptx::tmem_alloc(tmem_slot, 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t d3 = 256;   // TMEM columns: D1 {parity 0, 1} at 0 and 128, D3 at 256
+
+    auto wait = [&](uint64_t* bar, uint32_t parity, int where) {
+        if (*abort_flag) return;
+        if (!ptx::mbar_wait(bar, parity, kWaitLimitNs)) {
+            *abort_flag = 1;
+            if (atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = where;
+        }
+    };
+    const uint32_t idesc = ptx::umma_idesc_bf16(128, 128) | ptx::kIdescBMajorMN;
+    const uint32_t sbf_a = ptx::smem_u32(sbf), vn_a = ptx::smem_u32(vn);
+
+    if (warp == 18) {
+        // ---- loader ----
+        if (lane == 0) {
+            ptx::grid_dep_wait();   // the tiles come from the intra-chunk kernel launched just before
+            int nA = 0, nB = 0, nG = 0;
+            for (int p = 0; p < nchunks && !*abort_flag; ++p) {
+                const char* tile = tiles + ((size_t)(cb + p - a.g0) * a.H + h) * tc::TILE_BYTES;
+                const int s2 = p & 1, s3 = p % 3;
+                if (p >= 3) wait(&emptyG[s3], (uint32_t)(p / 3 - 1) & 1u, 31);
+                if (*abort_flag) break;
+                ptx::mbar_expect_tx(&fullG[s3], tc::GV_BYTES);
+                ptx::bulk_g2s(smem + Cfg::kG + s3 * tc::GV_BYTES, tile + tc::OFF_GV, tc::GV_BYTES, &fullG[s3]);
+                ++nG;
+                if (p >= 2) wait(&emptyA[s2], (uint32_t)(p / 2 - 1) & 1u, 32);
+                if (*abort_flag) break;
+                ptx::mbar_expect_tx(&fullA[s2], Cfg::kABytes);
+                ptx::bulk_g2s(smem + Cfg::kA + s2 * Cfg::kABytes, tile + tc::OFF_QW, Cfg::kABytes, &fullA[s2]);
+                ++nA;
+                if (p >= 2) wait(&emptyB[s2], (uint32_t)(p / 2 - 1) & 1u, 33);
+                if (*abort_flag) break;
+                uint8_t* sbB = smem + Cfg::kB + s2 * Cfg::kBBytes;
+                ptx::mbar_expect_tx(&fullB[s2], Cfg::kBBytes);
+                ptx::bulk_g2s(sbB, tile + tc::OFF_KI, 24576, &fullB[s2]);
+                ptx::bulk_g2s(sbB + Cfg::kBU, tile + tc::OFF_U, 16384, &fullB[s2]);
+                ++nB;
+            }
+            if (*abort_flag) {   // drain the copies still in flight before the shared memory goes away
+                for (int j = (nG > 3 ? nG - 3 : 0); j < nG; ++j) ptx::mbar_wait(&fullG[j % 3], (uint32_t)(j / 3) & 1u, kWaitLimitNs / 8);
+                for (int j = (nA > 2 ? nA - 2 : 0); j < nA; ++j) ptx::mbar_wait(&fullA[j & 1], (uint32_t)(j >> 1) & 1u, kWaitLimitNs / 8);
+                for (int j = (nB > 2 ? nB - 2 : 0); j < nB; ++j) ptx::mbar_wait(&fullB[j & 1], (uint32_t)(j >> 1) & 1u, kWaitLimitNs / 8);
+            }
+        }
+    } else if (warp == 16) {
+        // ---- control thread A: the first product ----
+        if (lane == 0) {
+            for (int it = 0; it < nchunks; ++it) {
+                const int s = it & 1;
+                const uint32_t sa = ptx::smem_u32(smem + Cfg::kA + s * Cfg::kABytes);
+                const uint32_t d1 = tmem_base + (uint32_t)(it & 1) * 128;
+                wait(&fullA[s], (uint32_t)(it >> 1) & 1u, 1);
+                wait(sbf_ready, (uint32_t)it & 1u, 4);
+                ptx::tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    ptx::umma_bf16(d1, ptx::umma_desc_sw128(sa + (kk >> 2) * tc::QW_HALF + (kk & 3) * 32),
+                                   ptx::umma_desc_sw128_mn(sbf_a + kk * 2048, Cfg::kSbfHalf), idesc, kk > 0);
+                ptx::umma_commit(mma1_bar);
+                ptx::umma_commit(&emptyA[s]);
+            }
+            if (nchunks > 0) wait(&emptyA[(nchunks - 1) & 1], (uint32_t)((nchunks - 1) >> 1) & 1u, 7);
+        }
+    } else if (warp == 17) {
+        // ---- control thread B: the state product and the output product ----
+        if (lane == 0) {
+            for (int it = 0; it < nchunks; ++it) {
+                const int s = it & 1;
+                const uint32_t sbB = ptx::smem_u32(smem + Cfg::kB + s * Cfg::kBBytes);
+                const uint32_t d1 = tmem_base + (uint32_t)(it & 1) * 128;
+                wait(&fullB[s], (uint32_t)(it >> 1) & 1u, 2);
+                wait(vn_ready, (uint32_t)it & 1u, 5);
+                ptx::tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    ptx::umma_bf16(tmem_base + d3, ptx::umma_desc_sw128_mn(sbB + kk * 2048, tc::KI_HALF),
+                                   ptx::umma_desc_sw128_mn(vn_a + kk * 2048, Cfg::kVnHalf),
+                                   idesc | ptx::kIdescAMajorMN, kk > 0);
+                ptx::umma_commit(mma2_bar);
+                if (op) {
+                    // D1[64:128] += Aqk V_new (the 128-row A operand starts 64 rows before Aqk, in the
+                    // second half of the K' image; those rows only touch accumulator rows 0-63, dead
+                    // once V_new has been taken)
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        ptx::umma_bf16(d1, ptx::umma_desc_sw128(sbB + 8192 + kk * 32),
+                                       ptx::umma_desc_sw128_mn(vn_a + kk * 2048, Cfg::kVnHalf), idesc, 1);
+                    ptx::umma_commit(&out_bar[it & 1]);
+                }
+                ptx::umma_commit(&emptyB[s]);
+            }
+            // every product of this thread has completed before the TMEM goes away
+            if (nchunks > 0) wait(&emptyB[(nchunks - 1) & 1], (uint32_t)((nchunks - 1) >> 1) & 1u, 8);
+        }
+    } else if (warp < 16) {
+        // ---- compute warps ----
+        const int quad = warp & 3, ch = warp >> 2;
+        const int row = quad * 32 + lane;                  // token row for V_new / O, dk row for the state
+        const int half = ch >> 1, c0 = (ch & 1) * 4;       // column half of the operand images, first 16-byte chunk
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)ch * 32;
+        auto warp_arrive = [&](uint64_t* bar) {
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar);
+        };
+        float S[32];
+        const size_t sbase = ((size_t)n * a.H + h) * (size_t)(kD * kD) + (size_t)row * kD + ch * 32;
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (a.S_in) x = *reinterpret_cast<const float4*>(a.S_in + sbase + j);
+            S[j] = x.x; S[j + 1] = x.y; S[j + 2] = x.z; S[j + 3] = x.w;
+        }
+        auto ref_scale_of = [&](int g) {   // exp(G_m) of chunk g (0 past the last one)
+            if (g >= nchunks) return 0.f;
+            wait(&fullG[g % 3], (uint32_t)(g / 3) & 1u, 9);
+            return reinterpret_cast<const float*>(smem + Cfg::kG + (g % 3) * tc::GV_BYTES + 512)[row];
+        };
+        auto store_scaled = [&](float cgn) {
+            float z[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) z[j] = cgn * S[j];
+            store_row32_at(sbf + half * Cfg::kSbfHalf, row, c0, z);
+        };
+        store_scaled(ref_scale_of(0));
+        ptx::fence_async_smem();
+        warp_arrive(sbf_ready);
+
+        for (int it = 0; it < nchunks; ++it) {
+            const int s = it & 1;
+            const uint8_t* sbB = smem + Cfg::kB + s * Cfg::kBBytes;
+            const uint32_t d1 = (uint32_t)(it & 1) * 128;
+            const uint32_t par = (uint32_t)it & 1u;
+            if (quad < 2) {   // V_new = U - W S  (token row = row)
+                wait(&fullB[s], (uint32_t)(it >> 1) & 1u, 1);
+                uint4 uq[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    uq[c] = *reinterpret_cast<const uint4*>(sbB + Cfg::kBU + ch * tc::U_BLOCK + tc::u_off(row, c));
+                warp_arrive(&emptyB[s]);
+                const __nv_bfloat16* U = reinterpret_cast<const __nv_bfloat16*>(uq);
+                wait(mma1_bar, par, 2);
+                ptx::tc_fence_after();
+                float x[32];
+                tmem_ld32(tmem_lane + d1, x);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[j] = __bfloat162float(U[j]) - x[j];
+                store_row32_at(vn + half * Cfg::kVnHalf, row, c0, x);
+                ptx::fence_async_smem();
+                ptx::tc_fence_before();
+                warp_arrive(vn_ready);
+            }
+            wait(&fullG[it % 3], (uint32_t)(it / 3) & 1u, 10);
+            const float* gv = reinterpret_cast<const float*>(smem + Cfg::kG + (it % 3) * tc::GV_BYTES);
+            const float gc = gv[row];          // gamma^C
+            const float ct = gv[256 + row];    // exp(G_C - G_m)
+            const float cgn = ref_scale_of(it + 1);   // fetched off the chain, before the wait below
+            warp_arrive(&emptyG[it % 3]);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) S[j] *= gc;
+            wait(mma2_bar, par, 3);
+            ptx::tc_fence_after();
+            {
+                float ds[32];
+                tmem_ld32(tmem_lane + d3, ds);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) S[j] = fmaf(ct, ds[j], S[j]);
+                store_scaled(cgn);   // next chunk's operand copy: bf16(exp(G_m') . S_new)
+                ptx::fence_async_smem();
+                ptx::tc_fence_before();
+                warp_arrive(sbf_ready);
+            }
+            if (quad >= 2 && op) {   // O = (Gamma.Q) S + Aqk V_new  (token row = row - 64)
+                const int i = row - 64;
+                const int64_t tok0 = tok_begin + (cb + it - seq_c0) * kC;
+                const int len = (tok_end - tok0) < kC ? (int)(tok_end - tok0) : kC;
+                __nv_bfloat16* orow = op + ((tok0 + i) * a.H + h) * kD + ch * 32;
+                wait(&out_bar[it & 1], (uint32_t)(it >> 1) & 1u, 6);
+                ptx::tc_fence_after();
+                float ov[32];
+                tmem_ld32(tmem_lane + d1, ov);
+                if (i < len) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8)
+                        *reinterpret_cast<uint4*>(orow + j) =
+                            make_uint4(pack2(ov[j], ov[j + 1]), pack2(ov[j + 2], ov[j + 3]),
+                                       pack2(ov[j + 4], ov[j + 5]), pack2(ov[j + 6], ov[j + 7]));
+                }
+                ptx::tc_fence_before();
+            }
+        }
+        if (*abort_flag == 0) {
+            float* so = a.S_out + sbase;
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(so + j) = make_float4(S[j], S[j + 1], S[j + 2], S[j + 3]);
+        }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) ptx::tmem_dealloc(tmem_base, 512);
+}
+
 template <int NS>
 kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begin, int n_count,
                                WsHeader* hdr, bool after_intra, cudaStream_t st)
@@ -513,6 +827,34 @@ kda_status_t launch_inter_tc_t(const ChunkArgs& a, const char* tiles, int n_begi
         return KDA_OK;
     }
     KDA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kda_inter_tc<NS, false>, a, tiles, n_begin, hdr, tm_g));
+    count_launch();
+    return KDA_OK;
+}
+
+kda_status_t launch_inter_tc_wide(const ChunkArgs& a, const char* tiles, int n_begin, int n_count, WsHeader* hdr,
+                                  bool after_intra, cudaStream_t st)
+{
+    {
+        DeviceLock lk;
+        if (!lk.st) return lk.rc;
+        if (!lk.st->attr_done[9]) {
+            KDA_CUDA_TRY(cudaFuncSetAttribute(kda_inter_tc_wide, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)WideCfg::kSmem));
+            lk.st->attr_done[9] = true;
+        }
+    }
+    ProfScope ps(PROF_INTER, st);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, (unsigned)a.H, (unsigned)n_count);
+    cfg.blockDim = dim3(WideCfg::kThreads);
+    cfg.dynamicSmemBytes = WideCfg::kSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_intra ? 1 : 0;
+    KDA_CUDA_TRY(cudaLaunchKernelEx(&cfg, kda_inter_tc_wide, a, tiles, n_begin, hdr));
     count_launch();
     return KDA_OK;
 }
@@ -586,6 +928,7 @@ bool inter_can_fuse_epilogue(int64_t groups)
 }
 
 size_t tc_tile_bytes() { return tc::TILE_BYTES; }
+void set_inter_wide(bool on) { g_inter_wide = on; }
 
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
                              WsHeader* hdr, bool clear_status, cudaStream_t st)
@@ -610,6 +953,11 @@ kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n
     if (n_count > 65535)
         return fail(KDA_ERR_UNSUPPORTED, "kda_chunk_fwd: more than 65535 sequences in one two-kernel pass "
                     "(use kda_set_chunk_path(2) or fewer sequences per call)");
+    // more chains than SMs: the throughput form (all 128 columns per CTA); not with the fused output
+    // stage.  Decided on the whole call, not on the pass, so that every pass of a call sums in the
+    // same order.
+    if (g_inter_wide && (int64_t)a.n_seqs * a.H > (int64_t)n_sm && a.out_gate == nullptr)
+        return launch_inter_tc_wide(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);
     if ((int64_t)n_count * a.H * 4 > 2 * (int64_t)n_sm)
         return launch_inter_tc_t<64>(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);
     return launch_inter_tc_t<32>(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);

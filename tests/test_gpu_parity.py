@@ -535,3 +535,27 @@ def test_fused_kernel_matches_two_kernel_path(oracle_mod, lens, H):
         check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
     finally:
         K.kda_set_chunk_path(0)
+
+
+def test_many_chains_wide_inter_kernel(oracle_mod):
+    """More (sequence, head) chains than the device has SMs: the inter-chunk stage then runs in its
+    128-columns-per-CTA form.  Against the oracle, with several passes (bit-identical: the form is
+    chosen per call, not per pass), state-only, and without an initial state."""
+    lens = [100, 64, 1, 200, 0, 333]
+    H = 40                                              # 240 chains
+    d = inputs.chunk_inputs(lens, H=H, dtype=torch.bfloat16, seed=51, s0_std=0.02)
+    check_chunk(oracle_mod, d, TOL[K.KDA_BF16])
+    full = run_chunk(d)
+    N, T = len(lens), sum(lens)
+    lo = K.kda_chunk_fwd_min_workspace_bytes(T, N, H, dt=K.KDA_BF16)
+    hi = K.kda_chunk_fwd_workspace_bytes(T, N, H, dt=K.KDA_BF16)
+    try:
+        K.kda_set_chunk_path(1)                         # (a small workspace would otherwise pick the fused kernel)
+        part = run_chunk(d, workspace_bytes=lo + (hi - lo) // 3)
+        state_only = run_chunk(d, want_o=False)
+    finally:
+        K.kda_set_chunk_path(0)
+    assert torch.equal(part[0], full[0]) and torch.equal(part[1], full[1])
+    assert torch.equal(state_only[1], full[1])
+    d0 = inputs.chunk_inputs([700] * 5, H=32, dtype=torch.bfloat16, seed=52, s0_std=0.0)
+    check_chunk(oracle_mod, d0, TOL[K.KDA_BF16])
