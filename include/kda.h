@@ -371,6 +371,14 @@ int kda_selftest_device_table(void);
 int kda_selftest_fused_plan(const int32_t *chunks_per_seq, int n_seqs, int H, int64_t avail_tiles,
                             int n_sm, int64_t out[4]);
 
+/*
+ * Upper bound, in nanoseconds, of every wait inside the tensor-core kernels (on a barrier, a flag or
+ * a peer CTA); a wait that runs out makes its kernel return with KDA_ERR_TIMEOUT in the status word.
+ * Default 1 s; the environment variable KDA_WAIT_LIMIT_MS (1 .. 600000), read once per process,
+ * overrides it.  No counterpart in the paper.
+ */
+uint64_t kda_wait_limit_ns(void);
+
 /* Description of the calling thread's last error ("" if none); static storage, never NULL. */
 const char *kda_last_error(void);
 

@@ -28,6 +28,17 @@ kda_status_t fail(kda_status_t code, const char* fmt, ...)
 }
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+unsigned long long wait_limit_ns()
+{
+    static const unsigned long long v = [] {
+        const char* e = std::getenv("KDA_WAIT_LIMIT_MS");
+        long ms = e ? std::strtol(e, nullptr, 10) : 0;
+        if (ms < 1 || ms > 600000) ms = 1000;
+        return (unsigned long long)ms * 1000000ull;
+    }();
+    return v;
+}
+
 // ---- per-device state -------------------------------------------------------------------------------
 namespace {
 std::mutex g_dev_mu;
@@ -223,6 +234,8 @@ int kda_selftest_fused_plan(const int32_t* chunks_per_seq, int n_seqs, int H, in
     return 0;
 }
 
+uint64_t kda_wait_limit_ns(void) { return wait_limit_ns(); }
+
 kda_status_t kda_set_chunk_path(int mode)
 {
     if (mode < 0 || mode > 2) return fail(KDA_ERR_INVALID_ARG, "kda_set_chunk_path: mode must be 0, 1 or 2");
@@ -381,6 +394,7 @@ kda_status_t chunk_fwd_impl(const void* q, const void* k, const void* v, const f
         f.a.cu_seqlens = cu_seqlens_dev; f.a.chunk_cu = nullptr;
         f.a.n_seqs = n_seqs; f.a.H = H; f.a.total_tokens = total_tokens; f.a.seq_len = seq_len;
         f.a.chunks_per_seq = chunks_per_seq; f.a.g0 = 0; f.a.g1 = total_chunks; f.a.scale = scale;
+        f.a.wait_limit_ns = wait_limit_ns();
         f.ring = wsb + FL.off_ring;
         f.ready = reinterpret_cast<unsigned long long*>(wsb + FL.off_ready);
         f.consumed = reinterpret_cast<unsigned long long*>(wsb + FL.off_consumed);
@@ -428,6 +442,7 @@ kda_status_t chunk_fwd_impl(const void* q, const void* k, const void* v, const f
     a.chunks_per_seq = chunks_per_seq; a.scale = scale;
     a.S_out = state;
     a.gate_rate = lm.rate; a.gate_bias = lm.bias; a.l2_eps = lm.l2_eps;
+    a.wait_limit_ns = wait_limit_ns();
     a.out_gate = lm.out_gate; a.rms_weight = lm.rms_weight; a.rms_eps = lm.rms_eps;
 
     int64_t g0 = 0;

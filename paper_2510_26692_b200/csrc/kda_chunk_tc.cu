@@ -35,7 +35,6 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, boo
 
 namespace {
 
-constexpr uint64_t kWaitLimitNs = 1000000000ull;   // 1 s per wait
 constexpr int kNCtrl = 2;                          // MMA-issuing threads (one per control warp)
 bool g_inter_wide = true;                          // (debug switch) use the 128-column form for large batches
 
@@ -188,7 +187,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
 
     auto wait = [&](uint64_t* bar, uint32_t parity, int where) {
         if (*abort_flag) return;
-        if (!ptx::mbar_wait(bar, parity, kWaitLimitNs)) {
+        if (!ptx::mbar_wait(bar, parity, a.wait_limit_ns)) {
             *abort_flag = 1;
             if (atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = where;
         }
@@ -224,7 +223,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 ptx::st_async_cluster_f32(ptx::map_to_cta(slot, (uint32_t)r), part, ptx::map_to_cta(bar, (uint32_t)r));
             // one thread per CTA and chunk arms the own barrier: the 64 rows of every slice, 4 bytes each
             if (i == 0) ptx::mbar_expect_tx(&ssq_bar[b], NSL * kC * 4);
-            if (!*abort_flag && !ptx::mbar_wait_cluster(&ssq_bar[b], (uint32_t)(it >> 1) & 1u, kWaitLimitNs)) {
+            if (!*abort_flag && !ptx::mbar_wait_cluster(&ssq_bar[b], (uint32_t)(it >> 1) & 1u, a.wait_limit_ns)) {
                 *abort_flag = 1;
                 if (atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = 9;
             }
@@ -354,7 +353,7 @@ kda_inter_tc(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHeader*
                 if (*abort_flag) {
                     // drain the bulk copies still in flight before the shared memory goes away
                     for (int j = (loads_issued > NSTG ? loads_issued - NSTG : 0); j < loads_issued; ++j)
-                        ptx::mbar_wait(&full[j % NSTG], (uint32_t)(j / NSTG) & 1u, kWaitLimitNs);
+                        ptx::mbar_wait(&full[j % NSTG], (uint32_t)(j / NSTG) & 1u, a.wait_limit_ns);
                 }
             }
         }
@@ -569,7 +568,7 @@ kda_inter_tc_wide(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHe
 
     auto wait = [&](uint64_t* bar, uint32_t parity, int where) {
         if (*abort_flag) return;
-        if (!ptx::mbar_wait(bar, parity, kWaitLimitNs)) {
+        if (!ptx::mbar_wait(bar, parity, a.wait_limit_ns)) {
             *abort_flag = 1;
             if (atomicCAS(&hdr->status, 0, (int)KDA_ERR_TIMEOUT) == 0) hdr->where = where;
         }
@@ -604,9 +603,9 @@ kda_inter_tc_wide(ChunkArgs a, const char* __restrict__ tiles, int n_begin, WsHe
                 ++nB;
             }
             if (*abort_flag) {   // drain the copies still in flight before the shared memory goes away
-                for (int j = (nG > 3 ? nG - 3 : 0); j < nG; ++j) ptx::mbar_wait(&fullG[j % 3], (uint32_t)(j / 3) & 1u, kWaitLimitNs / 8);
-                for (int j = (nA > 2 ? nA - 2 : 0); j < nA; ++j) ptx::mbar_wait(&fullA[j & 1], (uint32_t)(j >> 1) & 1u, kWaitLimitNs / 8);
-                for (int j = (nB > 2 ? nB - 2 : 0); j < nB; ++j) ptx::mbar_wait(&fullB[j & 1], (uint32_t)(j >> 1) & 1u, kWaitLimitNs / 8);
+                for (int j = (nG > 3 ? nG - 3 : 0); j < nG; ++j) ptx::mbar_wait(&fullG[j % 3], (uint32_t)(j / 3) & 1u, a.wait_limit_ns / 8);
+                for (int j = (nA > 2 ? nA - 2 : 0); j < nA; ++j) ptx::mbar_wait(&fullA[j & 1], (uint32_t)(j >> 1) & 1u, a.wait_limit_ns / 8);
+                for (int j = (nB > 2 ? nB - 2 : 0); j < nB; ++j) ptx::mbar_wait(&fullB[j & 1], (uint32_t)(j >> 1) & 1u, a.wait_limit_ns / 8);
             }
         }
     } else if (warp == 16) {

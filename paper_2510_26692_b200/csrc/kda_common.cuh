@@ -73,6 +73,9 @@ struct ChunkArgs {
     float l2_eps = 0.f;
     // Output stage of the layer wrap inside the inter-chunk kernel (off when out_gate is nullptr):
     // o is replaced by sigmoid(out_gate) . RMSNorm(o) . rms_weight before it is stored.
+    // Upper bound of every device-side wait of the tensor-core kernels (ns); set from the environment
+    // variable KDA_WAIT_LIMIT_MS by the host entry points (default 1 s).
+    unsigned long long wait_limit_ns = 1000000000ull;
     const void* out_gate = nullptr;     // bf16 [T_total, H, dv]
     const float* rms_weight = nullptr;  // [dv]
     float rms_eps = 0.f;
@@ -178,6 +181,7 @@ size_t tc_tile_bytes();
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
                              WsHeader* hdr, bool clear_status, cudaStream_t st);
 bool inter_can_fuse_epilogue(int64_t groups);
+unsigned long long wait_limit_ns();   // KDA_WAIT_LIMIT_MS (1 .. 600000) in ns, default 1 s
 void set_inter_wide(bool on);
 kda_status_t make_plain_tmap(CUtensorMap* tm, const void* base, int64_t total_tokens, int H, int cols, int rows);
 

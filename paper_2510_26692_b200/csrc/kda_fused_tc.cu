@@ -43,7 +43,6 @@
 namespace kda {
 namespace {
 
-constexpr uint64_t kWaitLimitNs = 1000000000ull;          // 1 s per wait
 constexpr int kThreads = 512;
 constexpr int kEngThreads = 256;
 constexpr int LDT = 68;                                   // padded fp32 row of the 64x64 matrix
@@ -312,7 +311,7 @@ __device__ void wait_slot_free(const FusedArgs& f, const TileDesc& d, const Sche
             if ((uint32_t)(v >> 32) == f.epoch && (uint32_t)v >= d.need) break;
             if (t0 == 0) t0 = ptx::globaltimer_ns();
             if (*abort_word || call_aborted(f)) { *abort_word = 1; return; }
-            if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
+            if (ptx::globaltimer_ns() - t0 > f.a.wait_limit_ns) {
                 *abort_word = 1;
                 report_timeout(f, 20);
                 return;
@@ -556,8 +555,8 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
             const uint64_t now_ = ptx::globaltimer_ns();
         }
 #endif
-        if (!ptx::mbar_wait(bar_k, tma_parity, kWaitLimitNs)) timed_out = true;   // raw k, q have landed
-        if (has_q && !ptx::mbar_wait(bar_q, tma_parity, kWaitLimitNs)) timed_out = true;
+        if (!ptx::mbar_wait(bar_k, tma_parity, f.a.wait_limit_ns)) timed_out = true;   // raw k, q have landed
+        if (has_q && !ptx::mbar_wait(bar_q, tma_parity, f.a.wait_limit_ns)) timed_out = true;
         pend_k = pend_q = false;
         KT_MARK(te == 0, 2);   // prefix + TMA wait
         // ---- gated operands ---------------------------------------------------------------------------
@@ -685,7 +684,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                 next_static += stride;
             }
         }
-        if (!ptx::mbar_wait(mma_bar, 0, kWaitLimitNs)) timed_out = true;
+        if (!ptx::mbar_wait(mma_bar, 0, f.a.wait_limit_ns)) timed_out = true;
         // Q' and K' have been read out of shared memory by now: Aqk goes over the Q' rows next
         if (te == kBulkThread) ptx::bulk_wait_read0();
         ebar();
@@ -803,7 +802,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
             if (has_next && has_q) request_q(Dn);
         }
         if (has_next) pend_q = has_q;
-        if (!ptx::mbar_wait(bar_v, tma_parity, kWaitLimitNs)) timed_out = true;   // v has landed
+        if (!ptx::mbar_wait(bar_v, tma_parity, f.a.wait_limit_ns)) timed_out = true;   // v has landed
         pend_v = false;
         tma_parity ^= 1;
         if (D.len < kC) {   // short last chunk: rows past the end hold other tokens' v; zero them
@@ -866,7 +865,7 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
                                ptx::umma_desc_sw128_mn(v0 + k * 2048, E_V_BLOCK), idesc, k > 0);
             ptx::umma_commit(mma_bar);
         }
-        if (!ptx::mbar_wait(mma_bar, 1, kWaitLimitNs)) timed_out = true;
+        if (!ptx::mbar_wait(mma_bar, 1, f.a.wait_limit_ns)) timed_out = true;
         KT_MARK(te == 0, 7);   // Mm + MMA B
         if (has_next) {   // V and beta are free: the next tile's may land
             if (te == kBulkThread) request_v(Dn);
@@ -940,9 +939,9 @@ __device__ void engine_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_e, i
     // an aborted engine may still have a TMA load in flight (requested for a tile it never started)
     if (te == 0) {
         // tma_parity is the parity of the current / next tile's K and Q loads; V's flips in the Mm phase
-        if (pend_k) ptx::mbar_wait(bar_k, tma_parity, kWaitLimitNs);
-        if (pend_q) ptx::mbar_wait(bar_q, tma_parity, kWaitLimitNs);
-        if (pend_v) ptx::mbar_wait(bar_v, tma_parity, kWaitLimitNs);
+        if (pend_k) ptx::mbar_wait(bar_k, tma_parity, f.a.wait_limit_ns);
+        if (pend_q) ptx::mbar_wait(bar_q, tma_parity, f.a.wait_limit_ns);
+        if (pend_v) ptx::mbar_wait(bar_v, tma_parity, f.a.wait_limit_ns);
     }
     ptx::tc_fence_before();
     ebar();
@@ -1039,7 +1038,7 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
             if ((++spins & 15u) == 0) {
                 if (*abort_flag) return;
                 if (call_aborted(f)) { *abort_flag = 1; return; }
-                if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
+                if (ptx::globaltimer_ns() - t0 > f.a.wait_limit_ns) {
                     *abort_flag = 1;
                     report_timeout(f, where);
                     return;
@@ -1108,7 +1107,7 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                     if (*s_exit && *s_done == published) break;
                     if (t0 == 0) t0 = ptx::globaltimer_ns();
                     if (call_aborted(f)) { *abort_flag = 1; break; }
-                    if (jobs_left && ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
+                    if (jobs_left && ptx::globaltimer_ns() - t0 > f.a.wait_limit_ns) {
                         *abort_flag = 1;
                         report_timeout(f, 30);
                         break;
@@ -1148,7 +1147,7 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                         while (*s_ready <= p) {
                             if (t0 == 0) t0 = ptx::globaltimer_ns();
                             if (*abort_flag) break;
-                            if (ptx::globaltimer_ns() - t0 > 2 * kWaitLimitNs) {   // (the flag thread gives up first)
+                            if (ptx::globaltimer_ns() - t0 > 2 * f.a.wait_limit_ns) {   // (the flag thread gives up first)
                                 *abort_flag = 1;
                                 report_timeout(f, 37);
                                 break;
@@ -1209,11 +1208,11 @@ __device__ void chain_run(const FusedArgs& f, uint8_t* smem, uint32_t tmem_c, in
                 // drain: the copies already requested must land before the shared memory goes away
                 // (bounded waits without the abort short-cut; a completed phase returns at once)
                 for (uint32_t pp = (nG > 3 ? nG - 3 : 0); pp < nG; ++pp)
-                    ptx::mbar_wait(&fullG[pp % 3], (pp / 3) & 1u, kWaitLimitNs / 8);
+                    ptx::mbar_wait(&fullG[pp % 3], (pp / 3) & 1u, f.a.wait_limit_ns / 8);
                 for (uint32_t pp = (nA > 2 ? nA - 2 : 0); pp < nA; ++pp)
-                    ptx::mbar_wait(&fullA[pp & 1], (pp >> 1) & 1u, kWaitLimitNs / 8);
+                    ptx::mbar_wait(&fullA[pp & 1], (pp >> 1) & 1u, f.a.wait_limit_ns / 8);
                 for (uint32_t pp = (nB > 2 ? nB - 2 : 0); pp < nB; ++pp)
-                    ptx::mbar_wait(&fullB[pp & 1], (pp >> 1) & 1u, kWaitLimitNs / 8);
+                    ptx::mbar_wait(&fullB[pp & 1], (pp >> 1) & 1u, f.a.wait_limit_ns / 8);
             }
         }
     } else if (warp == 8 || warp == 9) {

@@ -206,3 +206,18 @@ def test_side_entry_points_reject_bad_arguments(lib):
     assert rc == 1 and "g_o" in K.kda_last_error()
     assert lib.kda_layer_fwd_workspace_bytes(4096, 1, 32, 128, 128, 64) >= \
         lib.kda_layer_fwd_min_workspace_bytes(4096, 1, 32, 128, 128, 64) > 0
+
+
+def test_wait_limit_from_environment(lib):
+    """KDA_WAIT_LIMIT_MS bounds every device-side wait; read once per process, so checked in children."""
+    import subprocess
+    import sys
+    lib.kda_wait_limit_ns.restype = ctypes.c_uint64
+    assert lib.kda_wait_limit_ns() == 1_000_000_000      # (this process: variable not set)
+    code = ("import ctypes; from paper_2510_26692_b200 import api; l = api.load(); "
+            "l.kda_wait_limit_ns.restype = ctypes.c_uint64; print(l.kda_wait_limit_ns())")
+    for val, want in (("250", 250_000_000), ("0", 1_000_000_000), ("junk", 1_000_000_000), ("9999999", 1_000_000_000)):
+        env = dict(os.environ, KDA_WAIT_LIMIT_MS=val)
+        out = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True)
+        assert out.returncode == 0, out.stderr
+        assert int(out.stdout.strip().splitlines()[-1]) == want, (val, out.stdout)
