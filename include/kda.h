@@ -189,6 +189,22 @@ kda_status_t kda_layer_fwd(const void *q_c, const void *k_c, const void *v, cons
                            size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Decode step of the layer wrap: kda_decode_step with the same element-wise stages as kda_layer_fwd
+ * (L2Norm of q_c and k_c, the decay function on g_a, sigmoid on b_pre, head-wise RMSNorm and sigmoid
+ * output gate on the output row) computed inside the decode kernel; one token per sequence.
+ *
+ *   q_c, k_c, g_a [n_seqs,H,dk], v, g_o, y [n_seqs,H,dv]   bf16 device;  b_pre [n_seqs,H] fp32 device
+ *   A_log [H], dt_bias [H,dk], rms_weight [dv]              fp32 device
+ *   S, state_slot, scale                                    as in kda_decode_step (state in place)
+ * Only dk = dv = 128.  Asynchronous on `cuda_stream`; errors as for kda_decode_step.
+ */
+kda_status_t kda_layer_decode_step(const void *q_c, const void *k_c, const void *v, const void *g_a,
+                                   const float *b_pre, const void *g_o, const float *A_log,
+                                   const float *dt_bias, const float *rms_weight, float l2_eps,
+                                   float rms_eps, float *S, const int32_t *state_slot, void *y,
+                                   int n_seqs, int H, int dk, int dv, float scale, void *cuda_stream);
+
+/*
  * Backward pass of kda_chunk_fwd: gradients of Eq. 1 (the operator is trained end to end, Section 5;
  * the paper prints no backward algorithm, so this is the adjoint of Eq. 1 itself).  For
  *

@@ -79,6 +79,8 @@ def load():
     lib.kda_layer_fwd.restype = i32
     lib.kda_layer_fwd.argtypes = [vp] * 9 + [f32, f32, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32,
                                              vp, sz, vp]
+    lib.kda_layer_decode_step.restype = i32
+    lib.kda_layer_decode_step.argtypes = [vp] * 9 + [f32, f32, vp, vp, vp, i32, i32, i32, i32, f32, vp]
     lib.kda_decode_step.restype = i32
     lib.kda_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp]
     lib.kda_decode_multi.restype = i32
@@ -282,6 +284,20 @@ def kda_layer_fwd(q_c, k_c, v, g_a, b_pre, g_o, A_log, dt_bias, rms_weight, l2_e
         _ptr(cu_seqlens_host, False, torch.int32, "cu_seqlens_host"),
         int(n_seqs), int(total_tokens), int(H), int(dk), int(dv), int(chunk), float(scale),
         _ptr(workspace, True, None, "workspace"), int(workspace_bytes), _stream(stream))
+    _check(rc)
+
+
+def kda_layer_decode_step(q_c, k_c, v, g_a, b_pre, g_o, A_log, dt_bias, rms_weight, l2_eps, rms_eps, S,
+                          state_slot, y, n_seqs, H, dk, dv, scale, stream=None):
+    """``kda_layer_decode_step`` of ``include/kda.h``: one decode token per sequence with the layer's
+    element-wise stages inside the kernel (bf16 activations, fp32 state in place)."""
+    f32, bf = torch.float32, torch.bfloat16
+    rc = load().kda_layer_decode_step(
+        _ptr(q_c, True, bf, "q_c"), _ptr(k_c, True, bf, "k_c"), _ptr(v, True, bf, "v"), _ptr(g_a, True, bf, "g_a"),
+        _ptr(b_pre, True, f32, "b_pre"), _ptr(g_o, True, bf, "g_o"), _ptr(A_log, True, f32, "A_log"),
+        _ptr(dt_bias, True, f32, "dt_bias"), _ptr(rms_weight, True, f32, "rms_weight"), float(l2_eps),
+        float(rms_eps), _ptr(S, True, f32, "S"), _ptr(state_slot, True, torch.int32, "state_slot"),
+        _ptr(y, True, bf, "y"), int(n_seqs), int(H), int(dk), int(dv), float(scale), _stream(stream))
     _check(rc)
 
 

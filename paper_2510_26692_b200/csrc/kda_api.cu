@@ -558,6 +558,28 @@ kda_status_t kda_decode_step(const void* q, const void* k, const void* v, const 
                          static_cast<cudaStream_t>(cuda_stream));
 }
 
+kda_status_t kda_layer_decode_step(const void* q_c, const void* k_c, const void* v, const void* g_a,
+                                   const float* b_pre, const void* g_o, const float* A_log,
+                                   const float* dt_bias, const float* rms_weight, float l2_eps, float rms_eps,
+                                   float* S, const int32_t* state_slot, void* y, int n_seqs, int H, int dk,
+                                   int dv, float scale, void* cuda_stream)
+{
+    if (dk != kD || dv != kD)
+        return fail(KDA_ERR_UNSUPPORTED, "kda_layer_decode_step: only dk=dv=128 is supported (got dk=%d dv=%d)",
+                    dk, dv);
+    if (n_seqs < 0 || H <= 0 || (int64_t)n_seqs * H > 0x7fffffff)
+        return fail(KDA_ERR_INVALID_ARG, "kda_layer_decode_step: bad sizes n_seqs=%d H=%d", n_seqs, H);
+    if (n_seqs == 0) return KDA_OK;
+    if (!q_c || !k_c || !v || !g_a || !b_pre || !g_o || !A_log || !dt_bias || !rms_weight || !S || !y)
+        return fail(KDA_ERR_INVALID_ARG, "kda_layer_decode_step: NULL pointer argument");
+    const void* ptrs[] = {q_c, k_c, v, g_a, b_pre, g_o, A_log, dt_bias, rms_weight, S, y, state_slot};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return fail(KDA_ERR_INVALID_ARG, "kda_layer_decode_step: pointer %p is not "
+                                       "16-byte aligned", p);
+    return launch_layer_decode(q_c, k_c, v, g_a, b_pre, g_o, A_log, dt_bias, rms_weight, l2_eps, rms_eps, S,
+                               state_slot, y, n_seqs, H, scale, static_cast<cudaStream_t>(cuda_stream));
+}
+
 kda_status_t kda_decode_multi(const void* q, const void* k, const void* v, const float* log_alpha,
                               const float* beta, float* S, const int32_t* state_slot, void* o,
                               int n_seqs, int n_tokens, int H, int dk, int dv, float scale,

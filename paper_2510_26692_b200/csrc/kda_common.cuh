@@ -167,6 +167,11 @@ kda_status_t launch_decode(const void* q, const void* k, const void* v, const fl
                            const float* beta, float* S, const int32_t* slot, void* o, int n_seqs,
                            int H, float scale, kda_dtype_t dt, cudaStream_t st);
 
+kda_status_t launch_layer_decode(const void* q_c, const void* k_c, const void* v, const void* g_a,
+                                 const float* b_pre, const void* g_o, const float* A_log, const float* dt_bias,
+                                 const float* rms_weight, float l2_eps, float rms_eps, float* S,
+                                 const int32_t* slot, void* y, int n_seqs, int H, float scale, cudaStream_t st);
+
 kda_status_t launch_decode_multi(const void* q, const void* k, const void* v, const float* log_alpha,
                                  const float* beta, float* S, const int32_t* slot, void* o, int n_seqs,
                                  int n_tok, int H, float scale, kda_dtype_t dt, cudaStream_t st);

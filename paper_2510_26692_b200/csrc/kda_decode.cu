@@ -45,11 +45,24 @@ template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 x
     return __bfloat162float(x);
 }
 
-template <typename T>
+// Layer mode (kda_layer_decode_step, paper Section 4 "Neural Parameterization"): q and k arrive
+// un-normalised, `log_alpha` points to the bf16 pre-activations of the decay function, `beta` to the
+// pre-activations of beta, and the output row goes through the head-wise RMSNorm and the sigmoid
+// output gate before it is stored.  All of it is arithmetic on 128-vectors beside a 64 KiB state
+// stream: free at the HBM bound.
+struct DecodeLayer {
+    const float* A_log;        // [H]
+    const float* dt_bias;      // [H, dk]
+    const void* g_o;           // bf16 [n_seqs, H, dv]
+    const float* rms_weight;   // [dv]
+    float l2_eps, rms_eps;
+};
+
+template <typename T, bool kLayer>
 __global__ void __launch_bounds__(256, 2)
 kda_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                   const float* __restrict__ log_alpha, const float* __restrict__ beta, float* S,
-                  const int32_t* __restrict__ slot, T* __restrict__ o, int H, float scale)
+                  const int32_t* __restrict__ slot, T* __restrict__ o, int H, float scale, DecodeLayer lay)
 {
     __shared__ float s_a[kD], s_k[kD], s_q[kD];
     __shared__ float4 s_red[2][8][32];
@@ -65,24 +78,46 @@ kda_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
 
     const size_t vec = (size_t)item * kD;
     if (t < kD) {
-        s_a[t] = expf(log_alpha[vec + t]);
+        if (kLayer) {
+            const float z = to_f<T>(reinterpret_cast<const T*>(log_alpha)[vec + t]) + lay.dt_bias[(size_t)h * kD + t];
+            const float sp = fmaxf(z, 0.f) + log1pf(expf(-fabsf(z)));
+            s_a[t] = expf(-expf(lay.A_log[h]) * sp);
+        } else {
+            s_a[t] = expf(log_alpha[vec + t]);
+        }
         s_k[t] = to_f<T>(k[vec + t]);
         s_q[t] = to_f<T>(q[vec + t]);
     }
     __syncthreads();
 
-    // q.k, redundantly per warp (4 rows per lane, butterfly reduce)
-    float qk = 0.f;
+    // q.k, redundantly per warp (4 rows per lane, butterfly reduce); layer mode: the norms as well
+    float qk = 0.f, ssk = 0.f, ssq = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) qk += s_q[lane * 4 + i] * s_k[lane * 4 + i];
+    for (int i = 0; i < 4; ++i) {
+        const float kv = s_k[lane * 4 + i], qv = s_q[lane * 4 + i];
+        qk += qv * kv;
+        if (kLayer) {
+            ssk += kv * kv;
+            ssq += qv * qv;
+        }
+    }
 #pragma unroll
-    for (int ofs = 16; ofs > 0; ofs >>= 1) qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
+    for (int ofs = 16; ofs > 0; ofs >>= 1) {
+        qk += __shfl_xor_sync(0xffffffffu, qk, ofs);
+        if (kLayer) {
+            ssk += __shfl_xor_sync(0xffffffffu, ssk, ofs);
+            ssq += __shfl_xor_sync(0xffffffffu, ssq, ofs);
+        }
+    }
+    const float rk = kLayer ? rsqrtf(ssk + lay.l2_eps) : 1.f;   // 1 / |k|, 1 / |q| (L2Norm)
+    const float rq = kLayer ? rsqrtf(ssq + lay.l2_eps) : 1.f;
+    if (kLayer) qk *= rk * rq;
 
     float4 p = make_float4(0.f, 0.f, 0.f, 0.f), s = p;
 #pragma unroll
     for (int m = 0; m < 16; ++m) {
         const int row = warp + 8 * m;
-        const float a = s_a[row], kk = s_k[row], qq = s_q[row];
+        const float a = s_a[row], kk = kLayer ? s_k[row] * rk : s_k[row], qq = kLayer ? s_q[row] * rq : s_q[row];
         x[m].x *= a; x[m].y *= a; x[m].z *= a; x[m].w *= a;
         p.x += kk * x[m].x; p.y += kk * x[m].y; p.z += kk * x[m].z; p.w += kk * x[m].w;
         s.x += qq * x[m].x; s.y += qq * x[m].y; s.z += qq * x[m].z; s.w += qq * x[m].w;
@@ -98,19 +133,31 @@ kda_decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __r
         p.x += a.x; p.y += a.y; p.z += a.z; p.w += a.w;
         s.x += b.x; s.y += b.y; s.z += b.z; s.w += b.w;
     }
-    const float bt = beta[item];
+    const float bt = kLayer ? 1.f / (1.f + expf(-beta[item])) : beta[item];
     float4 vv = IO<T>::load4(v + vec + lane * 4);
     float4 r = make_float4(vv.x - p.x, vv.y - p.y, vv.z - p.z, vv.w - p.w);
     if (warp == 0) {
         const float c = bt * qk;
         float4 ov = make_float4(scale * (s.x + c * r.x), scale * (s.y + c * r.y),
                                 scale * (s.z + c * r.z), scale * (s.w + c * r.w));
+        if (kLayer) {   // head-wise RMSNorm over the 128 values of the row (4 per lane), weight, sigmoid gate
+            float ss = ov.x * ov.x + ov.y * ov.y + ov.z * ov.z + ov.w * ov.w;
+#pragma unroll
+            for (int ofs = 16; ofs > 0; ofs >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, ofs);
+            const float rstd = rsqrtf(ss * (1.f / kD) + lay.rms_eps);
+            const float4 w4 = *reinterpret_cast<const float4*>(lay.rms_weight + lane * 4);
+            const float4 g4 = IO<T>::load4(reinterpret_cast<const T*>(lay.g_o) + vec + lane * 4);
+            ov.x *= rstd * w4.x / (1.f + expf(-g4.x));
+            ov.y *= rstd * w4.y / (1.f + expf(-g4.y));
+            ov.z *= rstd * w4.z / (1.f + expf(-g4.z));
+            ov.w *= rstd * w4.w / (1.f + expf(-g4.w));
+        }
         IO<T>::store4(o + vec + lane * 4, ov);
     }
 #pragma unroll
     for (int m = 0; m < 16; ++m) {
         const int row = warp + 8 * m;
-        const float c = bt * s_k[row];
+        const float c = kLayer ? bt * s_k[row] * rk : bt * s_k[row];
         x[m].x += c * r.x; x[m].y += c * r.y; x[m].z += c * r.z; x[m].w += c * r.w;
         st_stream(Sp + (size_t)row * kD, x[m]);
     }
@@ -328,13 +375,33 @@ kda_status_t launch_decode(const void* q, const void* k, const void* v, const fl
     ProfScope ps(PROF_DECODE, st);
     if (dt == KDA_BF16) {
         using T = __nv_bfloat16;
-        kda_decode_kernel<T><<<grid, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v,
-                                                   log_alpha, beta, S, slot, (T*)o, H, scale);
+        kda_decode_kernel<T, false><<<grid, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v,
+                                                          log_alpha, beta, S, slot, (T*)o, H, scale, DecodeLayer());
     } else {
-        kda_decode_kernel<float><<<grid, 256, 0, st>>>((const float*)q, (const float*)k,
-                                                       (const float*)v, log_alpha, beta, S, slot,
-                                                       (float*)o, H, scale);
+        kda_decode_kernel<float, false><<<grid, 256, 0, st>>>((const float*)q, (const float*)k,
+                                                              (const float*)v, log_alpha, beta, S, slot,
+                                                              (float*)o, H, scale, DecodeLayer());
     }
+    count_launch();
+    KDA_CUDA_TRY(cudaGetLastError());
+    return KDA_OK;
+}
+
+kda_status_t launch_layer_decode(const void* q_c, const void* k_c, const void* v, const void* g_a,
+                                 const float* b_pre, const void* g_o, const float* A_log, const float* dt_bias,
+                                 const float* rms_weight, float l2_eps, float rms_eps, float* S,
+                                 const int32_t* slot, void* y, int n_seqs, int H, float scale, cudaStream_t st)
+{
+    if (n_seqs == 0) return KDA_OK;
+    using T = __nv_bfloat16;
+    DecodeLayer lay;
+    lay.A_log = A_log; lay.dt_bias = dt_bias; lay.g_o = g_o; lay.rms_weight = rms_weight;
+    lay.l2_eps = l2_eps; lay.rms_eps = rms_eps;
+    const unsigned grid = (unsigned)((size_t)n_seqs * H);
+    ProfScope ps(PROF_DECODE, st);
+    kda_decode_kernel<T, true><<<grid, 256, 0, st>>>((const T*)q_c, (const T*)k_c, (const T*)v,
+                                                     reinterpret_cast<const float*>(g_a), b_pre, S, slot, (T*)y, H,
+                                                     scale, lay);
     count_launch();
     KDA_CUDA_TRY(cudaGetLastError());
     return KDA_OK;

@@ -108,3 +108,45 @@ def test_layer_output_stage_fused_and_separate_agree(oracle_mod):
         print("output stage", lens, H, "separate", e_sep, "fused", e_fus)
         assert e_sep <= TOL and e_fus <= TOL
         assert rel_l2(to_np32(y_fus), to_np32(y_sep)) <= 1e-2
+
+
+def test_layer_decode_step_matches_oracle(oracle_mod):
+    """One decode token per sequence with the layer's element-wise stages inside the kernel: against the
+    layer oracle's inputs -> oracle.decode_step -> output gate, two steps in place, with slot
+    indirection.  Tolerance 2e-2 on the bf16 output row, 1e-4 on the fp32 state (fp32 arithmetic on
+    bf16 inputs; the only reduced precision is the stored output)."""
+    N, H = 5, 3
+    dev = "cuda:0"
+    g = torch.Generator().manual_seed(77)
+    A_log = torch.randn((H,), generator=g) * 0.3
+    dt_bias = torch.randn((H, 128), generator=g) * 0.3
+    w = 1 + 0.1 * torch.randn((128,), generator=g)
+    n_slots = 9
+    slot = torch.tensor([7, 0, 3, 8, 2], dtype=torch.int32)
+    S = (torch.randn((n_slots, H, 128, 128), generator=g) * 0.05)
+    S_dev = S.clone().to(dev)
+    S_ref = S.double().numpy().copy()
+    for step in range(2):
+        bf = torch.bfloat16
+        q_c = (torch.randn((N, H, 128), generator=g) * 2).to(bf)
+        k_c = (torch.randn((N, H, 128), generator=g) * 0.7).to(bf)
+        v = torch.randn((N, H, 128), generator=g).to(bf)
+        g_a = (torch.randn((N, H, 128), generator=g) - 3).to(bf)
+        b_pre = torch.randn((N, H), generator=g)
+        g_o = torch.randn((N, H, 128), generator=g).to(bf)
+        y = torch.full((N, H, 128), float("nan"), dtype=bf, device=dev)
+        K.kda_layer_decode_step(q_c.to(dev), k_c.to(dev), v.to(dev), g_a.to(dev), b_pre.to(dev), g_o.to(dev),
+                                A_log.to(dev), dt_bias.to(dev), w.to(dev), 1e-6, 1e-5, S_dev, slot.to(dev), y, N, H,
+                                128, 128, 128 ** -0.5)
+        torch.cuda.synchronize()
+        q, k, la, beta = layer_oracle.layer_inputs(q_c.float().numpy(), k_c.float().numpy(), g_a.float().numpy(),
+                                                   b_pre.numpy(), A_log.numpy(), dt_bias.numpy(), 1e-6)
+        o_ref = oracle_mod.decode_step(q.astype(np.float32), k.astype(np.float32), v.float().numpy(),
+                                       la.astype(np.float32), beta.astype(np.float32), S_ref,
+                                       state_slot=slot.numpy(), scale=128 ** -0.5)
+        y_ref = layer_oracle.output_gate(o_ref, g_o.float().numpy(), w.numpy(), 1e-5)
+        ey = rel_l2(to_np32(y), y_ref)
+        es = rel_l2(to_np32(S_dev), S_ref)
+        print("layer decode step", step, ey, es)
+        assert torch.isfinite(y.float()).all()
+        assert ey <= TOL and es <= 1e-4
