@@ -36,7 +36,6 @@ kda_status_t launch_intra_tc(const ChunkArgs& a, void* tiles, WsHeader* hdr, boo
 namespace {
 
 constexpr int kNCtrl = 2;                          // MMA-issuing threads (one per control warp)
-bool g_inter_wide = true;                          // (debug switch) use the 128-column form for large batches
 
 template <int NS> struct InterCfg {
     static_assert(NS == 32 || NS == 64, "state columns per CTA: one or two 32-column blocks");
@@ -927,7 +926,6 @@ bool inter_can_fuse_epilogue(int64_t groups)
 }
 
 size_t tc_tile_bytes() { return tc::TILE_BYTES; }
-void set_inter_wide(bool on) { g_inter_wide = on; }
 
 kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n_count,
                              WsHeader* hdr, bool clear_status, cudaStream_t st)
@@ -955,7 +953,7 @@ kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n
     // more chains than SMs: the throughput form (all 128 columns per CTA); not with the fused output
     // stage.  Decided on the whole call, not on the pass, so that every pass of a call sums in the
     // same order.
-    if (g_inter_wide && (int64_t)a.n_seqs * a.H > (int64_t)n_sm && a.out_gate == nullptr)
+    if ((int64_t)a.n_seqs * a.H > (int64_t)n_sm && a.out_gate == nullptr)
         return launch_inter_tc_wide(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);
     if ((int64_t)n_count * a.H * 4 > 2 * (int64_t)n_sm)
         return launch_inter_tc_t<64>(a, (const char*)tiles, n_begin, n_count, hdr, a.g1 > a.g0, st);

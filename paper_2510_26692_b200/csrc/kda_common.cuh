@@ -187,7 +187,6 @@ kda_status_t launch_chunk_tc(const ChunkArgs& a, void* tiles, int n_begin, int n
                              WsHeader* hdr, bool clear_status, cudaStream_t st);
 bool inter_can_fuse_epilogue(int64_t groups);
 unsigned long long wait_limit_ns();   // KDA_WAIT_LIMIT_MS (1 .. 600000) in ns, default 1 s
-void set_inter_wide(bool on);
 kda_status_t make_plain_tmap(CUtensorMap* tm, const void* base, int64_t total_tokens, int H, int cols, int rows);
 
 // fused bf16 path: workspace bytes besides the ring (flags and round table), and the launcher
