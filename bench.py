@@ -360,7 +360,7 @@ def layer_figure(K, inputs, torch, dev, peaks):
     return {"workload": "B=1 T=4096 H=32, bf16 pre-activations (q_c, k_c, v, g_a, g_o), fp32 b_pre; inputs rotate over 3 copies",
             "ms": ms, "tokens_per_s": T / (ms * 1e-3), "algorithmic_bytes": nbytes,
             "achieved_gbs": nbytes / (ms * 1e-3) / 1e9, "frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-            "note": "three kernels per call: intra-chunk (with the prologue), inter-chunk, output stage"}
+            "note": "two kernels per call: intra-chunk with the prologue inside, inter-chunk with the output stage inside (clusters of the four slice CTAs)"}
 
 
 def decode_only(args, K, inputs, torch, dev, peaks):

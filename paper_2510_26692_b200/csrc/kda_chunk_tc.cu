@@ -883,12 +883,13 @@ kda_status_t launch_wait_selftest(WsHeader* hdr, uint64_t limit_ns, cudaStream_t
 }
 
 namespace {
-bool clusters_fit(int64_t groups, int n_sm)
+// resident clusters of the four slice CTAs of kda_inter_tc<32, true> on the current device
+int query_max_clusters()
 {
     using Cfg = InterCfg<32>;
     if (cudaFuncSetAttribute(kda_inter_tc<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)Cfg::kSmem) != cudaSuccess)
-        return false;
+        return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kD / 32, 1, 1);
     cfg.blockDim = dim3(384);
@@ -903,26 +904,32 @@ bool clusters_fit(int64_t groups, int n_sm)
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kda_inter_tc<32, true>, &cfg) != cudaSuccess) {
         (void)cudaGetLastError();
-        return false;
+        return 0;
     }
-    const int64_t plain = n_sm / (kD / 32);   // groups of slice CTAs that a launch without clusters holds
-    return n >= (groups < plain ? groups : plain);
+    return n;
 }
 }  // namespace
 
 // Whether the output stage of the layer wrap can run inside the inter-chunk kernel for a call with
 // `groups` (sequence, head) pairs: its slice CTAs then form clusters, and a GPC holds fewer clusters
 // than its SM count suggests; if the device cannot keep as many (sequence, head) pairs in flight as
-// without clusters, or the call is large enough for 64-column slices, the stage runs as a separate
-// pass instead.
+// without clusters, or the call is large enough for wider slices, the stage runs as a separate pass
+// instead.  The device's answer is asked once and kept in its slot of the per-device table.
 bool inter_can_fuse_epilogue(int64_t groups)
 {
-    int n_sm = 0, dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-        return false;
-    if (groups * 4 > 2 * (int64_t)n_sm) return false;   // the launcher picks 64-column slices there
-    return clusters_fit(groups, n_sm);
+    DeviceLock lk;
+    if (!lk.st) return false;
+    if (lk.st->n_sm == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&lk.st->n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return false;
+    }
+    const int n_sm = lk.st->n_sm;
+    if (groups * 4 > 2 * (int64_t)n_sm) return false;   // the launcher picks wider slices there
+    if (lk.st->max_clusters < 0) lk.st->max_clusters = query_max_clusters();
+    const int64_t plain = n_sm / (kD / 32);   // groups of slice CTAs that a launch without clusters holds
+    return lk.st->max_clusters >= (groups < plain ? groups : plain);
 }
 
 size_t tc_tile_bytes() { return tc::TILE_BYTES; }

@@ -207,6 +207,7 @@ struct DeviceState {
     int n_sm = 0;
     bool attr_done[kAttrSlots] = {};
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    int max_clusters = -1;   // resident 4-CTA clusters of the inter-chunk kernel with the output stage (-1: not asked yet)
 };
 // Locks the table and returns the slot of the calling thread's current device (nullptr + error set
 // on failure); the lock is released by ~DeviceLock.
